@@ -1,0 +1,90 @@
+"""Pins for the oracle's top-k selection (Eq. 11) and decode keep decision (Eq. 5 / 6)."""
+import itertools
+
+import numpy as np
+import pytest
+
+from oracle import dl_oracle as orc
+from paper_2412_00876_b200 import workloads as wl
+
+
+def brute_topk(s, k):
+    s = [(-np.inf if (x != x) else float(x)) for x in s]
+    order = sorted(range(len(s)), key=lambda i: (-s[i], i))
+    return sorted(order[:k])
+
+
+def test_matches_brute_force_sort_on_tiny_inputs():
+    rng = np.random.default_rng(0)
+    for n in range(0, 9):
+        for trial in range(20):
+            # few distinct values => many ties
+            s = rng.integers(-2, 3, size=n).astype(np.float32)
+            for k in range(n + 1):
+                idx, keep = orc.topk_select(s, k)
+                assert list(idx) == brute_topk(s, k)
+                assert keep.sum() == k and len(idx) == k
+                assert all(keep[i] == 1 for i in idx)
+
+
+def test_all_orderings_of_distinct_values():
+    vals = [0.5, -1.0, 3.0, 2.0, -0.25]
+    for perm in itertools.permutations(vals):
+        for k in range(6):
+            idx, _ = orc.topk_select(np.array(perm), k)
+            top = sorted(vals, reverse=True)[:k]
+            assert sorted(perm[i] for i in idx) == sorted(top)
+            assert list(idx) == sorted(idx)
+
+
+def test_order_property_and_ascending_output():
+    rng = np.random.default_rng(5)
+    s = np.round(rng.normal(size=300), 1)
+    for k in (0, 1, 75, 299, 300):
+        idx, keep = orc.topk_select(s, k)
+        assert np.all(np.diff(idx) > 0)
+        kept, dropped = np.flatnonzero(keep == 1), np.flatnonzero(keep == 0)
+        for i in kept:
+            for j in dropped:
+                assert s[i] > s[j] or (s[i] == s[j] and i < j)
+
+
+def test_degenerate_cases():
+    idx, keep = orc.topk_select(np.ones(10), 4)           # all equal: lowest indices win
+    assert list(idx) == [0, 1, 2, 3]
+    idx, _ = orc.topk_select(np.array([0.0, -0.0, 0.0, -0.0]), 2)   # -0 == +0: a tie
+    assert list(idx) == [0, 1]
+    idx, _ = orc.topk_select(np.array([-0.0, 0.0, -1.0]), 1)
+    assert list(idx) == [0]
+    idx, _ = orc.topk_select(np.array([np.nan, -np.inf, 1.0, np.nan]), 3)   # NaN ranks as -inf
+    assert list(idx) == [0, 1, 2]
+    idx, _ = orc.topk_select(np.array([np.inf, 1.0, np.inf]), 2)
+    assert list(idx) == [0, 2]
+    assert orc.topk_select(np.arange(5.0), 0)[1].sum() == 0
+    assert orc.topk_select(np.arange(5.0), 5)[1].sum() == 5
+    with pytest.raises(ValueError):
+        orc.topk_select(np.arange(5.0), 6)
+
+
+def test_batch_form_respects_ragged_lengths():
+    rng = np.random.default_rng(6)
+    score = rng.normal(size=(3, 12)).astype(np.float32)
+    score[1, 8:] = 100.0           # padding slots with huge scores must never be selected
+    n_vis, k = np.array([12, 8, 5]), np.array([3, 8, 0])
+    kept_idx, keep = orc.prefill_select(score, n_vis, k)
+    assert kept_idx.shape == (3, 8)
+    assert list(kept_idx[0, :3]) == brute_topk(score[0], 3) and np.all(kept_idx[0, 3:] == -1)
+    assert list(kept_idx[1]) == list(range(8)) and keep[1, 8:].sum() == 0
+    assert np.all(kept_idx[2] == -1) and keep[2].sum() == 0
+    assert list(keep.sum(axis=1)) == [3, 8, 0]
+
+
+def test_decode_keep_counts_positive_logits():
+    z = np.array([0.3, -0.1, 0.0, -0.0, 1e-30, -1e-30, np.nan, np.inf, -np.inf])
+    m = orc.decode_keep(z)
+    assert list(m) == [1, 0, 0, 0, 1, 0, 0, 1, 0]          # strict '>' ; NaN drops
+    assert m.sum() == sum(1 for v in z if v > 0)
+    assert list(orc.decode_keep(np.array([0.5, 1.5]), threshold=1.0)) == [0, 1]
+    # alternating-sign logits reproduce the paper's "Structure" static mask (every other token)
+    alt = np.where(np.arange(10) % 2 == 0, 1.0, -1.0)
+    assert list(orc.decode_keep(alt)) == list(wl.static_keep_pattern("structure", 10))
