@@ -1,0 +1,205 @@
+/*
+ * dl.h -- C ABI of the Dynamic-LLaVA sparsified-inference hot path for NVIDIA B200 (sm_100a).
+ *
+ * The calls follow the method's statement in the paper (arXiv 2412.00876):
+ *   prefill  (Eq. 5, Eq. 11): a predictor scores every vision token, the k best are kept,
+ *            the kept rows plus all text rows form the reduced set S^{P*}, and every later
+ *            layer attends over that reduced set only (Eq. 1 on S^{P*});
+ *   decoding with KV cache (Eq. 6): the current token always takes part in its own attention,
+ *            and its K/V are appended to the cache only if the predictor's decision is 1;
+ *            the decision is taken once per token and shared by all later layers (Sec. 3.3.1).
+ *
+ * Conventions
+ *   - Plain C.  Every call returns an int32_t status: DL_OK (0) or a negative DL_ERR_*.
+ *   - "dev" pointers are device memory owned by the caller; "host" pointers are host memory.
+ *     The library allocates no device memory: scratch comes from the caller (dl_set_workspace).
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     unless stated otherwise.  One context serves one stream at a time.
+ *   - Tensors are dense, innermost dimension contiguous, every tensor pointer 16-byte aligned.
+ *     Element type `dtype` (DL_F32 or DL_BF16) applies to activations, Q/K/V, caches, outputs
+ *     and W1; scores, logits, b1, w2 are always float32.
+ *   - Cache layout (what compaction is judged on, bit for bit): per layer, K and V are separate
+ *     tensors [B][H][cap][D], D contiguous.  Rows [0, cache_len[b]) of sequence b are valid;
+ *     rows beyond are unspecified.
+ *   - Errors found on the device (capacity overflow, NaN score) are recorded in a status word
+ *     inside the workspace; dl_device_status reads it back.  Nothing traps.
+ */
+#ifndef DL_SPARSE_H_
+#define DL_SPARSE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dl_ctx dl_ctx;
+
+enum { DL_F32 = 0, DL_BF16 = 1 };
+
+enum {
+  DL_OK = 0,
+  DL_ERR_INVALID_ARG = -1,   /* NULL pointer, negative size, k out of range, ... */
+  DL_ERR_ALIGNMENT = -2,     /* a tensor pointer is not 16-byte aligned */
+  DL_ERR_UNSUPPORTED = -3,   /* dtype / head_dim / size combination not built */
+  DL_ERR_WORKSPACE = -4,     /* workspace missing or too small for this call */
+  DL_ERR_CUDA = -5,          /* a CUDA runtime call failed (see dl_last_cuda_error) */
+  DL_ERR_CAPACITY = -6,      /* device status: kept rows did not fit into the cache */
+  DL_ERR_TIMEOUT = -7,       /* device status: a bounded wait ran out */
+  DL_WARN_NAN = 1            /* device status: a NaN score was ranked as -inf / dropped */
+};
+
+/* Implementation selectors for dl_set_option. */
+enum {
+  DL_OPT_PREDICTOR_IMPL = 1,    /* 0 auto, 1 CUDA-core kernel, 2 tcgen05 tensor-core kernel (bf16) */
+  DL_OPT_PREFILL_ATTN_IMPL = 2, /* 0 auto, 1 CUDA-core kernel, 2 tcgen05 tensor-core kernel (bf16, D=128) */
+  DL_OPT_DECODE_CHUNK = 3       /* cache rows per decode work item (0 = default) */
+};
+
+typedef struct {
+  int32_t hidden;      /* d: width of the hidden rows fed to the predictors */
+  int32_t n_heads;     /* H (multi-head attention: as many K/V heads as query heads) */
+  int32_t head_dim;    /* D: 64 or 128 */
+  int32_t pred_hidden; /* width of the predictor's hidden layer */
+  int32_t dtype;       /* DL_F32 or DL_BF16 */
+} dl_model_desc;
+
+/* One token predictor in per-token MLP form: score = w2 . GELU(W1 x + b1) + b2, GELU in its
+ * exact erf form.  With a single output the score is at once the ranking value of Eq. 11 and
+ * the folded two-way decision of Eq. 5 (keep iff score > 0). */
+typedef struct {
+  const void* w1;   /* dev [pred_hidden][hidden], dtype */
+  const float* b1;  /* dev [pred_hidden] */
+  const float* w2;  /* dev [pred_hidden] */
+  float b2;
+} dl_predictor;
+
+/* ---- context ------------------------------------------------------------------------- */
+
+/* Creates a context for `device` and `desc` (copied).  Host call; may initialise the CUDA
+ * context.  DL_ERR_UNSUPPORTED for head_dim not in {64,128}, hidden % 8 != 0 or unknown dtype. */
+int32_t dl_create(dl_ctx** out, int32_t device, const dl_model_desc* desc);
+int32_t dl_destroy(dl_ctx* ctx);
+
+/* Bytes of scratch the calls below need for up to `max_batch` sequences, `max_rows` predictor
+ * rows per call (B * n_vis_max in prefill) and caches of `cap` rows.  Negative on bad args. */
+int64_t dl_workspace_bytes(const dl_ctx* ctx, int32_t max_batch, int32_t max_rows, int32_t cap);
+
+/* Hands the context its scratch (dev, 256-byte aligned, caller keeps ownership) and clears the
+ * part that must start at zero (asynchronously on `stream`).  The sizes are the ones that were
+ * given to dl_workspace_bytes. */
+int32_t dl_set_workspace(dl_ctx* ctx, void* dev_ptr, int64_t bytes, int32_t max_batch,
+                         int32_t max_rows, int32_t cap, void* stream);
+
+int32_t dl_set_option(dl_ctx* ctx, int32_t option, int32_t value);
+
+/* Synchronises `stream`, copies the device status word back and clears it.  code_out gets
+ * DL_OK, DL_ERR_CAPACITY, DL_ERR_TIMEOUT or DL_WARN_NAN; detail_out the sequence index or row. */
+int32_t dl_device_status(dl_ctx* ctx, void* stream, int32_t* code_out, int64_t* detail_out);
+
+const char* dl_status_str(int32_t status);
+/* Text of the last CUDA error seen by this context (host string owned by the library). */
+const char* dl_last_cuda_error(const dl_ctx* ctx);
+
+/* ---- prefill: Eq. 5 / Eq. 11 --------------------------------------------------------- */
+
+/* Predictor alone (first line of Eq. 5 / Eq. 11): score_out[r] for `rows` hidden rows.
+ * x dev [rows][hidden] dtype; score_out dev [rows] float32. */
+int32_t dl_predictor_scores(dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows,
+                            float* score_out, void* stream);
+
+/* TopkArgmax_k of Eq. 11 on given scores.  For each sequence b the k[b] largest of its first
+ * n_vis[b] scores are kept; between equal scores the lower index wins; -0 equals +0; NaN ranks
+ * as -inf (and sets DL_WARN_NAN).
+ *   score dev [B][n_vis_max]; n_vis dev [B] or NULL (= n_vis_max); k dev [B], 0 <= k[b] <= n_vis[b]
+ *   (a larger k[b] is clamped to n_vis[b]); kept_idx_out dev [B][k_max] ascending, unused slots -1
+ *   (may be NULL); keep_out dev [B][n_vis_max] 0/1 (padding slots 0).  n_vis_max <= 16384. */
+int32_t dl_topk_from_scores(dl_ctx* ctx, const float* score, const int32_t* n_vis, const int32_t* k,
+                            int32_t B, int32_t n_vis_max, int32_t* kept_idx_out, int32_t k_max,
+                            uint8_t* keep_out, void* stream);
+
+/* Eq. 11 end to end: scores of all vision rows, then the selection above.
+ *   x_vis dev [B][n_vis_max][hidden]; score_out dev [B][n_vis_max]; others as above. */
+int32_t dl_prefill_select(dl_ctx* ctx, const dl_predictor* p_img, const void* x_vis,
+                          const int32_t* n_vis, const int32_t* k, int32_t B, int32_t n_vis_max,
+                          float* score_out, int32_t* kept_idx_out, int32_t k_max, uint8_t* keep_out,
+                          void* stream);
+
+/* ---- compaction: set builder of Eq. 5, reduced set of Eq. 11, append of Eq. 6 --------- */
+
+/* Appends to each sequence's cache, in token order, the source rows whose keep flag is 1,
+ * starting at row cache_len[b]; if `commit` != 0, cache_len[b] += number appended.
+ *   k_src, v_src dev [B][t_src_max][H][D] (v_src and v_cache may both be NULL: one tensor only);
+ *   keep dev [B][t_src_max] or NULL (= keep all); t_src dev [B] valid source rows or NULL;
+ *   k_cache, v_cache dev [B][H][cap][D]; cache_len dev [B], read, and written when commit != 0.
+ * Rows are copied bit for bit.  A sequence whose kept rows do not fit (cache_len + count > cap)
+ * is left untouched, its length unchanged, and DL_ERR_CAPACITY is recorded with its index.
+ * Several layers that share one decision pass commit = 0 for all but the last layer's call.
+ * Needs the workspace. */
+int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
+                      const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
+                      void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, void* stream);
+
+/* ---- attention over the reduced set --------------------------------------------------- */
+
+/* Prefill (Eq. 1 on S^{P*}): causal scaled-dot-product attention of the compact rows against
+ * themselves, per sequence and head: row i attends rows 0..i of the same cache.
+ *   q dev [B][H][cap][D] compact queries in the cache layout (built by dl_compact_kv);
+ *   k_cache, v_cache dev [B][H][cap][D]; cache_len dev [B]; n_max >= every cache_len[b], <= cap;
+ *   out dev [B][n_max][H][D] (rows >= cache_len[b] are not written); scale usually 1/sqrt(D). */
+int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max,
+                               float scale, void* out, void* stream);
+
+/* Decoding with KV cache (Eq. 6, second line): Attention(Q, S^K u K, S^V u V) for one new token
+ * per sequence: the query attends cache rows [0, cache_len[b]) plus the token's own (k_t, v_t).
+ *   q_t, k_t, v_t dev [B][H][D]; out dev [B][H][D].
+ * If `keep` (dev [B], may be NULL) is given, the call also performs Eq. 6's conditional append
+ * for this layer: where keep[b] != 0, (k_t, v_t) are written to row cache_len[b] of the caches
+ * (cache_len itself is not changed: call dl_commit_len once after the last layer).  A full
+ * cache (cache_len[b] == cap) records DL_ERR_CAPACITY and skips the write.  Needs the workspace. */
+int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t,
+                              void* k_cache, void* v_cache, const int32_t* cache_len,
+                              const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
+                              void* stream);
+
+/* ---- decode decision: Eq. 5 applied to the current token (Eq. 6) ----------------------- */
+
+/* logit[b] = P^{OT}(x_t[b]);  keep[b] = logit[b] > threshold (strict; NaN -> 0).
+ *   x_t dev [B][hidden] or NULL: with NULL the logits already in logit_inout are used as given.
+ *   logit_inout dev [B]; keep_out dev [B]. */
+int32_t dl_decode_keep(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B,
+                       float threshold, float* logit_inout, uint8_t* keep_out, void* stream);
+
+/* cache_len[b] += (keep[b] != 0) where cache_len[b] < cap: closes a decode step after every
+ * layer has appended with the shared decision (Sec. 3.3.2). */
+int32_t dl_commit_len(dl_ctx* ctx, const uint8_t* keep, int32_t B, int32_t cap, int32_t* cache_len,
+                      void* stream);
+
+/* One whole decode step over a stack of L layers that share the decision: dl_decode_keep, then
+ * per layer dl_sparse_attn_decode with the fused append, then dl_commit_len.
+ *   q_t, k_t, v_t, out: dev [L][B][H][D]; k_caches, v_caches: HOST arrays of L device pointers,
+ *   each [B][H][cap][D].  Other arguments as in the single calls. */
+int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B,
+                       float threshold, float* logit_inout, uint8_t* keep_out, int32_t L,
+                       const void* q_t, const void* k_t, const void* v_t, void* const* k_caches,
+                       void* const* v_caches, int32_t cap, int32_t* cache_len, float scale,
+                       void* out, void* stream);
+
+/* The same step fed from HOST buffers (pinned for full copy speed): copies x_t, q_t, k_t, v_t
+ * into the caller's device staging buffers, runs dl_decode_step, copies `out` and `keep` back to
+ * the host, all on `stream`; returns after the stream has been synchronised.
+ *   *_host: host counterparts of the dl_decode_step tensors; stage_* : dev buffers of the same
+ *   sizes (x [B][hidden]; q, k, v, out [L][B][H][D]); logit_dev [B], keep_dev [B] dev. */
+int32_t dl_decode_step_host(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_host, int32_t B,
+                            float threshold, int32_t L, const void* q_host, const void* k_host,
+                            const void* v_host, void* out_host, uint8_t* keep_host, void* stage_x,
+                            void* stage_q, void* stage_k, void* stage_v, void* stage_out,
+                            float* logit_dev, uint8_t* keep_dev, void* const* k_caches,
+                            void* const* v_caches, int32_t cap, int32_t* cache_len, float scale,
+                            void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DL_SPARSE_H_ */

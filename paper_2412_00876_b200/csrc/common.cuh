@@ -1,0 +1,133 @@
+// Shared declarations of the library's translation units: context, workspace layout,
+// device status word, small device helpers and the kernel launchers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/dl.h"
+
+namespace dl {
+
+// ---------------------------------------------------------------------------------------
+// Device status word (first bytes of the workspace).  Kernels record the FIRST error they
+// see with an atomic compare-and-swap on `code`; warnings never overwrite errors.
+// ---------------------------------------------------------------------------------------
+struct DeviceStatus {
+  int32_t code;
+  int32_t pad;
+  unsigned long long detail;
+};
+
+__device__ __forceinline__ void report_status(DeviceStatus* st, int32_t code, long long detail) {
+  if (st == nullptr) return;
+  int32_t old = atomicCAS(&st->code, 0, code);
+  if (old == 0) {
+    atomicExch(&st->detail, (unsigned long long)detail);
+  } else if (old > 0 && code < 0) {  // an error replaces a warning
+    if (atomicCAS(&st->code, old, code) == old) atomicExch(&st->detail, (unsigned long long)detail);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Workspace layout (all offsets 256-byte aligned).
+// ---------------------------------------------------------------------------------------
+constexpr int kDecodeMinChunk = 64;   // smallest rows-per-item the decode kernel may be asked for
+constexpr int kPredMaxSplit = 32;     // most column splits of the predictor's hidden layer
+constexpr int kPredRowTile = 128;     // rows per predictor row tile (tensor-core kernel)
+
+struct Workspace {
+  char* base = nullptr;
+  int64_t bytes = 0;
+  int32_t max_batch = 0, max_rows = 0, cap = 0;
+  // sub-buffers
+  DeviceStatus* status = nullptr;
+  int32_t* plan_base = nullptr;       // [max_batch] compaction: first destination row
+  int32_t* plan_count = nullptr;      // [max_batch] compaction: rows to append (-1: skip sequence)
+  int32_t* dec_ticket = nullptr;      // [max_batch * H] decode: arrivals per (b,h); zero between launches
+  float* dec_partial = nullptr;       // [max_batch * H * dec_slots * (D + 2)]
+  int32_t dec_slots = 0;              // partial slots per (b,h)
+  float* pred_partial = nullptr;      // [kPredMaxSplit][max_rows padded to kPredRowTile]
+  int32_t* pred_ticket = nullptr;     // [row tiles]; zero between launches
+  int32_t pred_rows_padded = 0;
+};
+
+int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_rows, int32_t cap,
+                         Workspace* ws /* may be null: size query only */);
+
+struct Options {
+  int32_t predictor_impl = 0;
+  int32_t prefill_attn_impl = 0;
+  int32_t decode_chunk = 0;
+};
+
+}  // namespace dl
+
+struct dl_ctx {
+  int32_t device = 0;
+  dl_model_desc desc{};
+  dl::Workspace ws{};
+  dl::Options opt{};
+  int32_t sm_count = 0;
+  int32_t smem_optin = 0;
+  cudaError_t last_cuda = cudaSuccess;
+  void* tmap_encode = nullptr;        // cuTensorMapEncodeTiled, resolved at create
+};
+
+namespace dl {
+
+// ---------------------------------------------------------------------------------------
+// element helpers
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// exact-erf GELU in fp32
+__device__ __forceinline__ float gelu_erf(float h) { return 0.5f * h * (1.0f + erff(h * 0.70710678118654752440f)); }
+
+// ---------------------------------------------------------------------------------------
+// kernel launchers (one per translation unit); all return the launch's cudaError_t
+// ---------------------------------------------------------------------------------------
+cudaError_t launch_topk(const float* score, const int32_t* n_vis, const int32_t* k, int32_t B,
+                        int32_t n_vis_max, int32_t* kept_idx, int32_t k_max, uint8_t* keep,
+                        DeviceStatus* st, cudaStream_t s);
+
+cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
+                           const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
+                           void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, cudaStream_t s);
+
+cudaError_t launch_commit_len(const uint8_t* keep, int32_t B, int32_t cap, int32_t* cache_len,
+                              cudaStream_t s);
+
+cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t,
+                               void* k_cache, void* v_cache, const int32_t* cache_len,
+                               const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
+                               cudaStream_t s);
+
+cudaError_t launch_predictor_simt(const dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows,
+                                  float* score, cudaStream_t s);
+cudaError_t launch_predictor_tc(dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows,
+                                float* score, cudaStream_t s);
+bool predictor_tc_supported(const dl_ctx* ctx);
+
+cudaError_t launch_decode_keep(const float* logit, int32_t B, float threshold, uint8_t* keep,
+                               DeviceStatus* st, cudaStream_t s);
+
+cudaError_t launch_attn_prefill_simt(const dl_ctx* ctx, const void* q, const void* k_cache,
+                                     const void* v_cache, const int32_t* cache_len, int32_t B,
+                                     int32_t cap, int32_t n_max, float scale, void* out, cudaStream_t s);
+cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                                   const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max,
+                                   float scale, void* out, cudaStream_t s);
+bool attn_prefill_tc_supported(const dl_ctx* ctx);
+
+}  // namespace dl
