@@ -130,14 +130,17 @@ int32_t dl_prefill_select(dl_ctx* ctx, const dl_predictor* p_img, const void* x_
 /* Appends to each sequence's cache, in token order, the source rows whose keep flag is 1,
  * starting at row cache_len[b]; if `commit` != 0, cache_len[b] += number appended.
  *   k_src, v_src dev [B][t_src_max][H][D] (v_src and v_cache may both be NULL: one tensor only);
- *   keep dev [B][t_src_max] or NULL (= keep all); t_src dev [B] valid source rows or NULL;
+ *   keep dev [B][keep_cols] or NULL (= keep all): the flags of the first keep_cols source rows;
+ *   source rows t >= keep_cols are always kept.  In prefill keep_cols is the number of vision
+ *   slots, so that the mask is M^I followed by ones for the text rows (S^{I*} u S^T of Eq. 11);
+ *   t_src dev [B] valid source rows or NULL (= t_src_max);
  *   k_cache, v_cache dev [B][H][cap][D]; cache_len dev [B], read, and written when commit != 0.
  * Rows are copied bit for bit.  A sequence whose kept rows do not fit (cache_len + count > cap)
  * is left untouched, its length unchanged, and DL_ERR_CAPACITY is recorded with its index.
  * Several layers that share one decision pass commit = 0 for all but the last layer's call.
  * Needs the workspace. */
 int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
-                      const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
+                      int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
                       void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, void* stream);
 
 /* ---- attention over the reduced set --------------------------------------------------- */

@@ -1,0 +1,238 @@
+"""ctypes binding of libdl_sparse.so: same names as include/dl.h, argument marshalling only.
+
+Tensors are torch CUDA tensors (device memory and streams are torch's); every step of the
+path runs in the library's kernels.  There is no fallback: if the library has not been
+built the import of this module's `lib()` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdl_sparse.so")
+
+DL_F32, DL_BF16 = 0, 1
+DL_OK = 0
+DL_ERR_INVALID_ARG, DL_ERR_ALIGNMENT, DL_ERR_UNSUPPORTED, DL_ERR_WORKSPACE = -1, -2, -3, -4
+DL_ERR_CUDA, DL_ERR_CAPACITY, DL_ERR_TIMEOUT, DL_WARN_NAN = -5, -6, -7, 1
+DL_OPT_PREDICTOR_IMPL, DL_OPT_PREFILL_ATTN_IMPL, DL_OPT_DECODE_CHUNK = 1, 2, 3
+
+EXPORTS = [
+    "dl_create", "dl_destroy", "dl_workspace_bytes", "dl_set_workspace", "dl_set_option",
+    "dl_device_status", "dl_status_str", "dl_last_cuda_error", "dl_predictor_scores",
+    "dl_topk_from_scores", "dl_prefill_select", "dl_compact_kv", "dl_sparse_attn_prefill",
+    "dl_sparse_attn_decode", "dl_decode_keep", "dl_commit_len", "dl_decode_step", "dl_decode_step_host",
+]
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("pred_hidden", C.c_int32), ("dtype", C.c_int32)]
+
+
+class PredictorDesc(C.Structure):
+    _fields_ = [("w1", C.c_void_p), ("b1", C.c_void_p), ("w2", C.c_void_p), ("b2", C.c_float)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Opens the CUDA library (once).  Raises if it is missing: build it with
+    `python -m paper_2412_00876_b200.build`."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: run `python -m paper_2412_00876_b200.build` "
+                               "(there is no CPU or PyTorch fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+        P = C.POINTER(PredictorDesc)
+        sig = {
+            "dl_create": (i32, [C.POINTER(vp), i32, C.POINTER(ModelDesc)]),
+            "dl_destroy": (i32, [vp]),
+            "dl_workspace_bytes": (i64, [vp, i32, i32, i32]),
+            "dl_set_workspace": (i32, [vp, vp, i64, i32, i32, i32, vp]),
+            "dl_set_option": (i32, [vp, i32, i32]),
+            "dl_device_status": (i32, [vp, vp, C.POINTER(i32), C.POINTER(i64)]),
+            "dl_status_str": (C.c_char_p, [i32]),
+            "dl_last_cuda_error": (C.c_char_p, [vp]),
+            "dl_predictor_scores": (i32, [vp, P, vp, i32, vp, vp]),
+            "dl_topk_from_scores": (i32, [vp, vp, vp, vp, i32, i32, vp, i32, vp, vp]),
+            "dl_prefill_select": (i32, [vp, P, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp]),
+            "dl_compact_kv": (i32, [vp, vp, vp, vp, i32, vp, i32, i32, vp, vp, i32, vp, i32, vp]),
+            "dl_sparse_attn_prefill": (i32, [vp, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp]),
+            "dl_sparse_attn_decode": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp]),
+            "dl_decode_keep": (i32, [vp, P, vp, i32, f32, vp, vp, vp]),
+            "dl_commit_len": (i32, [vp, vp, i32, i32, vp, vp]),
+            "dl_decode_step": (i32, [vp, P, vp, i32, f32, vp, vp, i32, vp, vp, vp, C.POINTER(vp),
+                                     C.POINTER(vp), i32, vp, f32, vp, vp]),
+            "dl_decode_step_host": (i32, [vp, P, vp, i32, f32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                          vp, vp, C.POINTER(vp), C.POINTER(vp), i32, vp, f32, vp]),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+class DlError(RuntimeError):
+    def __init__(self, code: int, where: str, extra: str = ""):
+        self.code = code
+        msg = lib().dl_status_str(code).decode()
+        super().__init__(f"{where}: {msg} ({code}){' - ' + extra if extra else ''}")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        if not t.is_contiguous():
+            raise ValueError("tensor must be contiguous")
+        return t.data_ptr()
+    return int(t)
+
+
+def _stream(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+class Predictor:
+    """Device copy of one predictor's weights (see dl_predictor in dl.h)."""
+
+    def __init__(self, w1: torch.Tensor, b1: torch.Tensor, w2: torch.Tensor, b2: float):
+        assert b1.dtype == torch.float32 and w2.dtype == torch.float32
+        self.w1, self.b1, self.w2, self.b2 = w1.contiguous(), b1.contiguous(), w2.contiguous(), float(b2)
+        self.desc = PredictorDesc(self.w1.data_ptr(), self.b1.data_ptr(), self.w2.data_ptr(), self.b2)
+
+
+class Context:
+    """Owns a dl_ctx and the torch tensor that serves as its workspace."""
+
+    def __init__(self, hidden: int, n_heads: int, head_dim: int, pred_hidden: int, dtype: torch.dtype,
+                 device: int = 0, max_batch: int = 1, max_rows: int = 0, cap: int = 64):
+        self._h = C.c_void_p()
+        self.dtype = dtype
+        self.device = torch.device("cuda", device)
+        self.H, self.D, self.hidden = n_heads, head_dim, hidden
+        d = ModelDesc(hidden, n_heads, head_dim, pred_hidden, DL_F32 if dtype == torch.float32 else DL_BF16)
+        st = lib().dl_create(C.byref(self._h), device, C.byref(d))
+        if st != DL_OK:
+            raise DlError(st, "dl_create")
+        self._ws = None
+        self.set_workspace(max_batch, max(max_rows, max_batch), cap)
+
+    def close(self):
+        if self._h:
+            lib().dl_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int, where: str):
+        if st != DL_OK:
+            extra = lib().dl_last_cuda_error(self._h).decode() if st == DL_ERR_CUDA else ""
+            raise DlError(st, where, extra)
+
+    # ---- context calls
+    def set_workspace(self, max_batch: int, max_rows: int, cap: int, stream=None):
+        n = lib().dl_workspace_bytes(self._h, max_batch, max_rows, cap)
+        if n < 0:
+            raise DlError(int(n), "dl_workspace_bytes")
+        self._ws = torch.empty(int(n) + 256, dtype=torch.uint8, device=self.device)
+        base = (self._ws.data_ptr() + 255) // 256 * 256
+        self._check(lib().dl_set_workspace(self._h, base, n, max_batch, max_rows, cap, _stream(stream)),
+                    "dl_set_workspace")
+        self.max_batch, self.max_rows, self.cap = max_batch, max_rows, cap
+
+    def set_option(self, option: int, value: int):
+        self._check(lib().dl_set_option(self._h, option, value), "dl_set_option")
+
+    def device_status(self, stream=None):
+        code, detail = C.c_int32(0), C.c_int64(0)
+        self._check(lib().dl_device_status(self._h, _stream(stream), C.byref(code), C.byref(detail)),
+                    "dl_device_status")
+        return code.value, detail.value
+
+    # ---- the path
+    def predictor_scores(self, p: Predictor, x, score_out, stream=None):
+        rows = x.numel() // self.hidden
+        self._check(lib().dl_predictor_scores(self._h, C.byref(p.desc), _ptr(x), rows, _ptr(score_out),
+                                              _stream(stream)), "dl_predictor_scores")
+
+    def topk_from_scores(self, score, n_vis, k, kept_idx_out, keep_out, stream=None):
+        B, n_max = score.shape
+        k_max = 0 if kept_idx_out is None else kept_idx_out.shape[1]
+        self._check(lib().dl_topk_from_scores(self._h, _ptr(score), _ptr(n_vis), _ptr(k), B, n_max,
+                                              _ptr(kept_idx_out), k_max, _ptr(keep_out), _stream(stream)),
+                    "dl_topk_from_scores")
+
+    def prefill_select(self, p: Predictor, x_vis, n_vis, k, score_out, kept_idx_out, keep_out, stream=None):
+        B, n_max = x_vis.shape[0], x_vis.shape[1]
+        k_max = 0 if kept_idx_out is None else kept_idx_out.shape[1]
+        self._check(lib().dl_prefill_select(self._h, C.byref(p.desc), _ptr(x_vis), _ptr(n_vis), _ptr(k), B,
+                                            n_max, _ptr(score_out), _ptr(kept_idx_out), k_max, _ptr(keep_out),
+                                            _stream(stream)), "dl_prefill_select")
+
+    def compact_kv(self, k_src, v_src, keep, t_src, k_cache, v_cache, cache_len, commit=True, stream=None):
+        B, T = k_src.shape[0], k_src.shape[1]
+        cap = k_cache.shape[2]
+        keep_cols = 0 if keep is None else keep.shape[1]
+        self._check(lib().dl_compact_kv(self._h, _ptr(k_src), _ptr(v_src), _ptr(keep), keep_cols, _ptr(t_src), B, T,
+                                        _ptr(k_cache), _ptr(v_cache), cap, _ptr(cache_len), int(bool(commit)),
+                                        _stream(stream)), "dl_compact_kv")
+
+    def sparse_attn_prefill(self, q, k_cache, v_cache, cache_len, n_max, scale, out, stream=None):
+        B, cap = k_cache.shape[0], k_cache.shape[2]
+        self._check(lib().dl_sparse_attn_prefill(self._h, _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(cache_len),
+                                                 B, cap, n_max, float(scale), _ptr(out), _stream(stream)),
+                    "dl_sparse_attn_prefill")
+
+    def sparse_attn_decode(self, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, scale, out, stream=None):
+        B, cap = k_cache.shape[0], k_cache.shape[2]
+        self._check(lib().dl_sparse_attn_decode(self._h, _ptr(q_t), _ptr(k_t), _ptr(v_t), _ptr(k_cache),
+                                                _ptr(v_cache), _ptr(cache_len), _ptr(keep), B, cap, float(scale),
+                                                _ptr(out), _stream(stream)), "dl_sparse_attn_decode")
+
+    def decode_keep(self, p: Predictor | None, x_t, logit_inout, keep_out, threshold=0.0, stream=None):
+        B = logit_inout.shape[0]
+        pd = C.byref(p.desc) if p is not None else None
+        self._check(lib().dl_decode_keep(self._h, pd, _ptr(x_t), B, float(threshold), _ptr(logit_inout),
+                                         _ptr(keep_out), _stream(stream)), "dl_decode_keep")
+
+    def commit_len(self, keep, cache_len, cap, stream=None):
+        self._check(lib().dl_commit_len(self._h, _ptr(keep), keep.shape[0], cap, _ptr(cache_len),
+                                        _stream(stream)), "dl_commit_len")
+
+    @staticmethod
+    def pointer_array(tensors):
+        arr = (C.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+        return arr
+
+    def decode_step(self, p: Predictor | None, x_t, logit_inout, keep_out, q_t, k_t, v_t, k_ptrs, v_ptrs, L,
+                    cap, cache_len, scale, out, threshold=0.0, stream=None):
+        B = logit_inout.shape[0]
+        pd = C.byref(p.desc) if p is not None else None
+        self._check(lib().dl_decode_step(self._h, pd, _ptr(x_t), B, float(threshold), _ptr(logit_inout),
+                                         _ptr(keep_out), L, _ptr(q_t), _ptr(k_t), _ptr(v_t), k_ptrs, v_ptrs, cap,
+                                         _ptr(cache_len), float(scale), _ptr(out), _stream(stream)),
+                    "dl_decode_step")
+
+    def decode_step_host(self, p: Predictor, x_host, q_host, k_host, v_host, out_host, keep_host, stage_x,
+                         stage_q, stage_k, stage_v, stage_out, logit_dev, keep_dev, k_ptrs, v_ptrs, L, cap,
+                         cache_len, scale, threshold=0.0, stream=None):
+        B = logit_dev.shape[0]
+        self._check(lib().dl_decode_step_host(
+            self._h, C.byref(p.desc), _ptr(x_host), B, float(threshold), L, _ptr(q_host), _ptr(k_host),
+            _ptr(v_host), _ptr(out_host), _ptr(keep_host), _ptr(stage_x), _ptr(stage_q), _ptr(stage_k),
+            _ptr(stage_v), _ptr(stage_out), _ptr(logit_dev), _ptr(keep_dev), k_ptrs, v_ptrs, cap,
+            _ptr(cache_len), float(scale), _stream(stream)), "dl_decode_step_host")

@@ -1,0 +1,337 @@
+// Host side of the C ABI: argument checks, workspace layout, dispatch to the kernel launchers.
+// No call here allocates device memory or synchronises, except where dl.h says so.
+#include <new>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace dl {
+
+static inline int64_t align256(int64_t v) { return (v + 255) & ~int64_t(255); }
+
+int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_rows, int32_t cap,
+                         Workspace* ws) {
+  int64_t off = 0;
+  auto take = [&](int64_t bytes) { int64_t o = off; off = align256(off + bytes); return o; };
+  const int64_t o_status = take(sizeof(DeviceStatus));
+  const int64_t o_pbase = take((int64_t)max_batch * 4);
+  const int64_t o_pcount = take((int64_t)max_batch * 4);
+  const int64_t o_ticket = take((int64_t)max_batch * d.n_heads * 4);
+  const int32_t slots = (cap + kDecodeMinChunk - 1) / kDecodeMinChunk + 1;
+  const int64_t o_partial = take((int64_t)max_batch * d.n_heads * slots * (d.head_dim + 2) * 4);
+  const int32_t rows_pad = (max_rows + kPredRowTile - 1) / kPredRowTile * kPredRowTile;
+  const int64_t o_ppart = take((int64_t)kPredMaxSplit * rows_pad * 4);
+  const int64_t o_ptick = take((int64_t)(rows_pad / kPredRowTile + 1) * 4);
+  if (ws) {
+    char* b = ws->base;
+    ws->status = reinterpret_cast<DeviceStatus*>(b + o_status);
+    ws->plan_base = reinterpret_cast<int32_t*>(b + o_pbase);
+    ws->plan_count = reinterpret_cast<int32_t*>(b + o_pcount);
+    ws->dec_ticket = reinterpret_cast<int32_t*>(b + o_ticket);
+    ws->dec_partial = reinterpret_cast<float*>(b + o_partial);
+    ws->dec_slots = slots;
+    ws->pred_partial = reinterpret_cast<float*>(b + o_ppart);
+    ws->pred_ticket = reinterpret_cast<int32_t*>(b + o_ptick);
+    ws->pred_rows_padded = rows_pad;
+    ws->max_batch = max_batch; ws->max_rows = max_rows; ws->cap = cap;
+  }
+  return off;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool changed = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) { cudaSetDevice(dev); changed = true; }
+  }
+  ~DeviceGuard() { if (changed) cudaSetDevice(prev); }
+};
+
+static inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+static inline int32_t cuda_status(dl_ctx* ctx, cudaError_t e) {
+  if (e == cudaSuccess) return DL_OK;
+  ctx->last_cuda = e;
+  return DL_ERR_CUDA;
+}
+
+static inline int elt_bytes(const dl_ctx* ctx) { return ctx->desc.dtype == DL_F32 ? 4 : 2; }
+
+static int32_t run_predictor(dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows, float* score,
+                             cudaStream_t s) {
+  if (!p || !p->w1 || !p->b1 || !p->w2 || !x || !score) return DL_ERR_INVALID_ARG;
+  if (misaligned(p->w1) || misaligned(x)) return DL_ERR_ALIGNMENT;
+  int impl = ctx->opt.predictor_impl;
+  if (impl == 0) impl = predictor_tc_supported(ctx) ? 2 : 1;
+  if (impl == 2) {
+    if (!predictor_tc_supported(ctx)) return DL_ERR_UNSUPPORTED;
+    if (!ctx->ws.base || rows > ctx->ws.max_rows) return DL_ERR_WORKSPACE;
+    return cuda_status(ctx, launch_predictor_tc(ctx, p, x, rows, score, s));
+  }
+  return cuda_status(ctx, launch_predictor_simt(ctx, p, x, rows, score, s));
+}
+
+}  // namespace dl
+
+using namespace dl;
+
+extern "C" {
+
+int32_t dl_create(dl_ctx** out, int32_t device, const dl_model_desc* desc) {
+  if (!out || !desc) return DL_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (desc->hidden <= 0 || desc->n_heads <= 0 || desc->pred_hidden <= 0) return DL_ERR_INVALID_ARG;
+  if (desc->dtype != DL_F32 && desc->dtype != DL_BF16) return DL_ERR_UNSUPPORTED;
+  if (desc->head_dim != 64 && desc->head_dim != 128) return DL_ERR_UNSUPPORTED;
+  if (desc->hidden % 8 != 0) return DL_ERR_UNSUPPORTED;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return DL_ERR_CUDA;
+  dl_ctx* c = new (std::nothrow) dl_ctx();
+  if (!c) return DL_ERR_INVALID_ARG;
+  c->device = device;
+  c->desc = *desc;
+  DeviceGuard g(device);
+  int v = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess) { c->sm_count = v; e = cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, device); }
+  if (e != cudaSuccess) { delete c; return DL_ERR_CUDA; }
+  c->smem_optin = v;
+  cudaDriverEntryPointQueryResult qres;
+  void* fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+      qres == cudaDriverEntryPointSuccess)
+    c->tmap_encode = fn;
+  (void)cudaGetLastError();
+  *out = c;
+  return DL_OK;
+}
+
+int32_t dl_destroy(dl_ctx* ctx) {
+  delete ctx;
+  return DL_OK;
+}
+
+int64_t dl_workspace_bytes(const dl_ctx* ctx, int32_t max_batch, int32_t max_rows, int32_t cap) {
+  if (!ctx || max_batch <= 0 || max_rows < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
+  return workspace_layout(ctx->desc, max_batch, max_rows, cap, nullptr);
+}
+
+int32_t dl_set_workspace(dl_ctx* ctx, void* dev_ptr, int64_t bytes, int32_t max_batch, int32_t max_rows,
+                         int32_t cap, void* stream) {
+  if (!ctx || !dev_ptr || max_batch <= 0 || max_rows < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(dev_ptr) & 255u) return DL_ERR_ALIGNMENT;
+  const int64_t need = workspace_layout(ctx->desc, max_batch, max_rows, cap, nullptr);
+  if (bytes < need) return DL_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  ctx->ws = Workspace();
+  ctx->ws.base = static_cast<char*>(dev_ptr);
+  ctx->ws.bytes = bytes;
+  workspace_layout(ctx->desc, max_batch, max_rows, cap, &ctx->ws);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemsetAsync(ctx->ws.status, 0, sizeof(DeviceStatus), s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.dec_ticket, 0, (size_t)max_batch * ctx->desc.n_heads * 4, s);
+  if (e == cudaSuccess)
+    e = cudaMemsetAsync(ctx->ws.pred_ticket, 0, (size_t)(ctx->ws.pred_rows_padded / kPredRowTile + 1) * 4, s);
+  return cuda_status(ctx, e);
+}
+
+int32_t dl_set_option(dl_ctx* ctx, int32_t option, int32_t value) {
+  if (!ctx || value < 0) return DL_ERR_INVALID_ARG;
+  switch (option) {
+    case DL_OPT_PREDICTOR_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.predictor_impl = value; break;
+    case DL_OPT_PREFILL_ATTN_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.prefill_attn_impl = value; break;
+    case DL_OPT_DECODE_CHUNK: ctx->opt.decode_chunk = value; break;
+    default: return DL_ERR_INVALID_ARG;
+  }
+  return DL_OK;
+}
+
+int32_t dl_device_status(dl_ctx* ctx, void* stream, int32_t* code_out, int64_t* detail_out) {
+  if (!ctx || !code_out) return DL_ERR_INVALID_ARG;
+  if (!ctx->ws.base) return DL_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  DeviceStatus h;
+  cudaError_t e = cudaMemcpyAsync(&h, ctx->ws.status, sizeof(h), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.status, 0, sizeof(DeviceStatus), s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_status(ctx, e);
+  *code_out = h.code;
+  if (detail_out) *detail_out = (int64_t)h.detail;
+  return DL_OK;
+}
+
+const char* dl_status_str(int32_t status) {
+  switch (status) {
+    case DL_OK: return "ok";
+    case DL_ERR_INVALID_ARG: return "invalid argument";
+    case DL_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case DL_ERR_UNSUPPORTED: return "unsupported dtype, head_dim or size";
+    case DL_ERR_WORKSPACE: return "workspace missing or too small";
+    case DL_ERR_CUDA: return "CUDA runtime error";
+    case DL_ERR_CAPACITY: return "kept rows do not fit into the cache";
+    case DL_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case DL_WARN_NAN: return "NaN score ranked as -inf / dropped";
+    default: return "unknown status";
+  }
+}
+
+const char* dl_last_cuda_error(const dl_ctx* ctx) {
+  return ctx ? cudaGetErrorString(ctx->last_cuda) : "no context";
+}
+
+int32_t dl_predictor_scores(dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows, float* score_out,
+                            void* stream) {
+  if (!ctx || rows < 0) return DL_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (rows == 0) return DL_OK;
+  return run_predictor(ctx, p, x, rows, score_out, static_cast<cudaStream_t>(stream));
+}
+
+int32_t dl_topk_from_scores(dl_ctx* ctx, const float* score, const int32_t* n_vis, const int32_t* k, int32_t B,
+                            int32_t n_vis_max, int32_t* kept_idx_out, int32_t k_max, uint8_t* keep_out,
+                            void* stream) {
+  if (!ctx || B < 0 || n_vis_max < 0 || k_max < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || n_vis_max == 0) return DL_OK;
+  if (!score || !k || !keep_out) return DL_ERR_INVALID_ARG;
+  if (n_vis_max > 16384) return DL_ERR_UNSUPPORTED;
+  DeviceGuard g(ctx->device);
+  return cuda_status(ctx, launch_topk(score, n_vis, k, B, n_vis_max, kept_idx_out, k_max, keep_out,
+                                      ctx->ws.status, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t dl_prefill_select(dl_ctx* ctx, const dl_predictor* p_img, const void* x_vis, const int32_t* n_vis,
+                          const int32_t* k, int32_t B, int32_t n_vis_max, float* score_out,
+                          int32_t* kept_idx_out, int32_t k_max, uint8_t* keep_out, void* stream) {
+  if (!ctx || B < 0 || n_vis_max < 0 || k_max < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || n_vis_max == 0) return DL_OK;
+  if ((int64_t)B * n_vis_max > INT32_MAX) return DL_ERR_UNSUPPORTED;
+  DeviceGuard g(ctx->device);
+  int32_t st = run_predictor(ctx, p_img, x_vis, B * n_vis_max, score_out, static_cast<cudaStream_t>(stream));
+  if (st != DL_OK) return st;
+  return dl_topk_from_scores(ctx, score_out, n_vis, k, B, n_vis_max, kept_idx_out, k_max, keep_out, stream);
+}
+
+int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
+                      int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache, void* v_cache,
+                      int32_t cap, int32_t* cache_len, int32_t commit, void* stream) {
+  if (!ctx || B < 0 || t_src_max < 0 || cap <= 0 || keep_cols < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || t_src_max == 0) return DL_OK;
+  if (!k_src || !k_cache || !cache_len) return DL_ERR_INVALID_ARG;
+  if ((v_src == nullptr) != (v_cache == nullptr)) return DL_ERR_INVALID_ARG;
+  if (misaligned(k_src) || misaligned(v_src) || misaligned(k_cache) || misaligned(v_cache)) return DL_ERR_ALIGNMENT;
+  if (!ctx->ws.base || B > ctx->ws.max_batch) return DL_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  return cuda_status(ctx, launch_compact(ctx, k_src, v_src, keep, keep_cols, t_src, B, t_src_max, k_cache, v_cache, cap,
+                                         cache_len, commit, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max, float scale,
+                               void* out, void* stream) {
+  if (!ctx || B < 0 || cap <= 0 || n_max < 0 || n_max > cap) return DL_ERR_INVALID_ARG;
+  if (B == 0 || n_max == 0) return DL_OK;
+  if (!q || !k_cache || !v_cache || !cache_len || !out) return DL_ERR_INVALID_ARG;
+  if (misaligned(q) || misaligned(k_cache) || misaligned(v_cache) || misaligned(out)) return DL_ERR_ALIGNMENT;
+  DeviceGuard g(ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int impl = ctx->opt.prefill_attn_impl;
+  if (impl == 0) impl = attn_prefill_tc_supported(ctx) ? 2 : 1;
+  if (impl == 2) {
+    if (!attn_prefill_tc_supported(ctx)) return DL_ERR_UNSUPPORTED;
+    return cuda_status(ctx, launch_attn_prefill_tc(ctx, q, k_cache, v_cache, cache_len, B, cap, n_max, scale, out, s));
+  }
+  return cuda_status(ctx, launch_attn_prefill_simt(ctx, q, k_cache, v_cache, cache_len, B, cap, n_max, scale, out, s));
+}
+
+int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
+                              void* v_cache, const int32_t* cache_len, const uint8_t* keep, int32_t B,
+                              int32_t cap, float scale, void* out, void* stream) {
+  if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
+  if (B == 0) return DL_OK;
+  if (!q_t || !k_t || !v_t || !k_cache || !v_cache || !cache_len || !out) return DL_ERR_INVALID_ARG;
+  if (misaligned(q_t) || misaligned(k_t) || misaligned(v_t) || misaligned(k_cache) || misaligned(v_cache) ||
+      misaligned(out))
+    return DL_ERR_ALIGNMENT;
+  if (!ctx->ws.base || B > ctx->ws.max_batch || cap > ctx->ws.cap) return DL_ERR_WORKSPACE;
+  if (B > 2048) return DL_ERR_UNSUPPORTED;
+  DeviceGuard g(ctx->device);
+  return cuda_status(ctx, launch_attn_decode(ctx, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, B, cap,
+                                             scale, out, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t dl_decode_keep(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
+                       float* logit_inout, uint8_t* keep_out, void* stream) {
+  if (!ctx || B < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0) return DL_OK;
+  if (!logit_inout || !keep_out) return DL_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (x_t) {
+    int32_t st = run_predictor(ctx, p_txt, x_t, B, logit_inout, s);
+    if (st != DL_OK) return st;
+  }
+  return cuda_status(ctx, launch_decode_keep(logit_inout, B, threshold, keep_out, ctx->ws.status, s));
+}
+
+int32_t dl_commit_len(dl_ctx* ctx, const uint8_t* keep, int32_t B, int32_t cap, int32_t* cache_len,
+                      void* stream) {
+  if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
+  if (B == 0) return DL_OK;
+  if (!keep || !cache_len) return DL_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  return cuda_status(ctx, launch_commit_len(keep, B, cap, cache_len, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
+                       float* logit_inout, uint8_t* keep_out, int32_t L, const void* q_t, const void* k_t,
+                       const void* v_t, void* const* k_caches, void* const* v_caches, int32_t cap,
+                       int32_t* cache_len, float scale, void* out, void* stream) {
+  if (!ctx || L < 0 || B < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0) return DL_OK;
+  if (L > 0 && (!k_caches || !v_caches || !q_t || !k_t || !v_t || !out)) return DL_ERR_INVALID_ARG;
+  int32_t st = dl_decode_keep(ctx, p_txt, x_t, B, threshold, logit_inout, keep_out, stream);
+  if (st != DL_OK) return st;
+  const size_t layer_bytes = (size_t)B * ctx->desc.n_heads * ctx->desc.head_dim * elt_bytes(ctx);
+  for (int32_t l = 0; l < L; ++l) {
+    const char* ql = static_cast<const char*>(q_t) + l * layer_bytes;
+    const char* kl = static_cast<const char*>(k_t) + l * layer_bytes;
+    const char* vl = static_cast<const char*>(v_t) + l * layer_bytes;
+    char* ol = static_cast<char*>(out) + l * layer_bytes;
+    st = dl_sparse_attn_decode(ctx, ql, kl, vl, k_caches[l], v_caches[l], cache_len, keep_out, B, cap, scale,
+                               ol, stream);
+    if (st != DL_OK) return st;
+  }
+  return dl_commit_len(ctx, keep_out, B, cap, cache_len, stream);
+}
+
+int32_t dl_decode_step_host(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_host, int32_t B,
+                            float threshold, int32_t L, const void* q_host, const void* k_host,
+                            const void* v_host, void* out_host, uint8_t* keep_host, void* stage_x,
+                            void* stage_q, void* stage_k, void* stage_v, void* stage_out, float* logit_dev,
+                            uint8_t* keep_dev, void* const* k_caches, void* const* v_caches, int32_t cap,
+                            int32_t* cache_len, float scale, void* stream) {
+  if (!ctx || L < 0 || B < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0) return DL_OK;
+  if (!x_host || !stage_x || !logit_dev || !keep_dev) return DL_ERR_INVALID_ARG;
+  if (L > 0 && (!q_host || !k_host || !v_host || !out_host || !stage_q || !stage_k || !stage_v || !stage_out))
+    return DL_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t xb = (size_t)B * ctx->desc.hidden * elt_bytes(ctx);
+  const size_t lb = (size_t)L * B * ctx->desc.n_heads * ctx->desc.head_dim * elt_bytes(ctx);
+  cudaError_t e = cudaMemcpyAsync(stage_x, x_host, xb, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess && lb) e = cudaMemcpyAsync(stage_q, q_host, lb, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess && lb) e = cudaMemcpyAsync(stage_k, k_host, lb, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess && lb) e = cudaMemcpyAsync(stage_v, v_host, lb, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return cuda_status(ctx, e);
+  int32_t st = dl_decode_step(ctx, p_txt, stage_x, B, threshold, logit_dev, keep_dev, L, stage_q, stage_k,
+                              stage_v, k_caches, v_caches, cap, cache_len, scale, stage_out, stream);
+  if (st != DL_OK) return st;
+  if (lb) e = cudaMemcpyAsync(out_host, stage_out, lb, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess && keep_host) e = cudaMemcpyAsync(keep_host, keep_dev, (size_t)B, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  return cuda_status(ctx, e);
+}
+
+}  // extern "C"

@@ -31,7 +31,7 @@ __device__ __forceinline__ int block_sum_256(int v, int* sh) {
 }
 
 __global__ void __launch_bounds__(kPlanThreads)
-compact_plan_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ t_src, int32_t t_max,
+compact_plan_kernel(const uint8_t* __restrict__ keep, int32_t keep_cols, const int32_t* __restrict__ t_src, int32_t t_max,
                     int32_t cap, int32_t* __restrict__ cache_len, int32_t commit,
                     int32_t* __restrict__ plan_base, int32_t* __restrict__ plan_count, DeviceStatus* st) {
   __shared__ int sh[8];
@@ -40,8 +40,8 @@ compact_plan_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict_
   tb = max(0, min(tb, t_max));
   int c = 0;
   if (keep) {
-    const uint8_t* kp = keep + (size_t)b * t_max;
-    for (int i = threadIdx.x; i < tb; i += kPlanThreads) c += (kp[i] != 0);
+    const uint8_t* kp = keep + (size_t)b * keep_cols;
+    for (int i = threadIdx.x; i < tb; i += kPlanThreads) c += (i >= keep_cols || kp[i] != 0);
   } else {
     for (int i = threadIdx.x; i < tb; i += kPlanThreads) c += 1;
   }
@@ -64,8 +64,8 @@ compact_plan_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict_
 // piece_units = D*elt/16 (units per head piece).
 __global__ void __launch_bounds__(kCopyThreads)
 compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v_src,
-                    const uint8_t* __restrict__ keep, const int32_t* __restrict__ t_src, int32_t t_max,
-                    uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, int32_t cap, int32_t H,
+                    const uint8_t* __restrict__ keep, int32_t keep_cols, const int32_t* __restrict__ t_src,
+                    int32_t t_max, uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, int32_t cap, int32_t H,
                     int32_t row_units, int32_t piece_units, const int32_t* __restrict__ plan_base,
                     const int32_t* __restrict__ plan_count) {
   __shared__ int sh[8];
@@ -78,12 +78,12 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
   tb = max(0, min(tb, t_max));
   const int t0 = blockIdx.x * kTileTokens;
   if (t0 >= tb) return;
-  const uint8_t* kp = keep ? keep + (size_t)b * t_max : nullptr;
+  const uint8_t* kp = keep ? keep + (size_t)b * keep_cols : nullptr;
 
   // kept tokens before this tile
   int before = 0;
   if (kp) {
-    for (int i = threadIdx.x; i < t0; i += kCopyThreads) before += (kp[i] != 0);
+    for (int i = threadIdx.x; i < t0; i += kCopyThreads) before += (i >= keep_cols || kp[i] != 0);
     before = block_sum_256(before, sh);
   } else {
     before = t0;
@@ -91,7 +91,7 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
   // rank the tile's kept tokens
   if (threadIdx.x < 32) {
     int t = t0 + threadIdx.x;
-    bool f = (t < tb) && (kp == nullptr || kp[t] != 0);
+    bool f = (t < tb) && (kp == nullptr || t >= keep_cols || kp[t] != 0);
     unsigned m = __ballot_sync(0xffffffffu, f);
     if (f) tile_tok[__popc(m & ((1u << threadIdx.x) - 1u))] = t;
     if (threadIdx.x == 0) tile_kept = __popc(m);
@@ -131,20 +131,20 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
 }
 
 cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
-                           const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
+                           int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
                            void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, cudaStream_t s) {
   if (B == 0 || t_src_max == 0) return cudaSuccess;
   const dl_model_desc& d = ctx->desc;
   const int elt = d.dtype == DL_F32 ? 4 : 2;
   const int piece_units = d.head_dim * elt / 16;
   const int row_units = piece_units * d.n_heads;
-  compact_plan_kernel<<<B, kPlanThreads, 0, s>>>(keep, t_src, t_src_max, cap, cache_len, commit,
+  compact_plan_kernel<<<B, kPlanThreads, 0, s>>>(keep, keep_cols, t_src, t_src_max, cap, cache_len, commit,
                                                  ctx->ws.plan_base, ctx->ws.plan_count, ctx->ws.status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   dim3 grid((t_src_max + kTileTokens - 1) / kTileTokens, B);
   compact_copy_kernel<<<grid, kCopyThreads, 0, s>>>(
-      (const uint4*)k_src, (const uint4*)v_src, keep, t_src, t_src_max, (uint4*)k_cache, (uint4*)v_cache,
+      (const uint4*)k_src, (const uint4*)v_src, keep, keep_cols, t_src, t_src_max, (uint4*)k_cache, (uint4*)v_cache,
       cap, d.n_heads, row_units, piece_units, ctx->ws.plan_base, ctx->ws.plan_count);
   return cudaGetLastError();
 }
