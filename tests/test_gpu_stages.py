@@ -1,0 +1,233 @@
+"""Stage-isolated GPU-vs-oracle parity through the C ABI: every kernel is fed inputs from
+the seeded generators (or the oracle's upstream output) and compared element by element."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dl_oracle as orc
+from paper_2412_00876_b200 import workloads as wl
+from tests import path_check as pc
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _ctx(dtype="bf16", H=4, D=128, hidden=256, pred=64, B=4, rows=0, cap=512):
+    from paper_2412_00876_b200 import binding as dl
+    return dl.Context(hidden, H, D, pred, wl.torch_dtype(dtype), 0, max_batch=B, max_rows=max(rows, B), cap=cap)
+
+
+# ------------------------------------------------------------------------------ top-k
+def _topk_case(score, n_vis, k):
+    ctx = _ctx(B=score.shape[0])
+    B, n = score.shape
+    k_max = max(1, int(np.max(k)))
+    s_d = torch.from_numpy(score.astype(np.float32)).to(DEV)
+    idx = torch.full((B, k_max), -7, dtype=torch.int32, device=DEV)
+    keep = torch.full((B, n), 9, dtype=torch.uint8, device=DEV)
+    nv = None if n_vis is None else torch.from_numpy(np.asarray(n_vis, np.int32)).to(DEV)
+    ctx.topk_from_scores(s_d, nv, torch.from_numpy(np.asarray(k, np.int32)).to(DEV), idx, keep)
+    ridx, rkeep = orc.prefill_select(score.astype(np.float32).astype(np.float64), n_vis, np.asarray(k), k_max)
+    assert np.array_equal(keep.cpu().numpy(), rkeep)
+    assert np.array_equal(idx.cpu().numpy(), ridx)
+    return ctx
+
+
+def test_topk_random_ties_and_sizes():
+    rng = np.random.default_rng(0)
+    for n in (1, 31, 144, 576, 2880, 5000, 16384):
+        B = 3
+        score = np.round(rng.normal(size=(B, n)), 1 if n < 3000 else 3)      # many exact ties
+        k = np.array([0, n, n // 4])
+        _topk_case(score, None, k)
+        n_vis = np.array([n, max(1, n // 2), max(1, n - 1)])
+        k = np.array([n // 5, max(1, n // 2), 1])
+        _topk_case(score, n_vis, k)
+
+
+def test_topk_special_values():
+    s = np.array([[0.0, -0.0, 0.0, -0.0, 1.0, -1.0, np.inf, -np.inf],
+                  [np.nan, 1.0, np.nan, -np.inf, 2.0, 2.0, 2.0, -0.0],
+                  [5.0] * 8])
+    for k in ([2, 3, 4], [8, 8, 8], [0, 0, 0], [5, 7, 1]):
+        ctx = _topk_case(s, None, np.array(k))
+    code, _ = ctx.device_status()
+    from paper_2412_00876_b200 import binding as dl
+    assert code == dl.DL_WARN_NAN
+
+
+def test_topk_paper_rate():
+    rng = np.random.default_rng(1)
+    k = orc.k_from_rate(576, 20, 100)
+    _topk_case(rng.normal(size=(2, 576)), None, np.array([k, k]))
+
+
+# ------------------------------------------------------------------------------ compaction
+@pytest.mark.parametrize("dtype,H,D", [("bf16", 32, 128), ("f32", 8, 64), ("bf16", 3, 64), ("f32", 2, 128)])
+def test_compaction_bit_exact(dtype, H, D):
+    rng = np.random.default_rng(2)
+    B, T, nv, cap = 3, 150, 110, 256
+    cfg = wl.CONFIGS[1]
+    ctx = _ctx(dtype, H, D, B=B, cap=cap)
+    ks = wl.host_normal(cfg, wl.S_K, (B, T, H, D), dtype=dtype)
+    vs = wl.host_normal(cfg, wl.S_V, (B, T, H, D), dtype=dtype)
+    keep = (rng.random((B, nv)) < 0.3).astype(np.uint8)
+    keep[1] = wl.static_keep_pattern("structure", nv)
+    keep[2] = 0
+    t_src = np.array([T, T - 17, nv + 3], np.int32)
+    start = np.array([0, 5, 40], np.int32)
+    tdt = wl.torch_dtype(dtype)
+    kc = torch.zeros(B, H, cap, D, dtype=tdt, device=DEV)
+    vc = torch.zeros_like(kc)
+    ln = torch.from_numpy(start.copy()).to(DEV)
+    ctx.compact_kv(wl.to_torch(ks, dtype, DEV), wl.to_torch(vs, dtype, DEV), torch.from_numpy(keep).to(DEV),
+                   torch.from_numpy(t_src).to(DEV), kc, vc, ln, commit=True)
+    udt = np.uint32 if dtype == "f32" else np.uint16
+    ok, ov = np.zeros((B, H, cap, D), udt), np.zeros((B, H, cap, D), udt)
+    oln = start.copy()
+    mask = np.ones((B, T), np.uint8)
+    mask[:, :nv] = keep
+    st, _ = orc.append_rows(pc.host_bits(ks, dtype), pc.host_bits(vs, dtype), mask, t_src, ok, ov, oln)
+    assert st == orc.OK
+    assert np.array_equal(ln.cpu().numpy(), oln)
+    gk, gv = pc.dev_bits(kc), pc.dev_bits(vc)
+    for b in range(B):
+        assert np.array_equal(gk[b, :, start[b]:oln[b]], ok[b, :, start[b]:oln[b]])
+        assert np.array_equal(gv[b, :, start[b]:oln[b]], ov[b, :, start[b]:oln[b]])
+        assert not gk[b, :, oln[b]:].any() and not gk[b, :, :start[b]].any()      # nothing written elsewhere
+    assert ctx.device_status()[0] == 0
+
+
+def test_compaction_keep_all_single_tensor_and_capacity():
+    from paper_2412_00876_b200 import binding as dl
+    B, T, H, D, cap = 2, 40, 4, 128, 48
+    cfg = wl.CONFIGS[2]
+    ctx = _ctx("bf16", H, D, B=B, cap=cap)
+    ks = wl.host_normal(cfg, wl.S_K, (B, T, H, D))
+    kc = torch.zeros(B, H, cap, D, dtype=torch.bfloat16, device=DEV)
+    ln = torch.tensor([0, 20], dtype=torch.int32, device=DEV)          # sequence 1: 20 + 40 > 48
+    ctx.compact_kv(wl.to_torch(ks, "bf16", DEV), None, None, None, kc, None, ln, commit=True)
+    assert list(ln.cpu().numpy()) == [T, 20]
+    g = pc.dev_bits(kc)
+    assert np.array_equal(g[0, :, :T], pc.host_bits(ks, "bf16")[0].transpose(1, 0, 2))
+    assert not g[1].any()
+    code, detail = ctx.device_status()
+    assert code == dl.DL_ERR_CAPACITY and detail == 1
+    assert ctx.device_status()[0] == 0                                 # reading clears it
+
+
+# ------------------------------------------------------------------------------ predictor
+@pytest.mark.parametrize("cid,rows", [(1, 144), (2, 576), (2, 7), (4, 33)])
+def test_predictor_scores(cid, rows):
+    from paper_2412_00876_b200 import binding as dl
+    cfg = wl.CONFIGS[cid]
+    p = wl.make_predictor(cfg, "img")
+    x = wl.host_normal(cfg, wl.S_X_VIS, (rows, cfg.hidden))
+    ctx = dl.Context(cfg.hidden, cfg.n_heads, cfg.head_dim, cfg.pred_hidden, wl.torch_dtype(cfg.dtype), 0,
+                     max_batch=1, max_rows=rows, cap=64)
+    pd = dl.Predictor(wl.to_torch(p.w1, cfg.dtype, DEV), torch.from_numpy(p.b1).to(DEV),
+                      torch.from_numpy(p.w2).to(DEV), p.b2)
+    ref = orc.predictor_logits(x, p.w1, p.b1, p.w2, p.b2)
+    for impl in (1, 2):
+        out = torch.zeros(rows, dtype=torch.float32, device=DEV)
+        ctx.set_option(dl.DL_OPT_PREDICTOR_IMPL, impl)
+        try:
+            ctx.predictor_scores(pd, wl.to_torch(x, cfg.dtype, DEV), out)
+        except dl.DlError as e:
+            assert impl == 2 and e.code == dl.DL_ERR_UNSUPPORTED
+            continue
+        err = float(np.abs(out.cpu().numpy() - ref).max())
+        assert err <= pc.LOGIT_TOL, (impl, err)
+        assert err <= 2e-4, (impl, err)          # fp32 accumulation is far inside the tolerance
+
+
+# ------------------------------------------------------------------------------ decode attention
+def _decode_case(dtype, H, D, lens, cap, chunk=0, with_keep=True, seed=0):
+    from paper_2412_00876_b200 import binding as dl
+    B = len(lens)
+    cfg = wl.CONFIGS[2]
+    ctx = _ctx(dtype, H, D, B=B, cap=cap)
+    if chunk:
+        ctx.set_option(dl.DL_OPT_DECODE_CHUNK, chunk)
+    kc = wl.host_normal(cfg, wl.S_CACHE_K, (B, H, cap, D), dtype=dtype, sub=seed)
+    vc = wl.host_normal(cfg, wl.S_CACHE_V, (B, H, cap, D), dtype=dtype, sub=seed)
+    q = wl.host_normal(cfg, wl.S_DEC_Q, (B, H, D), dtype=dtype, sub=seed)
+    kt = wl.host_normal(cfg, wl.S_DEC_K, (B, H, D), dtype=dtype, sub=seed)
+    vt = wl.host_normal(cfg, wl.S_DEC_V, (B, H, D), dtype=dtype, sub=seed)
+    keep = (np.arange(B) % 2).astype(np.uint8)
+    scale = 1 / np.sqrt(D)
+    tdt = wl.torch_dtype(dtype)
+    kc_d, vc_d = wl.to_torch(kc, dtype, DEV), wl.to_torch(vc, dtype, DEV)
+    ln = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    outs = []
+    for rep in range(2):
+        out = torch.zeros(B, H, D, dtype=tdt, device=DEV)
+        ctx.sparse_attn_decode(wl.to_torch(q, dtype, DEV), wl.to_torch(kt, dtype, DEV), wl.to_torch(vt, dtype, DEV),
+                               kc_d, vc_d, ln, torch.from_numpy(keep).to(DEV) if with_keep else None, scale, out)
+        outs.append(out)
+    assert torch.equal(outs[0].view(torch.uint8), outs[1].view(torch.uint8)), "not reproducible"
+    got = wl.from_torch(outs[0])
+    ref = np.empty((B, H, D))
+    for b in range(B):
+        for h in range(H):
+            ref[b, h] = orc.attention_decode_compact(q[b, h], kt[b, h], vt[b, h], kc[b, h], vc[b, h], lens[b], scale)
+    pc.check_att(got, ref, f"decode {dtype} D={D} lens={lens}")
+    # the append: kept sequences have (k_t, v_t) at row len, everything else is untouched
+    gk, gv = pc.dev_bits(kc_d), pc.dev_bits(vc_d)
+    ek, ev = pc.host_bits(kc, dtype).copy(), pc.host_bits(vc, dtype).copy()
+    full = False
+    for b in range(B):
+        if with_keep and keep[b]:
+            if lens[b] < cap:
+                ek[b, :, lens[b]] = pc.host_bits(kt, dtype)[b]
+                ev[b, :, lens[b]] = pc.host_bits(vt, dtype)[b]
+            else:
+                full = True
+    assert np.array_equal(gk, ek) and np.array_equal(gv, ev)
+    assert list(ln.cpu().numpy()) == list(lens)
+    code, _ = ctx.device_status()
+    assert code == (dl.DL_ERR_CAPACITY if full else 0)
+
+
+def test_decode_attention_lengths_and_chunks():
+    _decode_case("bf16", 4, 128, [0, 1, 7, 8, 9, 63, 64, 65], cap=128)
+    _decode_case("bf16", 4, 128, [255, 256, 257, 300, 511, 512, 640, 1], cap=640)            # several chunks
+    _decode_case("bf16", 2, 128, [64, 65, 129, 448, 449, 3], cap=512, chunk=64)             # many chunks
+    _decode_case("bf16", 32, 128, [336, 208, 700, 0, 1000], cap=1024, seed=1)                # more items than SMs
+    _decode_case("bf16", 2, 128, [100, 128], cap=128)                                        # full cache + keep
+
+
+def test_decode_attention_other_types():
+    _decode_case("f32", 8, 64, [0, 68, 132, 5], cap=192)
+    _decode_case("f32", 2, 128, [100, 300], cap=320)
+    _decode_case("bf16", 4, 64, [100, 300, 64], cap=320, with_keep=False)
+
+
+# ------------------------------------------------------------------------------ prefill attention
+@pytest.mark.parametrize("dtype,H,D,lens", [("f32", 8, 64, [68]), ("bf16", 4, 128, [208, 1, 130, 64]),
+                                             ("bf16", 2, 64, [33, 100]), ("f32", 2, 128, [40, 7])])
+def test_prefill_attention(dtype, H, D, lens):
+    from paper_2412_00876_b200 import binding as dl
+    B, cap = len(lens), (max(lens) + 63) // 64 * 64
+    cfg = wl.CONFIGS[2]
+    q = wl.host_normal(cfg, wl.S_Q, (B, H, cap, D), dtype=dtype)
+    k = wl.host_normal(cfg, wl.S_K, (B, H, cap, D), dtype=dtype)
+    v = wl.host_normal(cfg, wl.S_V, (B, H, cap, D), dtype=dtype)
+    scale = 1 / np.sqrt(D)
+    n_max = max(lens)
+    for impl in (1, 2):
+        ctx = _ctx(dtype, H, D, B=B, cap=cap)
+        ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, impl)
+        out = torch.full((B, n_max, H, D), 7.0, dtype=wl.torch_dtype(dtype), device=DEV)
+        try:
+            ctx.sparse_attn_prefill(wl.to_torch(q, dtype, DEV), wl.to_torch(k, dtype, DEV), wl.to_torch(v, dtype, DEV),
+                                    torch.tensor(lens, dtype=torch.int32, device=DEV), n_max, scale, out)
+        except dl.DlError as e:
+            assert impl == 2 and e.code == dl.DL_ERR_UNSUPPORTED
+            continue
+        got = wl.from_torch(out)
+        for b in range(B):
+            n = lens[b]
+            ref = np.stack([orc.attention_prefill_compact(q[b, h], k[b, h], v[b, h], n, scale) for h in range(H)], 1)
+            pc.check_att(got[b, :n], ref, f"prefill impl {impl} seq {b}")
+            assert np.all(got[b, n:] == 7.0)                  # rows past the length are not written
