@@ -34,7 +34,7 @@ __device__ __forceinline__ void report_status(DeviceStatus* st, int32_t code, lo
 // Workspace layout (all offsets 256-byte aligned).
 // ---------------------------------------------------------------------------------------
 constexpr int kDecodeMinChunk = 64;   // smallest rows-per-item the decode kernel may be asked for
-constexpr int kPredMaxSplit = 32;     // most column splits of the predictor's hidden layer
+constexpr int kPredMaxSplit = 80;     // most unit tiles of the predictor's hidden layer
 constexpr int kPredRowTile = 128;     // rows per predictor row tile (tensor-core kernel)
 
 struct Workspace {
