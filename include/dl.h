@@ -202,6 +202,37 @@ int32_t dl_decode_step_host(dl_ctx* ctx, const dl_predictor* p_txt, const void* 
                             void* const* v_caches, int32_t cap, int32_t* cache_len, float scale,
                             void* stream);
 
+/* ---- decode attention without any allocation ------------------------------------------- */
+
+/* Size of the library's built-in scratch array (bytes). */
+#define DL_STATIC_SCRATCH_BYTES (8u << 20)
+
+/* The paper has no counterpart to this call; it exists for integration reasons only.
+ *
+ * Same computation, arguments and results as dl_sparse_attn_decode, for callers that must not
+ * allocate device memory: code running inside another framework's memory pool or under a fixed
+ * memory budget, plugins that are handed their buffers and nothing else, or processes that are
+ * already close to the device's capacity and cannot afford a failing cudaMalloc.  Such callers
+ * have no workspace to give to dl_set_workspace; here the split partials and arrival tickets
+ * live in a fixed array of DL_STATIC_SCRATCH_BYTES that is part of the library image (each GPU
+ * that loads the library holds it until the process exits).  The context needs no workspace;
+ * without one, device-side conditions (a full cache on append) are skipped silently instead
+ * of being recorded.
+ *
+ *   - Needs  B*H*4 (rounded up to 256) + B*H*(cap/chunk + 2)*(D+2)*4  bytes of that array
+ *     (chunk = 256 rows unless DL_OPT_DECODE_CHUNK says otherwise); a larger problem is refused
+ *     with DL_ERR_WORKSPACE and nothing is launched.
+ *   - The first call on a device looks the array's device address up (cudaGetSymbolAddress, with
+ *     that device current); make that first call outside any stream capture.
+ *   - The call issues one asynchronous memset (the tickets must start at zero; the array keeps
+ *     the previous call's contents) and one kernel on `stream`.  It calls no cudaMalloc/cudaFree.
+ *   - All calls on a device share the one array: two calls that may overlap on the GPU (different
+ *     streams, or different contexts) race on it.  Serialise them on one stream. */
+int32_t dl_sparse_attn_decode_static(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t,
+                                     void* k_cache, void* v_cache, const int32_t* cache_len,
+                                     const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
+                                     void* stream);
+
 #ifdef __cplusplus
 }
 #endif

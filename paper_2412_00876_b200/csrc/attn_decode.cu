@@ -413,3 +413,89 @@ cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t
 }
 
 }  // namespace dl
+
+// =================================================================================================
+// dl_sparse_attn_decode_static: the same kernel for callers that cannot allocate device memory.
+//
+// Its scratch (split partials and arrival tickets) lives in the fixed array below instead of a
+// caller-provided workspace.  Every GPU that loads this library holds the array until the process
+// exits.  In host code `g_static_scratch` is only a handle for the runtime, not a device address:
+// the address is obtained once per device with cudaGetSymbolAddress while that device is current.
+// =================================================================================================
+namespace dl {
+
+constexpr size_t kStaticScratchBytes = DL_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_static_ptr[kMaxDevices];       // device address of g_static_scratch, per device (0 = not set up)
+
+// Looks the array's device address up (first call on this device) or returns the cached one.
+static cudaError_t static_scratch_for(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  void* p = __atomic_load_n(&g_static_ptr[device], __ATOMIC_ACQUIRE);
+  if (p == nullptr) {
+    int prev = -1;
+    cudaError_t e = cudaGetDevice(&prev);
+    if (e != cudaSuccess) return e;
+    if (prev != device && (e = cudaSetDevice(device)) != cudaSuccess) return e;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (prev != device) cudaSetDevice(prev);
+    if (e != cudaSuccess) return e;
+    __atomic_store_n(&g_static_ptr[device], p, __ATOMIC_RELEASE);
+  }
+  *out = p;
+  return cudaSuccess;
+}
+
+}  // namespace dl
+
+extern "C" int32_t dl_sparse_attn_decode_static(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t,
+                                                void* k_cache, void* v_cache, const int32_t* cache_len,
+                                                const uint8_t* keep, int32_t B, int32_t cap, float scale,
+                                                void* out, void* stream) {
+  using namespace dl;
+  if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
+  if (B == 0) return DL_OK;
+  if (!q_t || !k_t || !v_t || !k_cache || !v_cache || !cache_len || !out) return DL_ERR_INVALID_ARG;
+  const uintptr_t all = (uintptr_t)q_t | (uintptr_t)k_t | (uintptr_t)v_t | (uintptr_t)k_cache |
+                        (uintptr_t)v_cache | (uintptr_t)out;
+  if (all & 15u) return DL_ERR_ALIGNMENT;
+  if (B > kMaxDecodeBatch) return DL_ERR_UNSUPPORTED;
+  const dl_model_desc& d = ctx->desc;
+  int chunk = ctx->opt.decode_chunk > 0 ? ctx->opt.decode_chunk : 256;
+  chunk = max(kDecodeMinChunk, (chunk + kStageRows - 1) / kStageRows * kStageRows);
+  const int slots = (cap + chunk - 1) / chunk + 1;
+  // layout inside the array: tickets [B*H] int32 (256-byte padded) | partials [B*H*slots*(D+2)] float
+  const size_t ticket_bytes = ((size_t)B * d.n_heads * sizeof(int32_t) + 255) & ~size_t(255);
+  const size_t partial_bytes = (size_t)B * d.n_heads * slots * (d.head_dim + 2) * sizeof(float);
+  if (ticket_bytes + partial_bytes > kStaticScratchBytes) return DL_ERR_WORKSPACE;   // beyond the fixed maximum
+
+  void* base = nullptr;
+  cudaError_t e = static_scratch_for(ctx->device, &base);
+  if (e != cudaSuccess) { ctx->last_cuda = e; return DL_ERR_CUDA; }
+  int prev = -1;
+  cudaGetDevice(&prev);
+  if (prev != ctx->device) cudaSetDevice(ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // the array keeps whatever the last call left: the tickets must start at zero
+  e = cudaMemsetAsync(base, 0, ticket_bytes, s);
+  if (e == cudaSuccess) {
+    DecodeArgs a;
+    a.q = q_t; a.k_t = k_t; a.v_t = v_t; a.k_cache = k_cache; a.v_cache = v_cache;
+    a.cache_len = cache_len; a.keep = keep; a.out = out;
+    a.ticket = static_cast<int32_t*>(base);
+    a.partial = reinterpret_cast<float*>(static_cast<char*>(base) + ticket_bytes);
+    a.status = ctx->ws.base ? ctx->ws.status : nullptr;
+    a.B = B; a.H = d.n_heads; a.cap = cap; a.chunk = chunk; a.slots = slots; a.n_stages = 0;
+    a.scale_log2 = scale * 1.4426950408889634f;
+    if (d.dtype == DL_BF16 && d.head_dim == 128) e = launch_t<__nv_bfloat16, 128>(ctx, a, s);
+    else if (d.dtype == DL_BF16 && d.head_dim == 64) e = launch_t<__nv_bfloat16, 64>(ctx, a, s);
+    else if (d.dtype == DL_F32 && d.head_dim == 128) e = launch_t<float, 128>(ctx, a, s);
+    else if (d.dtype == DL_F32 && d.head_dim == 64) e = launch_t<float, 64>(ctx, a, s);
+    else e = cudaErrorInvalidValue;
+  }
+  if (prev != ctx->device) cudaSetDevice(prev);
+  if (e != cudaSuccess) { ctx->last_cuda = e; return DL_ERR_CUDA; }
+  return DL_OK;
+}
