@@ -37,7 +37,96 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-every", type=int, default=64, help="decode steps between timed attention launches")
+    ap.add_argument("--micro", default="", choices=["", "decode", "predictor", "compact", "prefill"],
+                    help="time one stage alone on the config's shapes (small memory; used for ncu captures)")
+    ap.add_argument("--micro-layers", type=int, default=2, help="layers of cache / source held in --micro mode")
+    ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
     return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------ single-stage timing
+def micro(args):
+    """Times one kernel family alone, launches rotating over `micro_layers` independent buffers so
+    that consecutive launches never find their inputs in L2.  Prints one JSON line."""
+    import numpy as np
+    import torch
+    from paper_2412_00876_b200 import binding as dl
+    from paper_2412_00876_b200 import build as dl_build
+    from paper_2412_00876_b200 import workloads as wl
+    dl_build.build()
+    cfg = wl.CONFIGS[args.config]
+    dev = torch.device("cuda", 0)
+    B, H, D, NL = cfg.B, cfg.n_heads, cfg.head_dim, args.micro_layers
+    tdt = wl.torch_dtype(cfg.dtype)
+    rows = B * cfg.n_vis
+    ctx = dl.Context(cfg.hidden, H, D, cfg.pred_hidden, tdt, 0, max_batch=B, max_rows=rows, cap=cfg.cap)
+    scale = 1.0 / float(np.sqrt(D))
+    i32 = dict(dtype=torch.int32, device=dev)
+    work, unit, calls = 0.0, "GB/s", []
+    if args.micro == "decode":
+        n = args.micro_len or min(cfg.cap - 1, cfg.n0 + int(cfg.n_gen * cfg.keep_rate))
+        kc = [wl.device_normal(cfg, wl.S_CACHE_K, (B, H, cfg.cap, D), dev, sub=i) for i in range(NL)]
+        vc = [wl.device_normal(cfg, wl.S_CACHE_V, (B, H, cfg.cap, D), dev, sub=i) for i in range(NL)]
+        q = wl.device_normal(cfg, wl.S_DEC_Q, (NL, B, H, D), dev)
+        kt = wl.device_normal(cfg, wl.S_DEC_K, (NL, B, H, D), dev)
+        vt = wl.device_normal(cfg, wl.S_DEC_V, (NL, B, H, D), dev)
+        out = torch.empty(NL, B, H, D, dtype=tdt, device=dev)
+        lens = np.clip(n + wl.host_rng(cfg.cid, wl.S_LEN).integers(-16, 17, B), 0, cfg.cap - 1).astype(np.int32)
+        ln = torch.from_numpy(lens).to(dev)
+        keep = torch.ones(B, dtype=torch.uint8, device=dev)
+        work = (2 * (int(lens.sum()) + B) + 2 * B) * H * D * cfg.elt_bytes
+        calls = [lambda l=l: ctx.sparse_attn_decode(q[l], kt[l], vt[l], kc[l], vc[l], ln, keep, scale, out[l])
+                 for l in range(NL)]
+    elif args.micro == "predictor":
+        p = wl.make_predictor(cfg, "img")
+        pd = dl.Predictor(wl.to_torch(p.w1, cfg.dtype, dev), torch.from_numpy(p.b1).to(dev),
+                          torch.from_numpy(p.w2).to(dev), p.b2)
+        xs = [wl.device_normal(cfg, wl.S_X_VIS, (rows, cfg.hidden), dev, sub=i) for i in range(NL)]
+        out = torch.empty(rows, dtype=torch.float32, device=dev)
+        work, unit = 2.0 * rows * cfg.hidden * cfg.pred_hidden, "TFLOP/s"
+        calls = [lambda l=l: ctx.predictor_scores(pd, xs[l], out) for l in range(NL)]
+    elif args.micro in ("compact", "prefill"):
+        T = cfg.n_vis + cfg.n_text
+        src = [wl.device_normal(cfg, wl.S_K, (B, T, H, D), dev, sub=i) for i in range(2 * NL)]
+        kc = [torch.empty(B, H, cfg.cap, D, dtype=tdt, device=dev) for _ in range(NL)]
+        vc = [torch.empty(B, H, cfg.cap, D, dtype=tdt, device=dev) for _ in range(NL)]
+        keep = torch.zeros(B, cfg.n_vis, dtype=torch.uint8, device=dev)
+        idx = torch.stack([torch.randperm(cfg.n_vis, device=dev)[: cfg.k_vis] for _ in range(B)])
+        keep.scatter_(1, idx, 1)
+        t_src = torch.full((B,), T, **i32)
+        ln = torch.zeros(B, **i32)
+        zero = torch.zeros(B, **i32)
+        if args.micro == "compact":
+            work = 2 * 2 * B * cfg.n0 * H * D * cfg.elt_bytes          # K and V: kept rows read + written
+            calls = [lambda l=l: (ln.copy_(zero), ctx.compact_kv(src[2 * l], src[2 * l + 1], keep, t_src, kc[l],
+                                                                vc[l], ln, commit=True)) for l in range(NL)]
+        else:
+            for l in range(NL):
+                ln.zero_()
+                ctx.compact_kv(src[2 * l], src[2 * l + 1], keep, t_src, kc[l], vc[l], ln, commit=True)
+            out = torch.empty(B, cfg.n0, H, D, dtype=tdt, device=dev)
+            work, unit = 2.0 * D * cfg.n0 * (cfg.n0 + 1) * H * B, "TFLOP/s"
+            calls = [lambda l=l: ctx.sparse_attn_prefill(kc[l], kc[l], vc[l], ln, cfg.n0, scale, out)
+                     for l in range(NL)]
+    for i in range(args.warmup):
+        calls[i % NL]()
+    torch.cuda.synchronize()
+    ev = []
+    for i in range(args.steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        calls[i % NL]()
+        b.record()
+        ev.append((a, b))
+    torch.cuda.synchronize()
+    ts = sorted(a.elapsed_time(b) for a, b in ev)
+    med = ts[len(ts) // 2]
+    code, detail = ctx.device_status()
+    rate = work / (med * 1e-3) / (1e9 if unit == "GB/s" else 1e12)
+    print(json.dumps({"micro": args.micro, "workload": cfg.name, "median_us": med * 1e3, "min_us": ts[0] * 1e3,
+                      "algorithmic_work": work, "rate": rate, "unit": unit, "launches": args.steps,
+                      "device_status": code}), flush=True)
+    ctx.close()
 
 
 # ------------------------------------------------------------------------------ clocks
@@ -183,6 +272,8 @@ def main():
     args = parse()
     if args.impl == "reference":
         return reference_arm(args)
+    if args.micro:
+        return micro(args)
     import torch
     import torch.distributed as dist
     from paper_2412_00876_b200 import build as dl_build

@@ -53,7 +53,8 @@ enum {
 enum {
   DL_OPT_PREDICTOR_IMPL = 1,    /* 0 auto, 1 CUDA-core kernel, 2 tcgen05 tensor-core kernel (bf16) */
   DL_OPT_PREFILL_ATTN_IMPL = 2, /* 0 auto, 1 CUDA-core kernel, 2 tcgen05 tensor-core kernel (bf16, D=128) */
-  DL_OPT_DECODE_CHUNK = 3       /* cache rows per decode work item (0 = default) */
+  DL_OPT_DECODE_CHUNK = 3,      /* cache rows per decode work item (0 = chosen by the library) */
+  DL_OPT_DECODE_IMPL = 4        /* 0 auto, 1 CUDA-core kernel, 2 tensor-core (mma.sync) kernel (bf16, D=128) */
 };
 
 typedef struct {
@@ -219,9 +220,11 @@ int32_t dl_decode_step_host(dl_ctx* ctx, const dl_predictor* p_txt, const void* 
  * without one, device-side conditions (a full cache on append) are skipped silently instead
  * of being recorded.
  *
- *   - Needs  B*H*4 (rounded up to 256) + B*H*(cap/chunk + 2)*(D+2)*4  bytes of that array
- *     (chunk = 256 rows unless DL_OPT_DECODE_CHUNK says otherwise); a larger problem is refused
- *     with DL_ERR_WORKSPACE and nothing is launched.
+ *   - Needs  B*H*4 (rounded up to 256) + B*H*(c + 1)*(D+2)*4  bytes of that array, where c is
+ *     the largest number of pieces one sequence may be split into: min(cap/64, max(1, W/(B*H)))
+ *     with W = 8 warps per SM of the device (16 for fp32 or head_dim 64), or ceil(cap/chunk)
+ *     when DL_OPT_DECODE_CHUNK is set.  Large batches are not split (c = 1).  A larger problem
+ *     is refused with DL_ERR_WORKSPACE and nothing is launched.
  *   - The first call on a device looks the array's device address up (cudaGetSymbolAddress, with
  *     that device current); make that first call outside any stream capture.
  *   - The call issues one asynchronous memset (the tickets must start at zero; the array keeps

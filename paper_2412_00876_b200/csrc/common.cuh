@@ -60,6 +60,7 @@ struct Options {
   int32_t predictor_impl = 0;
   int32_t prefill_attn_impl = 0;
   int32_t decode_chunk = 0;
+  int32_t decode_impl = 0;
 };
 
 }  // namespace dl
@@ -73,6 +74,11 @@ struct dl_ctx {
   int32_t smem_optin = 0;
   cudaError_t last_cuda = cudaSuccess;
   void* tmap_encode = nullptr;        // cuTensorMapEncodeTiled, resolved at create
+  // tensor maps of cache tensors seen before (decode attention); see attn_decode.cu
+  static constexpr int kMapCache = 256;
+  struct MapEntry { const void* base = nullptr; long long rows = 0; unsigned char map[128]; };
+  mutable MapEntry map_cache[kMapCache];
+  mutable int map_next = 0;
 };
 
 namespace dl {

@@ -53,7 +53,7 @@ def test_static_scratch_variant_matches_workspace_variant_twice():
 
 def test_static_scratch_variant_refuses_problems_beyond_its_array():
     from paper_2412_00876_b200 import binding as dl
-    B, H, D, cap = 64, 32, 128, 4096                 # 64*32*(4096/256+1)*130*4 B = 18 MB > 8 MiB
+    B, H, D, cap = 512, 32, 128, 4096                # 512*32 (b,h) pairs * 2 slots * 130 floats = 17 MB > 8 MiB
     ctx = dl.Context(256, H, D, 64, torch.bfloat16, 0, max_batch=1, max_rows=1, cap=64)
     t = torch.zeros(16, dtype=torch.bfloat16, device=DEV)          # never dereferenced: the call is refused
     ln = torch.zeros(B, dtype=torch.int32, device=DEV)
