@@ -339,7 +339,7 @@ def main():
     else:
         peak, peak_src = 6650.0, "fallback"
     achieved = tot_bytes / (tot_ms * 1e-3) / 1e9 if tot_ms > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "attn_decode_kernel", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "attn_decode_mma_kernel", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
                 "launches_timed": len(events),
                 "avg_launch_us": 1e3 * tot_ms / max(len(events), 1),

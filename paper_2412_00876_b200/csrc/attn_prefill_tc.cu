@@ -1,9 +1,291 @@
-// Tensor-core prefill attention (tcgen05): placeholder until the kernel lands.
+// Prefill attention over the reduced set on the tensor cores (Eq. 1 applied to S^{P*}):
+// row i of a sequence's compact context attends rows 0..i of the same context.
+// bf16, head_dim 128.  One CTA per (sequence, head, 128-row query tile); two CTAs share an SM so
+// that one CTA's softmax overlaps the other's MMAs.
+//   warp 0    : TMA producer.  Q once (two 64-dim halves), then 64-row K and V tiles through a
+//               2-stage ring, all with the 128-byte swizzle;
+//   warp 1    : tensor-memory allocation and the single MMA-issuing thread:
+//               S = Q K^T (128 x 64, K-major operands from shared memory) into one of two S buffers,
+//               O += P V (P read from tensor memory, V as an MN-major shared-memory operand);
+//               the next tile's Q K^T is issued before this tile's P V so it runs during the softmax;
+//   warps 2-5 : softmax, one query row per thread, straight out of tensor memory.  The running
+//               maximum is only raised when it grows by more than 2^8 (then O is rescaled in tensor
+//               memory), so most tiles never touch O.  P (bf16) overwrites the first half of its
+//               own S buffer.  The same warps normalise O and store the output rows.
+// Tensor memory: O 128 columns, S0 and S1 64 columns each (256 columns per CTA, 512 per SM).
+// Rows past a sequence's length are fetched with the tile (they are masked); in the last tile the
+// surplus V rows are zeroed in shared memory first, since 0 * x must stay 0 for any bit pattern.
+// Every wait is bounded (pipeline.cuh); an abort leaves DL_ERR_TIMEOUT in the status word.
 #include "common.cuh"
+#include "tc05.cuh"
+
 namespace dl {
-bool attn_prefill_tc_supported(const dl_ctx*) { return false; }
-cudaError_t launch_attn_prefill_tc(dl_ctx*, const void*, const void*, const void*, const int32_t*, int32_t,
-                                   int32_t, int32_t, float, void*, cudaStream_t) {
-  return cudaErrorNotSupported;
+
+constexpr int kAtBM = 128, kAtBN = 64, kAtStages = 2, kAtThreads = 192;
+constexpr int kAtQBytes = 2 * kAtBM * 128;            // 32 KB: two [128 rows][64 dims] halves
+constexpr int kAtTile = 2 * kAtBN * 128;              // 16 KB: two [64 rows][64 dims] halves
+constexpr int kAtStage = 2 * kAtTile;                 // K tile + V tile
+constexpr size_t kAtSmem = kAtQBytes + kAtStages * kAtStage + 1024 + 256;
+constexpr uint32_t kAtColO = 0, kAtColS = 128;        // tensor-memory columns: O | S0 | S1
+constexpr float kRescaleStep = 8.0f;                  // log2 units by which the maximum may lag
+
+struct AtMaps { alignas(64) unsigned char q[128]; alignas(64) unsigned char k[128]; alignas(64) unsigned char v[128]; };
+
+struct AtArgs {
+  const int32_t* cache_len; __nv_bfloat16* out; DeviceStatus* status;
+  int32_t H, cap, n_max;
+  float scale_log2;
+};
+
+__global__ void __launch_bounds__(kAtThreads, 2)
+attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
+  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int n = min(max(a.cache_len[b], 0), min(a.cap, a.n_max));
+  const int q0 = qt * kAtBM;
+  if (q0 >= n) return;
+  const int kv_end = min(n, q0 + kAtBM);                         // keys any row of this tile may see
+  const int n_tiles = (kv_end + kAtBN - 1) / kAtBN;
+  const int row_base = (b * a.H + h) * a.cap;                    // first row of this (b, h) in the caches
+
+  extern __shared__ char smem_raw[];
+  char* smem = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  char* q_s = smem;
+  char* st_s = smem + kAtQBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(st_s + kAtStages * kAtStage);
+  uint64_t* q_full = bars;                 // [1]
+  uint64_t* kv_full = bars + 1;            // [2]
+  uint64_t* kv_empty = bars + 3;           // [2]
+  uint64_t* s_full = bars + 5;             // [2]
+  uint64_t* p_full = bars + 7;             // [2]
+  uint64_t* pv_done = bars + 9;            // [1]
+  __shared__ uint32_t sh_tmem;
+  __shared__ int sh_abort;
+  volatile int* abort_flag = &sh_abort;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    sh_abort = 0;
+    mbar_init(smem_u32(q_full), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&kv_full[i]), 1);
+      mbar_init(smem_u32(&kv_empty[i]), 1);
+      mbar_init(smem_u32(&s_full[i]), 1);
+      mbar_init(smem_u32(&p_full[i]), 4);
+    }
+    mbar_init(smem_u32(pv_done), 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(&sh_tmem), 256); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh_tmem;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(maps.q);
+      const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(maps.k);
+      const CUtensorMap* mv = reinterpret_cast<const CUtensorMap*>(maps.v);
+      mbar_expect_tx(smem_u32(q_full), kAtQBytes);
+      tma_load_2d(smem_u32(q_s), mq, 0, row_base + q0, smem_u32(q_full));
+      tma_load_2d(smem_u32(q_s + kAtBM * 128), mq, 64, row_base + q0, smem_u32(q_full));
+      int issued = 0;
+      for (int j = 0; j < n_tiles && !*abort_flag; ++j, ++issued) {
+        const int s = j % kAtStages;
+        if (!mbar_wait(smem_u32(&kv_empty[s]), ((j / kAtStages) & 1) ^ 1, abort_flag)) break;
+        const uint32_t fb = smem_u32(&kv_full[s]);
+        mbar_expect_tx(fb, kAtStage);
+        char* st = st_s + (size_t)s * kAtStage;
+        const int r = row_base + j * kAtBN;
+        tma_load_2d(smem_u32(st), mk, 0, r, fb);
+        tma_load_2d(smem_u32(st + kAtBN * 128), mk, 64, r, fb);
+        tma_load_2d(smem_u32(st + kAtTile), mv, 0, r, fb);
+        tma_load_2d(smem_u32(st + kAtTile + kAtBN * 128), mv, 64, r, fb);
+      }
+      if (*abort_flag) {
+        report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
+        for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(q_full), 0); ++i) __nanosleep(40);
+        for (int j = max(0, issued - kAtStages); j < issued; ++j)
+          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&kv_full[j % kAtStages]), (j / kAtStages) & 1); ++i)
+            __nanosleep(40);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_qk = idesc_bf16(kAtBM, kAtBN);
+      const uint32_t idesc_pv = idesc_bf16(kAtBM, 128, 0, 1);        // B (= V) is MN-major
+      const uint32_t q_addr = smem_u32(q_s);
+      auto issue_qk = [&](int j) {
+        const int s = j % kAtStages;
+        mbar_wait(smem_u32(&kv_full[s]), (j / kAtStages) & 1, abort_flag);
+        tc_fence_after();
+        const uint32_t k_addr = smem_u32(st_s + (size_t)s * kAtStage);
+        const uint32_t d = tmem + kAtColS + (uint32_t)(j & 1) * kAtBN;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          mma_ss(d, smem_desc_sw128(q_addr + (ks >> 2) * (kAtBM * 128) + (ks & 3) * 32),
+                 smem_desc_sw128(k_addr + (ks >> 2) * (kAtBN * 128) + (ks & 3) * 32), idesc_qk, ks != 0);
+        mma_commit(smem_u32(&s_full[j & 1]));
+      };
+      mbar_wait(smem_u32(q_full), 0, abort_flag);
+      issue_qk(0);
+      for (int j = 0; j < n_tiles; ++j) {
+        if (j + 1 < n_tiles) issue_qk(j + 1);
+        const int s = j % kAtStages;
+        mbar_wait(smem_u32(&p_full[j & 1]), (j >> 1) & 1, abort_flag);
+        tc_fence_after();
+        const uint32_t v_addr = smem_u32(st_s + (size_t)s * kAtStage + kAtTile);
+        const uint32_t p_tmem = tmem + kAtColS + (uint32_t)(j & 1) * kAtBN;
+#pragma unroll
+        for (int ks = 0; ks < kAtBN / 16; ++ks)
+          mma_ts(tmem + kAtColO, p_tmem + ks * 8, smem_desc_sw128_mn(v_addr + ks * 2048, kAtBN * 128), idesc_pv,
+                 (j | ks) != 0);
+        mma_commit(smem_u32(&kv_empty[s]));
+        mma_commit(smem_u32(pv_done));
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax / epilogue warps
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;                                  // row within the query tile
+    const int grow = q0 + row;                                         // row within the sequence
+    const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+    float m_used = -INFINITY, l_run = 0.f;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int sb = j & 1;
+      mbar_wait(smem_u32(&s_full[sb]), (j >> 1) & 1, abort_flag);
+      tc_fence_after();
+      const uint32_t s_addr = tmem + lane_off + kAtColS + (uint32_t)sb * kAtBN;
+      uint32_t sr[64];
+      tmem_ld32(s_addr, sr);
+      tmem_ld32(s_addr + 32, sr + 32);
+      tmem_ld_wait();
+      const int c0 = j * kAtBN;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 64; ++c) {
+        float v = __uint_as_float(sr[c]) * a.scale_log2;
+        v = (c0 + c > grow) ? -INFINITY : v;
+        sr[c] = __float_as_uint(v);
+        mx = fmaxf(mx, v);
+      }
+      if (j == 0) {
+        m_used = mx;                        // column 0 is visible to every row, so mx is finite
+      } else {
+        const bool need = mx > m_used + kRescaleStep;
+        if (__any_sync(0xffffffffu, need)) {
+          mbar_wait(smem_u32(pv_done), (j - 1) & 1, abort_flag);      // O must be at rest
+          tc_fence_after();
+          const float corr = need ? exp2f(m_used - mx) : 1.0f;
+          if (need) m_used = mx;
+          l_run *= corr;
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) {
+            uint32_t o[32];
+            tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
+            tmem_st32(tmem + lane_off + kAtColO + cc * 32, o);
+          }
+          tmem_st_wait();
+        }
+      }
+      uint32_t pw[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        const float p0 = exp2f(__uint_as_float(sr[2 * c]) - m_used);
+        const float p1 = exp2f(__uint_as_float(sr[2 * c + 1]) - m_used);
+        l_run += p0 + p1;
+        __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+        pw[c] = *reinterpret_cast<uint32_t*>(&pk);
+      }
+      tmem_st32(s_addr, pw);                                             // P overwrites its own S buffer
+      tmem_st_wait();
+      if (j == n_tiles - 1 && kv_end < c0 + kAtBN) {
+        // ragged last tile: zero the V rows past the sequence's end (both 64-dim halves)
+        const int s = j % kAtStages;
+        mbar_wait(smem_u32(&kv_full[s]), (j / kAtStages) & 1, abort_flag);
+        char* vz = st_s + (size_t)s * kAtStage + kAtTile;
+        const int first = kv_end - c0;
+        for (int u = (warp - 2) * 32 + lane; u < 2 * kAtBN * 8; u += 128) {
+          const int r = (u >> 3) & (kAtBN - 1);
+          if (r >= first)
+            *reinterpret_cast<uint4*>(vz + (u >> 9) * (kAtBN * 128) + r * 128 + (u & 7) * 16) = make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&p_full[sb]));
+    }
+    // ---- epilogue: O / l -> bf16 -> out[b][row][h][:]
+    mbar_wait(smem_u32(pv_done), (n_tiles - 1) & 1, abort_flag);
+    tc_fence_after();
+    const float inv = 1.0f / l_run;
+    __nv_bfloat16* orow = a.out + (((size_t)b * a.n_max + grow) * a.H + h) * 128;
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+      uint32_t o[32];
+      tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
+      tmem_ld_wait();
+      if (grow < n) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 8) {
+          uint4 w;
+          __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+          __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+          __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+          __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+          w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
+          w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
+          *reinterpret_cast<uint4*>(orow + cc * 32 + i) = w;
+        }
+      }
+    }
+    if (*abort_flag && row == 0) report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 256); }
 }
+
+bool attn_prefill_tc_supported(const dl_ctx* ctx) {
+  const dl_model_desc& d = ctx->desc;
+  return d.dtype == DL_BF16 && d.head_dim == 128 && ctx->tmap_encode != nullptr && (size_t)ctx->smem_optin >= kAtSmem;
+}
+
+cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                                   const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max, float scale,
+                                   void* out, cudaStream_t s) {
+  if (B == 0 || n_max == 0) return cudaSuccess;
+  const dl_model_desc& d = ctx->desc;
+  const long long rows = (long long)B * d.n_heads * cap;
+  if (rows >= (1LL << 31)) return cudaErrorInvalidValue;
+  AtMaps maps;
+  const uint64_t dims[2] = {128ull, (uint64_t)rows};
+  const uint64_t strides[1] = {256ull};
+  const uint32_t box_q[2] = {64u, (uint32_t)kAtBM};
+  const uint32_t box_kv[2] = {64u, (uint32_t)kAtBN};
+  if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.q), q, 2, dims, strides, box_q) ||
+      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.k), k_cache, 2, dims, strides, box_kv) ||
+      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.v), v_cache, 2, dims, strides, box_kv))
+    return cudaErrorInvalidValue;
+  AtArgs a;
+  a.cache_len = cache_len; a.out = static_cast<__nv_bfloat16*>(out); a.status = ctx->ws.base ? ctx->ws.status : nullptr;
+  a.H = d.n_heads; a.cap = cap; a.n_max = n_max;
+  a.scale_log2 = scale * 1.4426950408889634f;
+  static int attr_set[64];
+  if (!attr_set[ctx->device & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
+    if (e != cudaSuccess) return e;
+    attr_set[ctx->device & 63] = 1;
+  }
+  dim3 grid((n_max + kAtBM - 1) / kAtBM, d.n_heads, B);
+  attn_prefill_tc_kernel<<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
+  return cudaGetLastError();
+}
+
 }  // namespace dl

@@ -118,10 +118,20 @@ class BatchRunner:
         self.launches += 3 + c.n_layers
 
     def run_batch(self, sample_every: int = 0, events: list | None = None):
+        """One whole batch.  With `sample_every`, every sample_every-th decode step is issued call by
+        call with events around its attention launches; the prefill and those steps sit inside an
+        NVTX range ("dl_sample") so that a profiler can be told to look at them only."""
+        nvtx = torch.cuda.nvtx
+        if sample_every:
+            nvtx.range_push("dl_sample")
         self.prefill()
+        if sample_every:
+            nvtx.range_pop()
         for t in range(self.cfg.n_gen):
             if sample_every and events is not None and t % sample_every == sample_every - 1:
+                nvtx.range_push("dl_sample")
                 self.decode_step_timed(t, events)
+                nvtx.range_pop()
             else:
                 self.decode_step(t)
 
