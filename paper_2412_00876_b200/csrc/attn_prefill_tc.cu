@@ -57,7 +57,8 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
   uint64_t* kv_empty = bars + 3;           // [2]
   uint64_t* s_full = bars + 5;             // [2]
   uint64_t* p_full = bars + 7;             // [2]
-  uint64_t* pv_done = bars + 9;            // [1]
+  uint64_t* pv_done = bars + 9;            // [1] one phase per tile: P V of tile j has completed
+  uint64_t* o_final = bars + 10;           // [1] single phase: the last P V has completed
   __shared__ uint32_t sh_tmem;
   __shared__ int sh_abort;
   volatile int* abort_flag = &sh_abort;
@@ -73,6 +74,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       mbar_init(smem_u32(&p_full[i]), 4);
     }
     mbar_init(smem_u32(pv_done), 1);
+    mbar_init(smem_u32(o_final), 1);
     fence_mbar_init();
   }
   if (warp == 1) { tmem_alloc(smem_u32(&sh_tmem), 256); tmem_relinquish(); }
@@ -144,6 +146,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
                  (j | ks) != 0);
         mma_commit(smem_u32(&kv_empty[s]));
         mma_commit(smem_u32(pv_done));
+        if (j == n_tiles - 1) mma_commit(smem_u32(o_final));
       }
     }
   } else {
@@ -222,7 +225,9 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       if (lane == 0) mbar_arrive(smem_u32(&p_full[sb]));
     }
     // ---- epilogue: O / l -> bf16 -> out[b][row][h][:]
-    mbar_wait(smem_u32(pv_done), (n_tiles - 1) & 1, abort_flag);
+    // (a parity wait on pv_done would be ambiguous here: a warp can get here while the P V of the
+    //  tile before the last is still running, two phases behind)
+    mbar_wait(smem_u32(o_final), 0, abort_flag);
     tc_fence_after();
     const float inv = 1.0f / l_run;
     __nv_bfloat16* orow = a.out + (((size_t)b * a.n_max + grow) * a.H + h) * 128;
