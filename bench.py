@@ -280,29 +280,21 @@ def main():
     from paper_2412_00876_b200 import workloads as wl
     from paper_2412_00876_b200.runner import BatchRunner
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2412_00876_b200 import dist_util as du
+    world, rank, local = du.env_world()
     if rank == 0:
         dl_build.build()
     torch.cuda.set_device(local)
     if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-        dist.barrier()
+        du.init("nccl", local)
+        du.barrier()                       # the other ranks load the library only after rank 0 has built it
     cfg = wl.CONFIGS[args.config]
     runner = BatchRunner(cfg, device=local, rank=rank, host_fed=not args.no_e2e)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+    barrier = du.barrier
 
     def max_over_ranks(ms: float) -> float:
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return du.max_over_ranks(ms, device="cuda")
 
     for _ in range(args.warmup):
         runner.run_batch()
@@ -326,7 +318,7 @@ def main():
     if code != 0:
         raise RuntimeError(f"device status {code} (detail {detail}) after the timed region")
     ms_step = ms_total / args.steps
-    value = world * cfg.B * cfg.n_gen / (ms_step * 1e-3)
+    value = du.job_throughput(cfg.B * cfg.n_gen, ms_step)
 
     # ---- roofline of the dominant kernel: decode attention, from the launches timed inside the region
     tot_bytes, tot_ms = 0, 0.0
@@ -347,7 +339,13 @@ def main():
                 "frac_of_nominal_8TBs": achieved / 8000.0}
     prof = os.path.join(ROOT, "profiles", "attn_decode_traffic.json")
     if os.path.exists(prof):
-        roofline["traffic"] = json.load(open(prof)).get("traffic_bytes_per_launch")
+        # DRAM bytes per launch from the committed ncu capture (a smaller case of the same kernel), scaled by
+        # the bytes one timed launch processes; dropped once the kernel source has changed since the capture
+        import hashlib
+        pj = json.load(open(prof))
+        src = os.path.join(ROOT, pj.get("source", ""))
+        if os.path.exists(src) and hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] == pj.get("source_sha256_16"):
+            roofline["traffic"] = pj["traffic_over_algorithmic"] * roofline["avg_algorithmic_bytes"]
 
     # ---- end to end: every input from pinned host memory, every result back to the host
     e2e = None
