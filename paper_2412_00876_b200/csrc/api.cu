@@ -245,9 +245,12 @@ int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, 
   return cuda_status(ctx, launch_attn_prefill_simt(ctx, q, k_cache, v_cache, cache_len, B, cap, n_max, scale, out, s));
 }
 
-int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
-                              void* v_cache, const int32_t* cache_len, const uint8_t* keep, int32_t B,
-                              int32_t cap, float scale, void* out, void* stream) {
+// One layer's decode attention.  `overlap_prev`: the launch may begin while the previous kernel of
+// the stream is still draining (only dl_decode_step asks for it, for layers 1.. of a stack whose
+// caches and outputs are distinct tensors).
+static int32_t decode_layer(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
+                            void* v_cache, const int32_t* cache_len, const uint8_t* keep, int32_t B,
+                            int32_t cap, float scale, void* out, bool overlap_prev, void* stream) {
   if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
   if (B == 0) return DL_OK;
   if (!q_t || !k_t || !v_t || !k_cache || !v_cache || !cache_len || !out) return DL_ERR_INVALID_ARG;
@@ -258,7 +261,13 @@ int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, con
   if (B > 2048) return DL_ERR_UNSUPPORTED;
   DeviceGuard g(ctx->device);
   return cuda_status(ctx, launch_attn_decode(ctx, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, B, cap,
-                                             scale, out, static_cast<cudaStream_t>(stream)));
+                                             scale, out, overlap_prev, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
+                              void* v_cache, const int32_t* cache_len, const uint8_t* keep, int32_t B,
+                              int32_t cap, float scale, void* out, void* stream) {
+  return decode_layer(ctx, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, B, cap, scale, out, false, stream);
 }
 
 int32_t dl_decode_keep(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
@@ -299,8 +308,10 @@ int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, 
     const char* kl = static_cast<const char*>(k_t) + l * layer_bytes;
     const char* vl = static_cast<const char*>(v_t) + l * layer_bytes;
     char* ol = static_cast<char*>(out) + l * layer_bytes;
-    st = dl_sparse_attn_decode(ctx, ql, kl, vl, k_caches[l], v_caches[l], cache_len, keep_out, B, cap, scale,
-                               ol, stream);
+    // consecutive layers touch different caches and outputs, so layer l may start while layer l-1 drains
+    const bool overlap = l > 0 && k_caches[l] != k_caches[l - 1] && v_caches[l] != v_caches[l - 1];
+    st = decode_layer(ctx, ql, kl, vl, k_caches[l], v_caches[l], cache_len, keep_out, B, cap, scale, ol, overlap,
+                      stream);
     if (st != DL_OK) return st;
   }
   return dl_commit_len(ctx, keep_out, B, cap, cache_len, stream);

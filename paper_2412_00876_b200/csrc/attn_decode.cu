@@ -85,6 +85,7 @@ struct DecodeArgs {
   void* out;
   float* partial; int32_t* ticket; DeviceStatus* status;
   int32_t B, H, cap, chunk, per_bh, slots, n_stages;
+  int32_t overlap;        // launched with programmatic stream serialisation (see launch_mma)
   float scale_log2;
 };
 
@@ -455,6 +456,9 @@ attn_decode_mma_kernel(const __grid_constant__ TmapPair maps, const DecodeArgs a
   __shared__ int sh_abort;
   volatile int* abort_flag = &sh_abort;
 
+  // Let the next kernel of the stream start as soon as SMs free up (it only matters when that kernel
+  // was launched with programmatic stream serialisation; a no-op otherwise).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) sh_abort = 0;
   if (lane == 0) {
     for (int s = 0; s < NS; ++s) mbar_init(smem_u32(&bars[s]), 1);
@@ -718,6 +722,9 @@ attn_decode_mma_kernel(const __grid_constant__ TmapPair maps, const DecodeArgs a
     }
   }
 
+  // A kernel that was allowed to start early must not finish before its predecessor has: whatever
+  // follows in the stream (the length commit) relies on all earlier layers being done.
+  if (a.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (*abort_flag) {
     if (lane == 0) {
       report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
@@ -773,8 +780,19 @@ static cudaError_t launch_mma(const dl_ctx* ctx, DecodeArgs& a, cudaStream_t s) 
   }
   const long long max_items = (long long)a.B * a.H * max_chunks(a);
   const int grid = (int)max(1LL, min((long long)ctx->sm_count, max_items));
-  attn_decode_mma_kernel<<<grid, kMmaWarps * 32, smem, s>>>(maps, a);
-  return cudaGetLastError();
+  if (!a.overlap) {
+    attn_decode_mma_kernel<<<grid, kMmaWarps * 32, smem, s>>>(maps, a);
+    return cudaGetLastError();
+  }
+  // Programmatic stream serialisation: this launch may begin while the previous kernel of the stream
+  // (the decode attention of the previous layer, which touches other caches and outputs) drains.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kMmaWarps * 32); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, attn_decode_mma_kernel, maps, a);
 }
 
 template <typename T, int D>
@@ -801,7 +819,7 @@ static int scratch_slots(const DecodeArgs& a) { return max_chunks(a) + 1; }
 cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t,
                                void* k_cache, void* v_cache, const int32_t* cache_len,
                                const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                               cudaStream_t s) {
+                               bool overlap_prev, cudaStream_t s) {
   if (B == 0) return cudaSuccess;
   if (B > kMaxDecodeBatch) return cudaErrorInvalidValue;
   const dl_model_desc& d = ctx->desc;
@@ -812,6 +830,8 @@ cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t
   a.B = B; a.H = d.n_heads; a.cap = cap;
   pick_split(ctx, a);
   a.slots = ctx->ws.dec_slots;
+  // overlapping launches share the split scratch, so only unsplit launches may overlap
+  a.overlap = (overlap_prev && max_chunks(a) == 1) ? 1 : 0;
   a.n_stages = 0;
   a.scale_log2 = scale * 1.4426950408889634f;
   if (d.dtype == DL_BF16) {
@@ -878,6 +898,7 @@ extern "C" int32_t dl_sparse_attn_decode_static(dl_ctx* ctx, const void* q_t, co
   DecodeArgs a;
   a.B = B; a.H = d.n_heads; a.cap = cap;
   pick_split(ctx, a);
+  a.overlap = 0;
   const int slots = scratch_slots(a);
   // layout inside the array: tickets [B*H] int32 (256-byte padded) | partials [B*H*slots*(D+2)] float
   const size_t ticket_bytes = ((size_t)B * d.n_heads * sizeof(int32_t) + 255) & ~size_t(255);

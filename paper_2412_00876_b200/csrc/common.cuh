@@ -117,7 +117,7 @@ cudaError_t launch_commit_len(const uint8_t* keep, int32_t B, int32_t cap, int32
 cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t,
                                void* k_cache, void* v_cache, const int32_t* cache_len,
                                const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                               cudaStream_t s);
+                               bool overlap_prev, cudaStream_t s);
 
 cudaError_t launch_predictor_simt(const dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows,
                                   float* score, cudaStream_t s);
