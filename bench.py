@@ -41,6 +41,7 @@ def parse():
                     help="time one stage alone on the config's shapes (small memory; used for ncu captures)")
     ap.add_argument("--micro-layers", type=int, default=2, help="layers of cache / source held in --micro mode")
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
+    ap.add_argument("--decode-chunk", type=int, default=0, help="--micro decode: rows per work item (0: library's choice)")
     return ap.parse_args()
 
 
@@ -60,6 +61,8 @@ def micro(args):
     tdt = wl.torch_dtype(cfg.dtype)
     rows = B * cfg.n_vis
     ctx = dl.Context(cfg.hidden, H, D, cfg.pred_hidden, tdt, 0, max_batch=B, max_rows=rows, cap=cfg.cap)
+    if args.decode_chunk:
+        ctx.set_option(dl.DL_OPT_DECODE_CHUNK, args.decode_chunk)
     scale = 1.0 / float(np.sqrt(D))
     i32 = dict(dtype=torch.int32, device=dev)
     work, unit, calls = 0.0, "GB/s", []

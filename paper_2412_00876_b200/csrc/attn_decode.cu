@@ -413,7 +413,9 @@ static cudaError_t launch_cfg(const dl_ctx* ctx, DecodeArgs& a, cudaStream_t s) 
 // Tiles are fetched with TMA tile copies using the 128-byte swizzle so that ldmatrix is free of
 // bank conflicts; each 16-row tile is four 2 KB boxes (K low/high 64 dims, V low/high 64 dims).
 // =================================================================================================
-constexpr int kMmaWarps = 8;
+constexpr int kMmaWarps = 4;                      // warps per CTA
+constexpr int kMmaCtas = 2;                       // CTAs per SM: with overlapped launches a CTA of the next
+                                                  // layer moves in as soon as one of the two has finished
 constexpr int kMmaRows = 16;                       // rows per stage
 constexpr int kMmaBox = kMmaRows * 128;            // one box: 16 rows x 64 bf16
 constexpr int kMmaStage = 4 * kMmaBox;             // K lo | K hi | V lo | V hi
@@ -442,7 +444,7 @@ __device__ __forceinline__ void tma_tile_2d(uint32_t dst, const void* map, int x
 
 struct TmapPair { alignas(64) unsigned char k[128]; alignas(64) unsigned char v[128]; };
 
-__global__ void __launch_bounds__(kMmaWarps * 32, 1)
+__global__ void __launch_bounds__(kMmaWarps * 32, kMmaCtas)
 attn_decode_mma_kernel(const __grid_constant__ TmapPair maps, const DecodeArgs a) {
   constexpr int D = 128, RB = 256, RS = kMmaRows;
   extern __shared__ char smem_raw[];
@@ -766,7 +768,8 @@ static cudaError_t launch_mma(const dl_ctx* ctx, DecodeArgs& a, cudaStream_t s) 
   if (!cached_cache_map(ctx, maps.k, a.k_cache, rows) || !cached_cache_map(ctx, maps.v, a.v_cache, rows))
     return cudaErrorInvalidValue;
   const size_t fixed = (size_t)(a.B + 1) * sizeof(int) + 1024 /*alignment*/ + 256;
-  int ns = (int)((ctx->smem_optin - 256 - (int)fixed) / (kMmaWarps * (kMmaStage + 8)));
+  const int per_cta = (ctx->smem_optin + 1024) / kMmaCtas - 1024;        // shared memory one CTA may take
+  int ns = (int)((per_cta - 256 - (int)fixed) / (kMmaWarps * (kMmaStage + 8)));
   ns = min(ns, 6);
   if (ns < 2) return cudaErrorInvalidConfiguration;
   a.n_stages = ns;
@@ -779,7 +782,7 @@ static cudaError_t launch_mma(const dl_ctx* ctx, DecodeArgs& a, cudaStream_t s) 
     attr_set_for = (int)smem;
   }
   const long long max_items = (long long)a.B * a.H * max_chunks(a);
-  const int grid = (int)max(1LL, min((long long)ctx->sm_count, max_items));
+  const int grid = (int)max(1LL, min((long long)ctx->sm_count * kMmaCtas, max_items));
   if (!a.overlap) {
     attn_decode_mma_kernel<<<grid, kMmaWarps * 32, smem, s>>>(maps, a);
     return cudaGetLastError();
