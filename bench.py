@@ -325,9 +325,11 @@ def main():
 
     # ---- roofline of the dominant kernel: decode attention, from the launches timed inside the region
     tot_bytes, tot_ms = 0, 0.0
-    for (a, b, lens) in events:
-        tot_bytes += runner.decode_bytes(lens)
+    n_timed = 0
+    for (a, b, lens, n_launch) in events:                 # one pair per sampled step: its L attention launches
+        tot_bytes += n_launch * runner.decode_bytes(lens)
         tot_ms += a.elapsed_time(b)
+        n_timed += n_launch
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(peaks_path):
         peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
@@ -336,9 +338,9 @@ def main():
     achieved = tot_bytes / (tot_ms * 1e-3) / 1e9 if tot_ms > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": "attn_decode_mma_kernel", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
-                "launches_timed": len(events),
-                "avg_launch_us": 1e3 * tot_ms / max(len(events), 1),
-                "avg_algorithmic_bytes": tot_bytes / max(len(events), 1),
+                "launches_timed": n_timed,
+                "avg_launch_us": 1e3 * tot_ms / max(n_timed, 1),
+                "avg_algorithmic_bytes": tot_bytes / max(n_timed, 1),
                 "frac_of_nominal_8TBs": achieved / 8000.0}
     prof = os.path.join(ROOT, "profiles", "attn_decode_traffic.json")
     if os.path.exists(prof):

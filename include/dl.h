@@ -167,6 +167,17 @@ int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, con
                               const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
                               void* stream);
 
+/* The same for a stack of L layers that share cache_len and keep (Eq. 6 applied per layer with the
+ * one decision of Sec. 3.3.1): q_t, k_t, v_t, out dev [L][B][H][D]; k_caches, v_caches HOST arrays of
+ * L device pointers, each [B][H][cap][D] and all distinct.  Equivalent to L calls of
+ * dl_sparse_attn_decode in layer order, except that a layer's kernel may begin while the previous
+ * layer's is still draining (they touch different caches and outputs); everything launched after
+ * this call still sees all L layers complete. */
+int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
+                                     void* const* k_caches, void* const* v_caches, const int32_t* cache_len,
+                                     const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
+                                     void* stream);
+
 /* ---- decode decision: Eq. 5 applied to the current token (Eq. 6) ----------------------- */
 
 /* logit[b] = P^{OT}(x_t[b]);  keep[b] = logit[b] > threshold (strict; NaN -> 0).

@@ -25,7 +25,7 @@ EXPORTS = [
     "dl_device_status", "dl_status_str", "dl_last_cuda_error", "dl_predictor_scores",
     "dl_topk_from_scores", "dl_prefill_select", "dl_compact_kv", "dl_sparse_attn_prefill",
     "dl_sparse_attn_decode", "dl_decode_keep", "dl_commit_len", "dl_decode_step", "dl_decode_step_host",
-    "dl_sparse_attn_decode_static",
+    "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers",
 ]
 
 
@@ -68,6 +68,8 @@ def lib() -> C.CDLL:
             "dl_sparse_attn_prefill": (i32, [vp, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp]),
             "dl_sparse_attn_decode": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp]),
             "dl_sparse_attn_decode_static": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp]),
+            "dl_sparse_attn_decode_layers": (i32, [vp, i32, vp, vp, vp, C.POINTER(vp), C.POINTER(vp), vp, vp, i32, i32,
+                                                  f32, vp, vp]),
             "dl_decode_keep": (i32, [vp, P, vp, i32, f32, vp, vp, vp]),
             "dl_commit_len": (i32, [vp, vp, i32, i32, vp, vp]),
             "dl_decode_step": (i32, [vp, P, vp, i32, f32, vp, vp, i32, vp, vp, vp, C.POINTER(vp),
@@ -213,6 +215,13 @@ class Context:
                                                        _ptr(v_cache), _ptr(cache_len), _ptr(keep), B, cap,
                                                        float(scale), _ptr(out), _stream(stream)),
                     "dl_sparse_attn_decode_static")
+
+    def sparse_attn_decode_layers(self, q_t, k_t, v_t, k_ptrs, v_ptrs, L, cap, cache_len, keep, scale, out,
+                                  stream=None):
+        B = cache_len.shape[0]
+        self._check(lib().dl_sparse_attn_decode_layers(self._h, L, _ptr(q_t), _ptr(k_t), _ptr(v_t), k_ptrs, v_ptrs,
+                                                       _ptr(cache_len), _ptr(keep), B, cap, float(scale), _ptr(out),
+                                                       _stream(stream)), "dl_sparse_attn_decode_layers")
 
     def decode_keep(self, p: Predictor | None, x_t, logit_inout, keep_out, threshold=0.0, stream=None):
         B = logit_inout.shape[0]

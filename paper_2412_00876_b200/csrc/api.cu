@@ -293,6 +293,28 @@ int32_t dl_commit_len(dl_ctx* ctx, const uint8_t* keep, int32_t B, int32_t cap, 
   return cuda_status(ctx, launch_commit_len(keep, B, cap, cache_len, static_cast<cudaStream_t>(stream)));
 }
 
+int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
+                                     void* const* k_caches, void* const* v_caches, const int32_t* cache_len,
+                                     const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
+                                     void* stream) {
+  if (!ctx || L < 0 || B < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || L == 0) return DL_OK;
+  if (!k_caches || !v_caches || !q_t || !k_t || !v_t || !out) return DL_ERR_INVALID_ARG;
+  const size_t layer_bytes = (size_t)B * ctx->desc.n_heads * ctx->desc.head_dim * elt_bytes(ctx);
+  for (int32_t l = 0; l < L; ++l) {
+    const char* ql = static_cast<const char*>(q_t) + l * layer_bytes;
+    const char* kl = static_cast<const char*>(k_t) + l * layer_bytes;
+    const char* vl = static_cast<const char*>(v_t) + l * layer_bytes;
+    char* ol = static_cast<char*>(out) + l * layer_bytes;
+    // consecutive layers touch different caches and outputs, so layer l may start while layer l-1 drains
+    const bool overlap = l > 0 && k_caches[l] != k_caches[l - 1] && v_caches[l] != v_caches[l - 1];
+    int32_t st = decode_layer(ctx, ql, kl, vl, k_caches[l], v_caches[l], cache_len, keep, B, cap, scale, ol, overlap,
+                              stream);
+    if (st != DL_OK) return st;
+  }
+  return DL_OK;
+}
+
 int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
                        float* logit_inout, uint8_t* keep_out, int32_t L, const void* q_t, const void* k_t,
                        const void* v_t, void* const* k_caches, void* const* v_caches, int32_t cap,
@@ -302,18 +324,9 @@ int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, 
   if (L > 0 && (!k_caches || !v_caches || !q_t || !k_t || !v_t || !out)) return DL_ERR_INVALID_ARG;
   int32_t st = dl_decode_keep(ctx, p_txt, x_t, B, threshold, logit_inout, keep_out, stream);
   if (st != DL_OK) return st;
-  const size_t layer_bytes = (size_t)B * ctx->desc.n_heads * ctx->desc.head_dim * elt_bytes(ctx);
-  for (int32_t l = 0; l < L; ++l) {
-    const char* ql = static_cast<const char*>(q_t) + l * layer_bytes;
-    const char* kl = static_cast<const char*>(k_t) + l * layer_bytes;
-    const char* vl = static_cast<const char*>(v_t) + l * layer_bytes;
-    char* ol = static_cast<char*>(out) + l * layer_bytes;
-    // consecutive layers touch different caches and outputs, so layer l may start while layer l-1 drains
-    const bool overlap = l > 0 && k_caches[l] != k_caches[l - 1] && v_caches[l] != v_caches[l - 1];
-    st = decode_layer(ctx, ql, kl, vl, k_caches[l], v_caches[l], cache_len, keep_out, B, cap, scale, ol, overlap,
-                      stream);
-    if (st != DL_OK) return st;
-  }
+  st = dl_sparse_attn_decode_layers(ctx, L, q_t, k_t, v_t, k_caches, v_caches, cache_len, keep_out, B, cap, scale, out,
+                                    stream);
+  if (st != DL_OK) return st;
   return dl_commit_len(ctx, keep_out, B, cap, cache_len, stream);
 }
 

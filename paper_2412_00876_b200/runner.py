@@ -103,17 +103,17 @@ class BatchRunner:
         self.launches += 3 + c.n_layers
 
     def decode_step_timed(self, t: int, events: list):
-        """The same step issued call by call, with an event pair around every attention launch."""
+        """The same step issued as keep decision, layer stack, commit, with one event pair around the
+        stack's L attention launches (issued exactly as dl_decode_step issues them)."""
         c, i, ctx = self.cfg, t % self.step_pool, self.ctx
         ctx.decode_keep(self.p_txt, self.x_dec[i], self.logit, self.keep_t)
         lens = self.cache_len.clone()
-        for l in range(c.n_layers):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            ctx.sparse_attn_decode(self.q_dec[i, l], self.k_dec[i, l], self.v_dec[i, l], self.k_cache[l],
-                                   self.v_cache[l], self.cache_len, self.keep_t, self.scale, self.dec_out[l])
-            e1.record()
-            events.append((e0, e1, lens))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.sparse_attn_decode_layers(self.q_dec[i], self.k_dec[i], self.v_dec[i], self.kp, self.vp, c.n_layers,
+                                      self.cap, self.cache_len, self.keep_t, self.scale, self.dec_out)
+        e1.record()
+        events.append((e0, e1, lens, c.n_layers))
         ctx.commit_len(self.keep_t, self.cache_len, self.cap)
         self.launches += 3 + c.n_layers
 
