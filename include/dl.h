@@ -186,6 +186,17 @@ int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, co
 int32_t dl_decode_keep(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B,
                        float threshold, float* logit_inout, uint8_t* keep_out, void* stream);
 
+/* Decoding WITHOUT KV cache (Eq. 12 and the sentence above Eq. 6): the decisions for ALL generated
+ * tokens of every sequence at once; the last generated token of a sequence is always kept, since it
+ * produces the next token.  keep[b][i] = i < n_gen[b] and (logit[b][i] > threshold or i == n_gen[b]-1).
+ *   x_gen dev [B][n_gen_max][hidden] or NULL (then logit_inout is used as given); n_gen dev [B] or NULL
+ *   (= n_gen_max); logit_inout dev [B][n_gen_max] float32; keep_out dev [B][n_gen_max] (padding 0).
+ * The reduced set S^{P*} u S^{OT*} is then built with dl_compact_kv (this mask, keep_cols = n_gen_max,
+ * t_src = n_gen, appended behind the compact prefill rows) and attended with dl_sparse_attn_prefill. */
+int32_t dl_decode_nocache_select(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_gen, const int32_t* n_gen,
+                                 int32_t B, int32_t n_gen_max, float threshold, float* logit_inout,
+                                 uint8_t* keep_out, void* stream);
+
 /* cache_len[b] += (keep[b] != 0) where cache_len[b] < cap: closes a decode step after every
  * layer has appended with the shared decision (Sec. 3.3.2). */
 int32_t dl_commit_len(dl_ctx* ctx, const uint8_t* keep, int32_t B, int32_t cap, int32_t* cache_len,

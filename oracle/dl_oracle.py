@@ -13,6 +13,7 @@ What each function follows
                         original token order (set builder of Eq. 5)
   decode_keep           Eq. 5 / Eq. 6: keep iff the "keep" value exceeds the "drop" value,
                         i.e. folded single logit > threshold (0), strictly
+  nocache_keep          Eq. 12 with the forced last token (decoding without KV cache)
   prefill_keep_mask /   Eq. 5 set builder, Eq. 11 (kept vision rows, then every text row),
   append_rows           Eq. 6 (append K, V of the current token iff its mask is 1)
   attention_masked_full Eq. 7 with diag(G) = 1 under the causal mask: THE definition of
@@ -103,6 +104,23 @@ def decode_keep(logit: np.ndarray, threshold: float = 0.0) -> np.ndarray:
     logit = np.asarray(logit, dtype=np.float64)
     with np.errstate(invalid="ignore"):
         return (logit > threshold).astype(np.uint8)
+
+
+def nocache_keep(logit: np.ndarray, n_gen, threshold: float = 0.0) -> np.ndarray:
+    """Decoding WITHOUT KV cache (Eq. 12, and the sentence above Eq. 6): the mask of all generated
+    tokens at once, M^OT = [logit > threshold], except that the last generated token of every
+    sequence is always kept (it produces the next token).  logit [B, n_max]; n_gen [B] valid
+    tokens per sequence (None = all); slots past n_gen[b] are 0."""
+    logit = np.asarray(logit, dtype=np.float64)
+    B, n_max = logit.shape
+    n_gen = np.full(B, n_max, dtype=np.int64) if n_gen is None else np.asarray(n_gen)
+    keep = np.zeros((B, n_max), dtype=np.uint8)
+    for b in range(B):
+        n = int(n_gen[b])
+        keep[b, :n] = decode_keep(logit[b, :n], threshold)
+        if n > 0:
+            keep[b, n - 1] = 1
+    return keep
 
 
 # --------------------------------------------------------------------------- compaction

@@ -25,7 +25,7 @@ EXPORTS = [
     "dl_device_status", "dl_status_str", "dl_last_cuda_error", "dl_predictor_scores",
     "dl_topk_from_scores", "dl_prefill_select", "dl_compact_kv", "dl_sparse_attn_prefill",
     "dl_sparse_attn_decode", "dl_decode_keep", "dl_commit_len", "dl_decode_step", "dl_decode_step_host",
-    "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers",
+    "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers", "dl_decode_nocache_select",
 ]
 
 
@@ -71,6 +71,7 @@ def lib() -> C.CDLL:
             "dl_sparse_attn_decode_layers": (i32, [vp, i32, vp, vp, vp, C.POINTER(vp), C.POINTER(vp), vp, vp, i32, i32,
                                                   f32, vp, vp]),
             "dl_decode_keep": (i32, [vp, P, vp, i32, f32, vp, vp, vp]),
+            "dl_decode_nocache_select": (i32, [vp, P, vp, vp, i32, i32, f32, vp, vp, vp]),
             "dl_commit_len": (i32, [vp, vp, i32, i32, vp, vp]),
             "dl_decode_step": (i32, [vp, P, vp, i32, f32, vp, vp, i32, vp, vp, vp, C.POINTER(vp),
                                      C.POINTER(vp), i32, vp, f32, vp, vp]),
@@ -228,6 +229,14 @@ class Context:
         pd = C.byref(p.desc) if p is not None else None
         self._check(lib().dl_decode_keep(self._h, pd, _ptr(x_t), B, float(threshold), _ptr(logit_inout),
                                          _ptr(keep_out), _stream(stream)), "dl_decode_keep")
+
+    def decode_nocache_select(self, p: Predictor | None, x_gen, n_gen, logit_inout, keep_out, threshold=0.0,
+                              stream=None):
+        B, n_max = logit_inout.shape
+        pd = C.byref(p.desc) if p is not None else None
+        self._check(lib().dl_decode_nocache_select(self._h, pd, _ptr(x_gen), _ptr(n_gen), B, n_max, float(threshold),
+                                                   _ptr(logit_inout), _ptr(keep_out), _stream(stream)),
+                    "dl_decode_nocache_select")
 
     def commit_len(self, keep, cache_len, cap, stream=None):
         self._check(lib().dl_commit_len(self._h, _ptr(keep), keep.shape[0], cap, _ptr(cache_len),

@@ -284,6 +284,23 @@ int32_t dl_decode_keep(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, 
   return cuda_status(ctx, launch_decode_keep(logit_inout, B, threshold, keep_out, ctx->ws.status, s));
 }
 
+int32_t dl_decode_nocache_select(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_gen, const int32_t* n_gen,
+                                 int32_t B, int32_t n_gen_max, float threshold, float* logit_inout,
+                                 uint8_t* keep_out, void* stream) {
+  if (!ctx || B < 0 || n_gen_max < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || n_gen_max == 0) return DL_OK;
+  if (!logit_inout || !keep_out) return DL_ERR_INVALID_ARG;
+  if ((int64_t)B * n_gen_max > INT32_MAX) return DL_ERR_UNSUPPORTED;
+  DeviceGuard g(ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (x_gen) {
+    int32_t st = run_predictor(ctx, p_txt, x_gen, B * n_gen_max, logit_inout, s);
+    if (st != DL_OK) return st;
+  }
+  return cuda_status(ctx, launch_nocache_mask(logit_inout, n_gen, B, n_gen_max, threshold, keep_out,
+                                              ctx->ws.status, s));
+}
+
 int32_t dl_commit_len(dl_ctx* ctx, const uint8_t* keep, int32_t B, int32_t cap, int32_t* cache_len,
                       void* stream) {
   if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;

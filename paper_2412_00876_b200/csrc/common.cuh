@@ -128,6 +128,9 @@ bool predictor_tc_supported(const dl_ctx* ctx);
 cudaError_t launch_decode_keep(const float* logit, int32_t B, float threshold, uint8_t* keep,
                                DeviceStatus* st, cudaStream_t s);
 
+cudaError_t launch_nocache_mask(const float* logit, const int32_t* n_gen, int32_t B, int32_t n_max,
+                                float threshold, uint8_t* keep, DeviceStatus* st, cudaStream_t s);
+
 cudaError_t launch_attn_prefill_simt(const dl_ctx* ctx, const void* q, const void* k_cache,
                                      const void* v_cache, const int32_t* cache_len, int32_t B,
                                      int32_t cap, int32_t n_max, float scale, void* out, cudaStream_t s);

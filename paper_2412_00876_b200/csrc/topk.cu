@@ -156,6 +156,32 @@ __global__ void decode_keep_kernel(const float* __restrict__ logit, int32_t B, f
   keep[b] = (z > threshold) ? 1 : 0;
 }
 
+// Decoding without KV cache (Eq. 12): the mask of all generated tokens of every sequence at once,
+// keep iff logit > threshold, with the last valid token of each sequence always kept.
+__global__ void nocache_mask_kernel(const float* __restrict__ logit, const int32_t* __restrict__ n_gen,
+                                    int32_t B, int32_t n_max, float threshold, uint8_t* __restrict__ keep,
+                                    DeviceStatus* st) {
+  const int b = blockIdx.y;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_max) return;
+  const int n = min(max(n_gen ? n_gen[b] : n_max, 0), n_max);
+  uint8_t k = 0;
+  if (i < n) {
+    const float z = logit[(size_t)b * n_max + i];
+    if (z != z) report_status(st, DL_WARN_NAN, (long long)b * n_max + i);
+    k = (z > threshold || i == n - 1) ? 1 : 0;
+  }
+  keep[(size_t)b * n_max + i] = k;
+}
+
+cudaError_t launch_nocache_mask(const float* logit, const int32_t* n_gen, int32_t B, int32_t n_max,
+                                float threshold, uint8_t* keep, DeviceStatus* st, cudaStream_t s) {
+  if (B == 0 || n_max == 0) return cudaSuccess;
+  dim3 grid((n_max + 255) / 256, B);
+  nocache_mask_kernel<<<grid, 256, 0, s>>>(logit, n_gen, B, n_max, threshold, keep, st);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_decode_keep(const float* logit, int32_t B, float threshold, uint8_t* keep,
                                DeviceStatus* st, cudaStream_t s) {
   if (B == 0) return cudaSuccess;

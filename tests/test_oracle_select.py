@@ -88,3 +88,21 @@ def test_decode_keep_counts_positive_logits():
     # alternating-sign logits reproduce the paper's "Structure" static mask (every other token)
     alt = np.where(np.arange(10) % 2 == 0, 1.0, -1.0)
     assert list(orc.decode_keep(alt)) == list(wl.static_keep_pattern("structure", 10))
+
+
+def test_nocache_mask_keeps_the_last_generated_token():
+    """Eq. 12 / text above Eq. 6: all generated tokens are decided at once and the last one is kept."""
+    z = np.array([[0.5, -1.0, 0.0, -2.0, 9.0], [-1.0, -1.0, -1.0, -1.0, -1.0], [3.0, 3.0, 3.0, 3.0, 3.0]])
+    m = orc.nocache_keep(z, np.array([4, 5, 0]))
+    assert m.tolist() == [[1, 0, 0, 1, 0], [0, 0, 0, 0, 1], [0, 0, 0, 0, 0]]
+    # brute force over random inputs: positives, plus the last valid slot, nothing in the padding
+    rng = np.random.default_rng(9)
+    z = rng.normal(size=(6, 17))
+    n = rng.integers(0, 18, size=6)
+    m = orc.nocache_keep(z, n)
+    for b in range(6):
+        for i in range(17):
+            want = i < n[b] and (z[b, i] > 0 or i == n[b] - 1)
+            assert m[b, i] == int(want)
+    # without the forced token it is Eq. 6's per-token decision
+    assert np.array_equal(orc.nocache_keep(z, None)[:, :-1], orc.decode_keep(z)[:, :-1])
