@@ -37,7 +37,7 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-every", type=int, default=64, help="decode steps between timed attention launches")
-    ap.add_argument("--micro", default="", choices=["", "decode", "predictor", "compact", "prefill"],
+    ap.add_argument("--micro", default="", choices=["", "decode", "predictor", "compact", "prefill", "nocache"],
                     help="time one stage alone on the config's shapes (small memory; used for ncu captures)")
     ap.add_argument("--micro-layers", type=int, default=2, help="layers of cache / source held in --micro mode")
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
@@ -111,6 +111,33 @@ def micro(args):
             work, unit = 2.0 * D * cfg.n0 * (cfg.n0 + 1) * H * B, "TFLOP/s"
             calls = [lambda l=l: ctx.sparse_attn_prefill(kc[l], kc[l], vc[l], ln, cfg.n0, scale, out)
                      for l in range(NL)]
+    elif args.micro == "nocache":
+        # one pass of decoding WITHOUT cache for one layer (Eq. 12): decide all N_OT generated tokens, rebuild the
+        # reduced set behind the compact prefill rows, attend over it
+        ng = cfg.n_gen
+        p = wl.make_predictor(cfg, "txt")
+        pd = dl.Predictor(wl.to_torch(p.w1, cfg.dtype, dev), torch.from_numpy(p.b1).to(dev),
+                          torch.from_numpy(p.w2).to(dev), p.b2)
+        ctx.set_workspace(B, B * max(ng, cfg.n_vis), cfg.cap)
+        xg = [wl.device_normal(cfg, wl.S_X_TXT, (B, ng, cfg.hidden), dev, sub=i) for i in range(NL)]
+        gen = [wl.device_normal(cfg, wl.S_DEC_K, (B, ng, H, D), dev, sub=i) for i in range(3 * NL)]
+        caches = [wl.device_normal(cfg, wl.S_CACHE_K, (B, H, cfg.cap, D), dev, sub=i) for i in range(3 * NL)]
+        logit = torch.empty(B, ng, dtype=torch.float32, device=dev)
+        keep = torch.empty(B, ng, dtype=torch.uint8, device=dev)
+        n_gen = torch.full((B,), ng, **i32)
+        ln, lq = torch.empty(B, **i32), torch.empty(B, **i32)
+        n0 = torch.full((B,), cfg.n0, **i32)
+        out = torch.empty(B, cfg.cap, H, D, dtype=tdt, device=dev)
+        n_exp = cfg.n0 + ng * cfg.keep_rate
+        work, unit = 2.0 * D * n_exp * (n_exp + 1) * H * B, "TFLOP/s"          # attention part, expected length
+
+        def one(l):
+            ln.copy_(n0); lq.copy_(n0)
+            ctx.decode_nocache_select(pd, xg[l], n_gen, logit, keep)
+            ctx.compact_kv(gen[3 * l], None, keep, n_gen, caches[3 * l], None, lq, commit=True)
+            ctx.compact_kv(gen[3 * l + 1], gen[3 * l + 2], keep, n_gen, caches[3 * l + 1], caches[3 * l + 2], ln, commit=True)
+            ctx.sparse_attn_prefill(caches[3 * l], caches[3 * l + 1], caches[3 * l + 2], ln, cfg.cap, scale, out)
+        calls = [lambda l=l: one(l) for l in range(NL)]
     for i in range(args.warmup):
         calls[i % NL]()
     torch.cuda.synchronize()
