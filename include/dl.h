@@ -150,7 +150,7 @@ int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const u
  * themselves, per sequence and head: row i attends rows 0..i of the same cache.
  *   q dev [B][H][cap][D] compact queries in the cache layout (built by dl_compact_kv);
  *   k_cache, v_cache dev [B][H][cap][D]; cache_len dev [B]; n_max >= every cache_len[b], <= cap;
- *   out dev [B][n_max][H][D] (rows >= cache_len[b] are not written); scale usually 1/sqrt(D). */
+ *   out dev [B][n_max][H][D] (rows >= cache_len[b] are not written); scale > 0, usually 1/sqrt(D). */
 int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max,
                                float scale, void* out, void* stream);

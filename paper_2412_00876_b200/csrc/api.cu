@@ -230,7 +230,7 @@ int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const u
 int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max, float scale,
                                void* out, void* stream) {
-  if (!ctx || B < 0 || cap <= 0 || n_max < 0 || n_max > cap) return DL_ERR_INVALID_ARG;
+  if (!ctx || B < 0 || cap <= 0 || n_max < 0 || n_max > cap || !(scale > 0.f)) return DL_ERR_INVALID_ARG;
   if (B == 0 || n_max == 0) return DL_OK;
   if (!q || !k_cache || !v_cache || !cache_len || !out) return DL_ERR_INVALID_ARG;
   if (misaligned(q) || misaligned(k_cache) || misaligned(v_cache) || misaligned(out)) return DL_ERR_ALIGNMENT;

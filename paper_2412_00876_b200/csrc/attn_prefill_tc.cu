@@ -29,6 +29,13 @@ constexpr size_t kAtSmem = kAtQBytes + kAtStages * kAtStage + 1024 + 256;
 constexpr uint32_t kAtColO = 0, kAtColS = 128;        // tensor-memory columns: O | S0 | S1
 constexpr float kRescaleStep = 8.0f;                  // log2 units by which the maximum may lag
 
+// 2^x on the special-function unit (x <= 0 here; -inf gives 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 struct AtMaps { alignas(64) unsigned char q[128]; alignas(64) unsigned char k[128]; alignas(64) unsigned char v[128]; };
 
 struct AtArgs {
@@ -166,14 +173,21 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       tmem_ld32(s_addr + 32, sr + 32);
       tmem_ld_wait();
       const int c0 = j * kAtBN;
+      // raw scores stay unscaled: max commutes with the (positive) scale and the scale is folded into
+      // the exponent's FMA.  Only tiles that reach past the tile's first row need the causal mask.
       float mx = -INFINITY;
+      if (c0 + kAtBN - 1 > q0) {
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        float v = __uint_as_float(sr[c]) * a.scale_log2;
-        v = (c0 + c > grow) ? -INFINITY : v;
-        sr[c] = __float_as_uint(v);
-        mx = fmaxf(mx, v);
+        for (int c = 0; c < 64; ++c) {
+          const float v = (c0 + c > grow) ? -INFINITY : __uint_as_float(sr[c]);
+          sr[c] = __float_as_uint(v);
+          mx = fmaxf(mx, v);
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
       }
+      mx *= a.scale_log2;
       if (j == 0) {
         m_used = mx;                        // column 0 is visible to every row, so mx is finite
       } else {
@@ -181,7 +195,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         if (__any_sync(0xffffffffu, need)) {
           mbar_wait(smem_u32(pv_done), (j - 1) & 1, abort_flag);      // O must be at rest
           tc_fence_after();
-          const float corr = need ? exp2f(m_used - mx) : 1.0f;
+          const float corr = need ? fast_exp2(m_used - mx) : 1.0f;
           if (need) m_used = mx;
           l_run *= corr;
 #pragma unroll
@@ -198,13 +212,18 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       }
       uint32_t pw[32];
 #pragma unroll
+      const float neg_m = -m_used;
+      float l0 = 0.f, l1 = 0.f;
+#pragma unroll
       for (int c = 0; c < 32; ++c) {
-        const float p0 = exp2f(__uint_as_float(sr[2 * c]) - m_used);
-        const float p1 = exp2f(__uint_as_float(sr[2 * c + 1]) - m_used);
-        l_run += p0 + p1;
+        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c]), a.scale_log2, neg_m));
+        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), a.scale_log2, neg_m));
+        l0 += p0;
+        l1 += p1;
         __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
         pw[c] = *reinterpret_cast<uint32_t*>(&pk);
       }
+      l_run += l0 + l1;
       tmem_st32(s_addr, pw);                                             // P overwrites its own S buffer
       tmem_st_wait();
       if (j == n_tiles - 1 && kv_end < c0 + kAtBN) {
