@@ -34,6 +34,8 @@ def parse():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=3)
     ap.add_argument("--impl", default="ours")
+    ap.add_argument("--graphs", type=int, default=-1,
+                    help="replay decode steps from CUDA graphs: 1 yes, 0 no, -1 only for launch-bound workloads (B*L < 64)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-every", type=int, default=64, help="decode steps between timed attention launches")
@@ -319,7 +321,8 @@ def main():
         du.init("nccl", local)
         du.barrier()                       # the other ranks load the library only after rank 0 has built it
     cfg = wl.CONFIGS[args.config]
-    runner = BatchRunner(cfg, device=local, rank=rank, host_fed=not args.no_e2e)
+    use_graphs = bool(args.graphs) if args.graphs >= 0 else (cfg.B * cfg.n_layers < 64)
+    runner = BatchRunner(cfg, device=local, rank=rank, host_fed=not args.no_e2e, use_graphs=use_graphs)
 
     barrier = du.barrier
 
@@ -407,7 +410,7 @@ def main():
                 "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
                 "config": {"workload": cfg.name, "B_per_gpu": cfg.B, "layers": cfg.n_layers, "n_vis": cfg.n_vis,
                            "k_vis": cfg.k_vis, "n_text": cfg.n_text, "n_gen": cfg.n_gen, "keep_rate": cfg.keep_rate,
-                           "parallelism": f"batch-shards x{world}",
+                           "parallelism": f"batch-shards x{world}", "decode_steps_from_cuda_graphs": use_graphs,
                            "l2": "inputs larger than L2 (caches tens of GB; input pools > 126 MB)"},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
                 "clocks": clocks}

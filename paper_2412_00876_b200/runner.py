@@ -19,7 +19,7 @@ class BatchRunner:
     """Buffers and call sequence for one workload configuration on one GPU."""
 
     def __init__(self, cfg: wl.Config, device: int = 0, rank: int = 0, src_pool: int = 4, step_pool: int = 8,
-                 host_fed: bool = False, options: dict | None = None):
+                 host_fed: bool = False, options: dict | None = None, use_graphs: bool = False):
         self.cfg, self.dev, self.rank = cfg, torch.device("cuda", device), rank
         B, L, H, D = cfg.B, cfg.n_layers, cfg.n_heads, cfg.head_dim
         self.T = cfg.n_vis + cfg.n_text
@@ -73,6 +73,8 @@ class BatchRunner:
         self.keep_t = torch.empty(B, dtype=torch.uint8, device=dev)
         self.dec_out = torch.empty(L, B, H, D, dtype=tdt, device=dev)
         self.launches = 0
+        self.use_graphs = use_graphs
+        self._graphs: dict = {}            # decode step captured once per input-pool slot
         self.host_fed = host_fed
         if host_fed:
             self._make_host_buffers()
@@ -97,10 +99,30 @@ class BatchRunner:
 
     def decode_step(self, t: int):
         c, i = self.cfg, t % self.step_pool
+        if self.use_graphs:
+            # The step's launches depend on the step only through device memory (lengths, flags, the pool
+            # slot's inputs), so one captured graph per pool slot replays any step.
+            g = self._graphs.get(i)
+            if g is None:
+                saved = self.cache_len.clone()
+                self._decode_step_eager(i)                     # warm run: attributes set, tensor maps cached
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    self._decode_step_eager(i)
+                self.cache_len.copy_(saved)                    # undo the warm run's commit (its appended row
+                self._graphs[i] = g                            # lies past the restored length)
+            g.replay()
+            self.launches += 3 + c.n_layers
+            return
+        self._decode_step_eager(i)
+        self.launches += 3 + c.n_layers
+
+    def _decode_step_eager(self, i: int):
+        c = self.cfg
         self.ctx.decode_step(self.p_txt, self.x_dec[i], self.logit, self.keep_t, self.q_dec[i], self.k_dec[i],
                              self.v_dec[i], self.kp, self.vp, c.n_layers, self.cap, self.cache_len, self.scale,
                              self.dec_out)
-        self.launches += 3 + c.n_layers
 
     def decode_step_timed(self, t: int, events: list):
         """The same step issued as keep decision, layer stack, commit, with one event pair around the
