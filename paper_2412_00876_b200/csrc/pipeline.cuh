@@ -34,10 +34,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (and raises *abort) when the bound is hit or another warp aborted.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
-  if (*abort) return false;
+  if (mbar_try_wait(bar, parity)) return !*abort;            // fast path: the phase is already complete
   for (int i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
     if (*abort) return false;
+    if (mbar_try_wait(bar, parity)) return true;
     if (i > 32) __nanosleep(40);
   }
   *abort = 1;

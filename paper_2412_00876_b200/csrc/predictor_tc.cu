@@ -98,6 +98,8 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16(kPtBM, (uint32_t)a.bn);
+      const uint64_t desc_a0 = smem_desc_sw128(smem_u32(smem));
+      const uint64_t desc_b0 = smem_desc_sw128(smem_u32(smem) + kPtATile);
       int it = 0, j = 0;
       for (int item = blockIdx.x; item < items; item += gridDim.x, ++j) {
         const int buf = j & 1;
@@ -108,11 +110,12 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
           const int s = it % kPtStages;
           mbar_wait(smem_u32(&full[s]), (it / kPtStages) & 1, abort_flag);
           tc_fence_after();
-          const uint32_t sa = smem_u32(smem + (size_t)s * kPtStageBytes);
-          const uint32_t sb = sa + kPtATile;
+          // descriptors differ from the stage-0, k-0 ones only in the start-address field (16-byte units)
+          const uint64_t da = desc_a0 + (uint64_t)((s * kPtStageBytes) >> 4);
+          const uint64_t db = desc_b0 + (uint64_t)((s * kPtStageBytes) >> 4);
 #pragma unroll
           for (int k = 0; k < kPtBK / 16; ++k)
-            mma_ss(d_tmem, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc, (kb | k) != 0);
+            mma_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
           mma_commit(smem_u32(&empty[s]));             // frees the stage when these MMAs have read it
         }
         mma_commit(smem_u32(&acc_full[buf]));          // accumulator complete
