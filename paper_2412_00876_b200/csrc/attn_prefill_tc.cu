@@ -1,9 +1,11 @@
 // Prefill attention over the reduced set on the tensor cores (Eq. 1 applied to S^{P*}):
 // row i of a sequence's compact context attends rows 0..i of the same context.
-// bf16, head_dim 128.  One CTA per (sequence, head, 128-row query tile); two CTAs share an SM so
-// that one CTA's softmax overlaps the other's MMAs.
-//   warp 0    : TMA producer.  Q once (two 64-dim halves), then 64-row K and V tiles through a
-//               2-stage ring, all with the 128-byte swizzle;
+// bf16, head_dim 128.  Persistent CTAs, two per SM (one CTA's softmax overlaps the other's MMAs),
+// walk work items (sequence, head, 128-row query tile), longest tiles first; tensor memory, barriers
+// and the pipelines live across items, so an item's loads start while the previous one finishes.
+//   warp 0    : TMA producer.  Q of an item (two 64-dim halves) as soon as the previous item's last
+//               Q K^T has read the Q buffer, 64-row K and V tiles through a 2-stage ring, all with
+//               the 128-byte swizzle;
 //   warp 1    : tensor-memory allocation and the single MMA-issuing thread:
 //               S = Q K^T (128 x 64, K-major operands from shared memory) into one of two S buffers,
 //               O += P V (P read from tensor memory, V as an MN-major shared-memory operand);
@@ -13,9 +15,12 @@
 //               memory), so most tiles never touch O.  P (bf16) overwrites the first half of its
 //               own S buffer.  The same warps normalise O and store the output rows.
 // Tensor memory: O 128 columns, S0 and S1 64 columns each (256 columns per CTA, 512 per SM).
-// Rows past a sequence's length are fetched with the tile (they are masked); in the last tile the
-// surplus V rows are zeroed in shared memory first, since 0 * x must stay 0 for any bit pattern.
-// Every wait is bounded (pipeline.cuh); an abort leaves DL_ERR_TIMEOUT in the status word.
+// Barrier phases are driven by running counters (tiles, K/V stages, items) that every role advances
+// identically.  Rows past a sequence's length are fetched with the tile (they are masked); in the
+// last tile the surplus V rows are zeroed in shared memory first, since 0 * x must stay 0 for any
+// bit pattern.  Every wait is bounded (pipeline.cuh); an abort leaves DL_ERR_TIMEOUT in the status word.
+#include <algorithm>
+
 #include "common.cuh"
 #include "tc05.cuh"
 
@@ -40,36 +45,49 @@ struct AtMaps { alignas(64) unsigned char q[128]; alignas(64) unsigned char k[12
 
 struct AtArgs {
   const int32_t* cache_len; __nv_bfloat16* out; DeviceStatus* status;
-  int32_t H, cap, n_max;
+  int32_t B, H, cap, n_max, q_tiles;
   float scale_log2;
 };
 
+// Work item -> (b, h, query tile); the last query tiles (the longest) come first.  Returns false for
+// an item that lies past its sequence's end.
+struct AtItem { int b, h, q0, n, n_tiles, row_base; };
+__device__ __forceinline__ bool at_item(const AtArgs& a, int item, AtItem& I) {
+  const int bh_count = a.B * a.H;
+  const int qt = a.q_tiles - 1 - item / bh_count;
+  const int bh = item - (item / bh_count) * bh_count;
+  I.b = bh / a.H;
+  I.h = bh - I.b * a.H;
+  I.n = min(max(a.cache_len[I.b], 0), min(a.cap, a.n_max));
+  I.q0 = qt * kAtBM;
+  if (I.q0 >= I.n) return false;
+  const int kv_end = min(I.n, I.q0 + kAtBM);                     // keys any row of this tile may see
+  I.n_tiles = (kv_end + kAtBN - 1) / kAtBN;
+  I.row_base = bh * a.cap;                                        // first row of this (b, h) in the caches
+  return true;
+}
+
 __global__ void __launch_bounds__(kAtThreads, 2)
 attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
-  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const int n = min(max(a.cache_len[b], 0), min(a.cap, a.n_max));
-  const int q0 = qt * kAtBM;
-  if (q0 >= n) return;
-  const int kv_end = min(n, q0 + kAtBM);                         // keys any row of this tile may see
-  const int n_tiles = (kv_end + kAtBN - 1) / kAtBN;
-  const int row_base = (b * a.H + h) * a.cap;                    // first row of this (b, h) in the caches
-
   extern __shared__ char smem_raw[];
   char* smem = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   char* q_s = smem;
   char* st_s = smem + kAtQBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(st_s + kAtStages * kAtStage);
-  uint64_t* q_full = bars;                 // [1]
-  uint64_t* kv_full = bars + 1;            // [2]
+  uint64_t* q_full = bars;                 // [1] per item: Q has landed
+  uint64_t* kv_full = bars + 1;            // [2] per stage use
   uint64_t* kv_empty = bars + 3;           // [2]
-  uint64_t* s_full = bars + 5;             // [2]
-  uint64_t* p_full = bars + 7;             // [2]
-  uint64_t* pv_done = bars + 9;            // [1] one phase per tile: P V of tile j has completed
-  uint64_t* o_final = bars + 10;           // [1] single phase: the last P V has completed
+  uint64_t* s_full = bars + 5;             // [2] per S-buffer use: Q K^T of a tile has completed
+  uint64_t* p_full = bars + 7;             // [2] per S-buffer use: P of a tile is in tensor memory (4 warps)
+  uint64_t* pv_done = bars + 9;            // [1] per tile: its P V has completed
+  uint64_t* o_final = bars + 10;           // [1] per item: its last P V has completed
+  uint64_t* q_empty = bars + 11;           // [1] per item: its last Q K^T has read the Q buffer
+  uint64_t* o_free = bars + 12;            // [1] per item: the epilogue has read O (4 warps)
   __shared__ uint32_t sh_tmem;
   __shared__ int sh_abort;
   volatile int* abort_flag = &sh_abort;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int items = a.B * a.H * a.q_tiles;
 
   if (tid == 0) {
     sh_abort = 0;
@@ -82,6 +100,8 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     }
     mbar_init(smem_u32(pv_done), 1);
     mbar_init(smem_u32(o_final), 1);
+    mbar_init(smem_u32(q_empty), 1);
+    mbar_init(smem_u32(o_free), 4);
     fence_mbar_init();
   }
   if (warp == 1) { tmem_alloc(smem_u32(&sh_tmem), 256); tmem_relinquish(); }
@@ -96,26 +116,37 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(maps.q);
       const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(maps.k);
       const CUtensorMap* mv = reinterpret_cast<const CUtensorMap*>(maps.v);
-      mbar_expect_tx(smem_u32(q_full), kAtQBytes);
-      tma_load_2d(smem_u32(q_s), mq, 0, row_base + q0, smem_u32(q_full));
-      tma_load_2d(smem_u32(q_s + kAtBM * 128), mq, 64, row_base + q0, smem_u32(q_full));
-      int issued = 0;
-      for (int j = 0; j < n_tiles && !*abort_flag; ++j, ++issued) {
-        const int s = j % kAtStages;
-        if (!mbar_wait(smem_u32(&kv_empty[s]), ((j / kAtStages) & 1) ^ 1, abort_flag)) break;
-        const uint32_t fb = smem_u32(&kv_full[s]);
-        mbar_expect_tx(fb, kAtStage);
-        char* st = st_s + (size_t)s * kAtStage;
-        const int r = row_base + j * kAtBN;
-        tma_load_2d(smem_u32(st), mk, 0, r, fb);
-        tma_load_2d(smem_u32(st + kAtBN * 128), mk, 64, r, fb);
-        tma_load_2d(smem_u32(st + kAtTile), mv, 0, r, fb);
-        tma_load_2d(smem_u32(st + kAtTile + kAtBN * 128), mv, 64, r, fb);
+      tma_prefetch_desc(mq); tma_prefetch_desc(mk); tma_prefetch_desc(mv);
+      int n_item = 0, g = 0;                                           // items / tiles issued so far
+      bool q_pending = false;
+      for (int item = blockIdx.x; item < items && !*abort_flag; item += gridDim.x) {
+        AtItem I;
+        if (!at_item(a, item, I)) continue;
+        if (!mbar_wait(smem_u32(q_empty), (n_item & 1) ^ 1, abort_flag)) break;
+        mbar_expect_tx(smem_u32(q_full), kAtQBytes);
+        tma_load_2d(smem_u32(q_s), mq, 0, I.row_base + I.q0, smem_u32(q_full));
+        tma_load_2d(smem_u32(q_s + kAtBM * 128), mq, 64, I.row_base + I.q0, smem_u32(q_full));
+        q_pending = true;
+        ++n_item;
+        for (int j = 0; j < I.n_tiles; ++j, ++g) {
+          const int s = g % kAtStages;
+          if (!mbar_wait(smem_u32(&kv_empty[s]), ((g / kAtStages) & 1) ^ 1, abort_flag)) break;
+          const uint32_t fb = smem_u32(&kv_full[s]);
+          mbar_expect_tx(fb, kAtStage);
+          char* st = st_s + (size_t)s * kAtStage;
+          const int r = I.row_base + j * kAtBN;
+          tma_load_2d(smem_u32(st), mk, 0, r, fb);
+          tma_load_2d(smem_u32(st + kAtBN * 128), mk, 64, r, fb);
+          tma_load_2d(smem_u32(st + kAtTile), mv, 0, r, fb);
+          tma_load_2d(smem_u32(st + kAtTile + kAtBN * 128), mv, 64, r, fb);
+        }
       }
       if (*abort_flag) {
+        // every copy that was issued must land before the CTA's shared memory is released
         report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
-        for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(q_full), 0); ++i) __nanosleep(40);
-        for (int j = max(0, issued - kAtStages); j < issued; ++j)
+        if (q_pending)
+          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(q_full), (n_item - 1) & 1); ++i) __nanosleep(40);
+        for (int j = max(0, g - kAtStages); j < g; ++j)
           for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&kv_full[j % kAtStages]), (j / kAtStages) & 1); ++i)
             __nanosleep(40);
       }
@@ -125,149 +156,171 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_bf16(kAtBM, kAtBN);
       const uint32_t idesc_pv = idesc_bf16(kAtBM, 128, 0, 1);        // B (= V) is MN-major
-      const uint32_t q_addr = smem_u32(q_s);
-      auto issue_qk = [&](int j) {
-        const int s = j % kAtStages;
-        mbar_wait(smem_u32(&kv_full[s]), (j / kAtStages) & 1, abort_flag);
-        tc_fence_after();
-        const uint32_t k_addr = smem_u32(st_s + (size_t)s * kAtStage);
-        const uint32_t d = tmem + kAtColS + (uint32_t)(j & 1) * kAtBN;
+      const uint64_t q_desc = smem_desc_sw128(smem_u32(q_s));
+      const uint64_t k_desc0 = smem_desc_sw128(smem_u32(st_s));
+      const uint64_t v_desc0 = smem_desc_sw128_mn(smem_u32(st_s) + kAtTile, kAtBN * 128);
+      int n_item = 0, g0 = 0;                                          // items / tiles before this item
+      for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        AtItem I;
+        if (!at_item(a, item, I)) continue;
+        auto issue_qk = [&](int j) {
+          const int g = g0 + j, s = g % kAtStages;
+          mbar_wait(smem_u32(&kv_full[s]), (g / kAtStages) & 1, abort_flag);
+          tc_fence_after();
+          const uint64_t kd = k_desc0 + (uint64_t)((s * kAtStage) >> 4);
+          const uint32_t d = tmem + kAtColS + (uint32_t)(g & 1) * kAtBN;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          mma_ss(d, smem_desc_sw128(q_addr + (ks >> 2) * (kAtBM * 128) + (ks & 3) * 32),
-                 smem_desc_sw128(k_addr + (ks >> 2) * (kAtBN * 128) + (ks & 3) * 32), idesc_qk, ks != 0);
-        mma_commit(smem_u32(&s_full[j & 1]));
-      };
-      mbar_wait(smem_u32(q_full), 0, abort_flag);
-      issue_qk(0);
-      for (int j = 0; j < n_tiles; ++j) {
-        if (j + 1 < n_tiles) issue_qk(j + 1);
-        const int s = j % kAtStages;
-        mbar_wait(smem_u32(&p_full[j & 1]), (j >> 1) & 1, abort_flag);
-        tc_fence_after();
-        const uint32_t v_addr = smem_u32(st_s + (size_t)s * kAtStage + kAtTile);
-        const uint32_t p_tmem = tmem + kAtColS + (uint32_t)(j & 1) * kAtBN;
+          for (int ks = 0; ks < 8; ++ks)
+            mma_ss(d, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
+                   kd + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
+          mma_commit(smem_u32(&s_full[g & 1]));
+          if (j == I.n_tiles - 1) mma_commit(smem_u32(q_empty));       // the Q buffer may be refilled
+        };
+        mbar_wait(smem_u32(q_full), n_item & 1, abort_flag);
+        issue_qk(0);
+        for (int j = 0; j < I.n_tiles; ++j) {
+          if (j + 1 < I.n_tiles) issue_qk(j + 1);
+          const int g = g0 + j, s = g % kAtStages;
+          mbar_wait(smem_u32(&p_full[g & 1]), (g >> 1) & 1, abort_flag);
+          if (j == 0) mbar_wait(smem_u32(o_free), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
+          tc_fence_after();
+          const uint64_t vd = v_desc0 + (uint64_t)((s * kAtStage) >> 4);
+          const uint32_t p_tmem = tmem + kAtColS + (uint32_t)(g & 1) * kAtBN;
 #pragma unroll
-        for (int ks = 0; ks < kAtBN / 16; ++ks)
-          mma_ts(tmem + kAtColO, p_tmem + ks * 8, smem_desc_sw128_mn(v_addr + ks * 2048, kAtBN * 128), idesc_pv,
-                 (j | ks) != 0);
-        mma_commit(smem_u32(&kv_empty[s]));
-        mma_commit(smem_u32(pv_done));
-        if (j == n_tiles - 1) mma_commit(smem_u32(o_final));
+          for (int ks = 0; ks < kAtBN / 16; ++ks)
+            mma_ts(tmem + kAtColO, p_tmem + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), idesc_pv, (j | ks) != 0);
+          mma_commit(smem_u32(&kv_empty[s]));
+          mma_commit(smem_u32(pv_done));
+          if (j == I.n_tiles - 1) mma_commit(smem_u32(o_final));
+        }
+        g0 += I.n_tiles;
+        ++n_item;
       }
     }
   } else {
     // ---------------------------------------------------------------- softmax / epilogue warps
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                                  // row within the query tile
-    const int grow = q0 + row;                                         // row within the sequence
     const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
-    float m_used = -INFINITY, l_run = 0.f;
-    for (int j = 0; j < n_tiles; ++j) {
-      const int sb = j & 1;
-      mbar_wait(smem_u32(&s_full[sb]), (j >> 1) & 1, abort_flag);
-      tc_fence_after();
-      const uint32_t s_addr = tmem + lane_off + kAtColS + (uint32_t)sb * kAtBN;
-      uint32_t sr[64];
-      tmem_ld32(s_addr, sr);
-      tmem_ld32(s_addr + 32, sr + 32);
-      tmem_ld_wait();
-      const int c0 = j * kAtBN;
-      // raw scores stay unscaled: max commutes with the (positive) scale and the scale is folded into
-      // the exponent's FMA.  Only tiles that reach past the tile's first row need the causal mask.
-      float mx = -INFINITY;
-      if (c0 + kAtBN - 1 > q0) {
+    int n_item = 0, g0 = 0;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+      AtItem I;
+      if (!at_item(a, item, I)) continue;
+      const int grow = I.q0 + row;                                     // row within the sequence
+      const int kv_end = min(I.n, I.q0 + kAtBM);
+      float m_used = -INFINITY, l_run = 0.f;
+      for (int j = 0; j < I.n_tiles; ++j) {
+        const int g = g0 + j, sb = g & 1;
+        mbar_wait(smem_u32(&s_full[sb]), (g >> 1) & 1, abort_flag);
+        tc_fence_after();
+        const uint32_t s_addr = tmem + lane_off + kAtColS + (uint32_t)sb * kAtBN;
+        uint32_t sr[64];
+        tmem_ld32(s_addr, sr);
+        tmem_ld32(s_addr + 32, sr + 32);
+        tmem_ld_wait();
+        const int c0 = j * kAtBN;
+        // raw scores stay unscaled: max commutes with the (positive) scale and the scale is folded into
+        // the exponent's FMA.  Only tiles that reach past the tile's first row need the causal mask.
+        float mx = -INFINITY;
+        if (c0 + kAtBN - 1 > I.q0) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          const float v = (c0 + c > grow) ? -INFINITY : __uint_as_float(sr[c]);
-          sr[c] = __float_as_uint(v);
-          mx = fmaxf(mx, v);
-        }
-      } else {
-#pragma unroll
-        for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
-      }
-      mx *= a.scale_log2;
-      if (j == 0) {
-        m_used = mx;                        // column 0 is visible to every row, so mx is finite
-      } else {
-        const bool need = mx > m_used + kRescaleStep;
-        if (__any_sync(0xffffffffu, need)) {
-          mbar_wait(smem_u32(pv_done), (j - 1) & 1, abort_flag);      // O must be at rest
-          tc_fence_after();
-          const float corr = need ? fast_exp2(m_used - mx) : 1.0f;
-          if (need) m_used = mx;
-          l_run *= corr;
-#pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
-            uint32_t o[32];
-            tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
-            tmem_st32(tmem + lane_off + kAtColO + cc * 32, o);
+          for (int c = 0; c < 64; ++c) {
+            const float v = (c0 + c > grow) ? -INFINITY : __uint_as_float(sr[c]);
+            sr[c] = __float_as_uint(v);
+            mx = fmaxf(mx, v);
           }
-          tmem_st_wait();
+        } else {
+#pragma unroll
+          for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
+        }
+        mx *= a.scale_log2;
+        if (j == 0) {
+          m_used = mx;                        // column 0 is visible to every row, so mx is finite
+        } else {
+          const bool need = mx > m_used + kRescaleStep;
+          if (__any_sync(0xffffffffu, need)) {
+            // O must be at rest: the P V of the previous tile.  (At this point that phase is either
+            // running or just completed, never further along, so the parity is unambiguous.)
+            mbar_wait(smem_u32(pv_done), (g - 1) & 1, abort_flag);
+            tc_fence_after();
+            const float corr = need ? fast_exp2(m_used - mx) : 1.0f;
+            if (need) m_used = mx;
+            l_run *= corr;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+              uint32_t o[32];
+              tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
+              tmem_st32(tmem + lane_off + kAtColO + cc * 32, o);
+            }
+            tmem_st_wait();
+          }
+        }
+        uint32_t pw[32];
+        const float neg_m = -m_used;
+        float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c]), a.scale_log2, neg_m));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), a.scale_log2, neg_m));
+          l0 += p0;
+          l1 += p1;
+          __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+          pw[c] = *reinterpret_cast<uint32_t*>(&pk);
+        }
+        l_run += l0 + l1;
+        tmem_st32(s_addr, pw);                                             // P overwrites its own S buffer
+        tmem_st_wait();
+        if (j == I.n_tiles - 1 && kv_end < c0 + kAtBN) {
+          // ragged last tile: zero the V rows past the sequence's end (both 64-dim halves)
+          const int s = g % kAtStages;
+          mbar_wait(smem_u32(&kv_full[s]), (g / kAtStages) & 1, abort_flag);
+          char* vz = st_s + (size_t)s * kAtStage + kAtTile;
+          const int first = kv_end - c0;
+          for (int u = (warp - 2) * 32 + lane; u < 2 * kAtBN * 8; u += 128) {
+            const int r = (u >> 3) & (kAtBN - 1);
+            if (r >= first)
+              *reinterpret_cast<uint4*>(vz + (u >> 9) * (kAtBN * 128) + r * 128 + (u & 7) * 16) = make_uint4(0, 0, 0, 0);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&p_full[sb]));
+      }
+      // ---- epilogue: O / l -> bf16 -> out[b][row][h][:]
+      mbar_wait(smem_u32(o_final), n_item & 1, abort_flag);
+      tc_fence_after();
+      const float inv = 1.0f / l_run;
+      __nv_bfloat16* orow = a.out + (((size_t)I.b * a.n_max + grow) * a.H + I.h) * 128;
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t o[32];
+        tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
+        tmem_ld_wait();
+        if (cc == 3) {                                   // O is in registers: the next item may overwrite it
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(o_free));
+        }
+        if (grow < I.n) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint4 w;
+            __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+            __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+            __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+            w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
+            w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
+            *reinterpret_cast<uint4*>(orow + cc * 32 + i) = w;
+          }
         }
       }
-      uint32_t pw[32];
-#pragma unroll
-      const float neg_m = -m_used;
-      float l0 = 0.f, l1 = 0.f;
-#pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c]), a.scale_log2, neg_m));
-        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), a.scale_log2, neg_m));
-        l0 += p0;
-        l1 += p1;
-        __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-        pw[c] = *reinterpret_cast<uint32_t*>(&pk);
-      }
-      l_run += l0 + l1;
-      tmem_st32(s_addr, pw);                                             // P overwrites its own S buffer
-      tmem_st_wait();
-      if (j == n_tiles - 1 && kv_end < c0 + kAtBN) {
-        // ragged last tile: zero the V rows past the sequence's end (both 64-dim halves)
-        const int s = j % kAtStages;
-        mbar_wait(smem_u32(&kv_full[s]), (j / kAtStages) & 1, abort_flag);
-        char* vz = st_s + (size_t)s * kAtStage + kAtTile;
-        const int first = kv_end - c0;
-        for (int u = (warp - 2) * 32 + lane; u < 2 * kAtBN * 8; u += 128) {
-          const int r = (u >> 3) & (kAtBN - 1);
-          if (r >= first)
-            *reinterpret_cast<uint4*>(vz + (u >> 9) * (kAtBN * 128) + r * 128 + (u & 7) * 16) = make_uint4(0, 0, 0, 0);
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&p_full[sb]));
-    }
-    // ---- epilogue: O / l -> bf16 -> out[b][row][h][:]
-    // (a parity wait on pv_done would be ambiguous here: a warp can get here while the P V of the
-    //  tile before the last is still running, two phases behind)
-    mbar_wait(smem_u32(o_final), 0, abort_flag);
-    tc_fence_after();
-    const float inv = 1.0f / l_run;
-    __nv_bfloat16* orow = a.out + (((size_t)b * a.n_max + grow) * a.H + h) * 128;
-#pragma unroll
-    for (int cc = 0; cc < 4; ++cc) {
-      uint32_t o[32];
-      tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
-      tmem_ld_wait();
-      if (grow < n) {
-#pragma unroll
-        for (int i = 0; i < 32; i += 8) {
-          uint4 w;
-          __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
-          __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-          __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
-          __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
-          w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
-          w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
-          *reinterpret_cast<uint4*>(orow + cc * 32 + i) = w;
-        }
-      }
+      g0 += I.n_tiles;
+      ++n_item;
     }
     if (*abort_flag && row == 0) report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
   }
@@ -299,7 +352,7 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
     return cudaErrorInvalidValue;
   AtArgs a;
   a.cache_len = cache_len; a.out = static_cast<__nv_bfloat16*>(out); a.status = ctx->ws.base ? ctx->ws.status : nullptr;
-  a.H = d.n_heads; a.cap = cap; a.n_max = n_max;
+  a.B = B; a.H = d.n_heads; a.cap = cap; a.n_max = n_max; a.q_tiles = (n_max + kAtBM - 1) / kAtBM;
   a.scale_log2 = scale * 1.4426950408889634f;
   static int attr_set[64];
   if (!attr_set[ctx->device & 63]) {
@@ -307,7 +360,9 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
     if (e != cudaSuccess) return e;
     attr_set[ctx->device & 63] = 1;
   }
-  dim3 grid((n_max + kAtBM - 1) / kAtBM, d.n_heads, B);
+  const long long items = (long long)B * d.n_heads * a.q_tiles;
+  if (items >= (1LL << 31)) return cudaErrorInvalidValue;
+  const int grid = (int)std::min<long long>(items, 2LL * ctx->sm_count);
   attn_prefill_tc_kernel<<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
   return cudaGetLastError();
 }
