@@ -1,0 +1,73 @@
+"""C-ABI behaviour on the GPU: argument checks return error codes (nothing traps), the layer-stack
+call equals per-layer calls bit for bit, and a decode step is reproducible."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_00876_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def test_invalid_arguments_are_refused_with_codes():
+    from paper_2412_00876_b200 import binding as dl
+    lib = dl.lib()
+    h = C.c_void_p()
+    bad = dl.ModelDesc(4096, 32, 96, 1024, dl.DL_BF16)                 # head_dim 96 is not built
+    assert lib.dl_create(C.byref(h), 0, C.byref(bad)) == dl.DL_ERR_UNSUPPORTED
+    assert lib.dl_create(C.byref(h), 99, C.byref(dl.ModelDesc(4096, 32, 128, 1024, dl.DL_BF16))) == dl.DL_ERR_CUDA
+    ctx = dl.Context(256, 4, 128, 64, torch.bfloat16, 0, max_batch=2, max_rows=8, cap=64)
+    t = torch.zeros(2 * 4 * 64 * 128 + 8, dtype=torch.bfloat16, device=DEV)
+    ln = torch.zeros(2, dtype=torch.int32, device=DEV)
+    p = t.data_ptr()
+    # NULL tensor, misaligned tensor, cap beyond the workspace, batch beyond the workspace
+    assert lib.dl_sparse_attn_decode(ctx._h, None, p, p, p, p, ln.data_ptr(), None, 2, 64, 0.1, p, None) == dl.DL_ERR_INVALID_ARG
+    assert lib.dl_sparse_attn_decode(ctx._h, p + 2, p, p, p, p, ln.data_ptr(), None, 2, 64, 0.1, p, None) == dl.DL_ERR_ALIGNMENT
+    assert lib.dl_sparse_attn_decode(ctx._h, p, p, p, p, p, ln.data_ptr(), None, 2, 128, 0.1, p, None) == dl.DL_ERR_WORKSPACE
+    assert lib.dl_sparse_attn_decode(ctx._h, p, p, p, p, p, ln.data_ptr(), None, 3, 64, 0.1, p, None) == dl.DL_ERR_WORKSPACE
+    assert lib.dl_sparse_attn_prefill(ctx._h, p, p, p, ln.data_ptr(), 2, 64, 65, 0.1, p, None) == dl.DL_ERR_INVALID_ARG   # n_max > cap
+    assert lib.dl_sparse_attn_prefill(ctx._h, p, p, p, ln.data_ptr(), 2, 64, 64, -1.0, p, None) == dl.DL_ERR_INVALID_ARG  # scale <= 0
+    assert lib.dl_compact_kv(ctx._h, p, p, None, 0, None, 2, 4, p, None, 64, ln.data_ptr(), 1, None) == dl.DL_ERR_INVALID_ARG  # v_src without v_cache
+    assert lib.dl_set_option(ctx._h, 77, 1) == dl.DL_ERR_INVALID_ARG
+    assert lib.dl_topk_from_scores(ctx._h, p, None, ln.data_ptr(), 1, 20000, None, 0, p, None) == dl.DL_ERR_UNSUPPORTED
+    # empty problems are fine
+    assert lib.dl_sparse_attn_decode(ctx._h, None, None, None, None, None, None, None, 0, 64, 0.1, None, None) == dl.DL_OK
+    assert ctx.device_status()[0] == 0
+    ctx.close()
+
+
+def test_layer_stack_equals_per_layer_calls_and_is_reproducible():
+    from paper_2412_00876_b200 import binding as dl
+    cfg = wl.CONFIGS[3]
+    B, H, D, L, cap = 32, 32, 128, 3, 512                  # 1024 (b,h) pairs: unsplit, overlapped launches
+    ctx = dl.Context(256, H, D, 64, torch.bfloat16, 0, max_batch=B, max_rows=B, cap=cap)
+    mk = lambda s, shape, sub=0: wl.device_normal(cfg, s, shape, DEV, sub=sub)
+    q, kt, vt = mk(wl.S_DEC_Q, (L, B, H, D)), mk(wl.S_DEC_K, (L, B, H, D)), mk(wl.S_DEC_V, (L, B, H, D))
+    base_k = [mk(wl.S_CACHE_K, (B, H, cap, D), l) for l in range(L)]
+    base_v = [mk(wl.S_CACHE_V, (B, H, cap, D), l) for l in range(L)]
+    ln = torch.from_numpy(wl.host_rng(3, wl.S_LEN).integers(0, cap, B).astype(np.int32)).to(DEV)
+    keep = torch.from_numpy((np.arange(B) % 3 != 0).astype(np.uint8)).to(DEV)
+    scale = 1 / np.sqrt(D)
+    results = []
+    for mode in ("per-layer", "stack", "stack"):
+        kc, vc = [t.clone() for t in base_k], [t.clone() for t in base_v]
+        out = torch.zeros(L, B, H, D, dtype=torch.bfloat16, device=DEV)
+        if mode == "per-layer":
+            for l in range(L):
+                ctx.sparse_attn_decode(q[l], kt[l], vt[l], kc[l], vc[l], ln, keep, scale, out[l])
+        else:
+            ctx.sparse_attn_decode_layers(q, kt, vt, ctx.pointer_array(kc), ctx.pointer_array(vc), L, cap, ln, keep,
+                                          scale, out)
+        torch.cuda.synchronize()
+        results.append((out, kc, vc))
+    ref = results[0]
+    for out, kc, vc in results[1:]:
+        assert torch.equal(out.view(torch.int16), ref[0].view(torch.int16))
+        for l in range(L):
+            assert torch.equal(kc[l].view(torch.int16), ref[1][l].view(torch.int16))
+            assert torch.equal(vc[l].view(torch.int16), ref[2][l].view(torch.int16))
+    assert ctx.device_status()[0] == 0
+    ctx.close()
