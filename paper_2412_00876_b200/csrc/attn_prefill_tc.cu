@@ -4,8 +4,9 @@
 // walk work items (sequence, head, 128-row query tile), longest tiles first; tensor memory, barriers
 // and the pipelines live across items, so an item's loads start while the previous one finishes.
 //   warp 0    : TMA producer.  Q of an item (two 64-dim halves) as soon as the previous item's last
-//               Q K^T has read the Q buffer, 64-row K and V tiles through a 2-stage ring, all with
-//               the 128-byte swizzle;
+//               Q K^T has read the Q buffer; 64-row K tiles and V tiles through two separate 2-slot
+//               rings (a K slot is free once its Q K^T has run, long before the V slot of the same
+//               tile, so the next K is in flight a whole softmax earlier), all with the 128-byte swizzle;
 //   warp 1    : tensor-memory allocation and the single MMA-issuing thread:
 //               S = Q K^T (128 x 64, K-major operands from shared memory) into one of two S buffers,
 //               O += P V (P read from tensor memory, V as an MN-major shared-memory operand);
@@ -39,6 +40,13 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// max of three in one instruction
+__device__ __forceinline__ float fmax3(float x, float y, float z) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(x), "f"(y), "f"(z));
+  return r;
 }
 
 struct AtMaps { alignas(64) unsigned char q[128]; alignas(64) unsigned char k[128]; alignas(64) unsigned char v[128]; };
@@ -75,14 +83,16 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
   char* st_s = smem + kAtQBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(st_s + kAtStages * kAtStage);
   uint64_t* q_full = bars;                 // [1] per item: Q has landed
-  uint64_t* kv_full = bars + 1;            // [2] per stage use
-  uint64_t* kv_empty = bars + 3;           // [2]
-  uint64_t* s_full = bars + 5;             // [2] per S-buffer use: Q K^T of a tile has completed
-  uint64_t* p_full = bars + 7;             // [2] per S-buffer use: P of a tile is in tensor memory (4 warps)
-  uint64_t* pv_done = bars + 9;            // [1] per tile: its P V has completed
-  uint64_t* o_final = bars + 10;           // [1] per item: its last P V has completed
-  uint64_t* q_empty = bars + 11;           // [1] per item: its last Q K^T has read the Q buffer
-  uint64_t* o_free = bars + 12;            // [1] per item: the epilogue has read O (4 warps)
+  uint64_t* k_full = bars + 1;             // [2] per K-slot use
+  uint64_t* k_empty = bars + 3;            // [2] the slot's Q K^T has completed
+  uint64_t* v_full = bars + 5;             // [2] per V-slot use
+  uint64_t* v_empty = bars + 7;            // [2] the slot's P V has completed
+  uint64_t* s_full = bars + 9;             // [2] per S-buffer use: Q K^T of a tile has completed
+  uint64_t* p_full = bars + 11;            // [2] per S-buffer use: P of a tile is in tensor memory (4 warps)
+  uint64_t* pv_done = bars + 13;           // [1] per tile: its P V has completed
+  uint64_t* o_final = bars + 14;           // [1] per item: its last P V has completed
+  uint64_t* q_empty = bars + 15;           // [1] per item: its last Q K^T has read the Q buffer
+  uint64_t* o_free = bars + 16;            // [1] per item: the epilogue has read O (4 warps)
   __shared__ uint32_t sh_tmem;
   __shared__ int sh_abort;
   volatile int* abort_flag = &sh_abort;
@@ -93,8 +103,10 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     sh_abort = 0;
     mbar_init(smem_u32(q_full), 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&kv_full[i]), 1);
-      mbar_init(smem_u32(&kv_empty[i]), 1);
+      mbar_init(smem_u32(&k_full[i]), 1);
+      mbar_init(smem_u32(&k_empty[i]), 1);
+      mbar_init(smem_u32(&v_full[i]), 1);
+      mbar_init(smem_u32(&v_empty[i]), 1);
       mbar_init(smem_u32(&s_full[i]), 1);
       mbar_init(smem_u32(&p_full[i]), 4);
     }
@@ -117,9 +129,20 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(maps.k);
       const CUtensorMap* mv = reinterpret_cast<const CUtensorMap*>(maps.v);
       tma_prefetch_desc(mq); tma_prefetch_desc(mk); tma_prefetch_desc(mv);
-      int n_item = 0, g = 0;                                           // items / tiles issued so far
-      bool q_pending = false;
-      for (int item = blockIdx.x; item < items && !*abort_flag; item += gridDim.x) {
+      int n_item = 0, gk = 0, gv = 0;                                  // items / K tiles / V tiles issued so far
+      bool q_pending = false, ok = true;
+      // tile g of this CTA's running count -> slot g & 1 of either ring
+      auto load_tile = [&](uint64_t* full, uint64_t* empty, const CUtensorMap* m, int g, int r, int off) {
+        const int s = g & 1;
+        if (!mbar_wait(smem_u32(&empty[s]), ((g >> 1) & 1) ^ 1, abort_flag)) return false;
+        const uint32_t fb = smem_u32(&full[s]);
+        mbar_expect_tx(fb, kAtTile);
+        char* st = st_s + (size_t)s * kAtStage + off;
+        tma_load_2d(smem_u32(st), m, 0, r, fb);
+        tma_load_2d(smem_u32(st + kAtBN * 128), m, 64, r, fb);
+        return true;
+      };
+      for (int item = blockIdx.x; item < items && ok && !*abort_flag; item += gridDim.x) {
         AtItem I;
         if (!at_item(a, item, I)) continue;
         if (!mbar_wait(smem_u32(q_empty), (n_item & 1) ^ 1, abort_flag)) break;
@@ -128,17 +151,17 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         tma_load_2d(smem_u32(q_s + kAtBM * 128), mq, 64, I.row_base + I.q0, smem_u32(q_full));
         q_pending = true;
         ++n_item;
-        for (int j = 0; j < I.n_tiles; ++j, ++g) {
-          const int s = g % kAtStages;
-          if (!mbar_wait(smem_u32(&kv_empty[s]), ((g / kAtStages) & 1) ^ 1, abort_flag)) break;
-          const uint32_t fb = smem_u32(&kv_full[s]);
-          mbar_expect_tx(fb, kAtStage);
-          char* st = st_s + (size_t)s * kAtStage;
-          const int r = I.row_base + j * kAtBN;
-          tma_load_2d(smem_u32(st), mk, 0, r, fb);
-          tma_load_2d(smem_u32(st + kAtBN * 128), mk, 64, r, fb);
-          tma_load_2d(smem_u32(st + kAtTile), mv, 0, r, fb);
-          tma_load_2d(smem_u32(st + kAtTile + kAtBN * 128), mv, 64, r, fb);
+        // same order as the MMA warp consumes them: K(0), then K(j+1) before V(j)
+        ok = load_tile(k_full, k_empty, mk, gk, I.row_base, 0);
+        if (ok) ++gk;
+        for (int j = 0; j < I.n_tiles && ok; ++j) {
+          if (j + 1 < I.n_tiles) {
+            ok = load_tile(k_full, k_empty, mk, gk, I.row_base + (j + 1) * kAtBN, 0);
+            if (!ok) break;
+            ++gk;
+          }
+          ok = load_tile(v_full, v_empty, mv, gv, I.row_base + j * kAtBN, kAtTile);
+          if (ok) ++gv;
         }
       }
       if (*abort_flag) {
@@ -146,9 +169,10 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
         if (q_pending)
           for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(q_full), (n_item - 1) & 1); ++i) __nanosleep(40);
-        for (int j = max(0, g - kAtStages); j < g; ++j)
-          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&kv_full[j % kAtStages]), (j / kAtStages) & 1); ++i)
-            __nanosleep(40);
+        for (int j = max(0, gk - 2); j < gk; ++j)
+          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&k_full[j & 1]), (j >> 1) & 1); ++i) __nanosleep(40);
+        for (int j = max(0, gv - 2); j < gv; ++j)
+          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&v_full[j & 1]), (j >> 1) & 1); ++i) __nanosleep(40);
       }
     }
   } else if (warp == 1) {
@@ -165,7 +189,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         if (!at_item(a, item, I)) continue;
         auto issue_qk = [&](int j) {
           const int g = g0 + j, s = g % kAtStages;
-          mbar_wait(smem_u32(&kv_full[s]), (g / kAtStages) & 1, abort_flag);
+          mbar_wait(smem_u32(&k_full[s]), (g / kAtStages) & 1, abort_flag);
           tc_fence_after();
           const uint64_t kd = k_desc0 + (uint64_t)((s * kAtStage) >> 4);
           const uint32_t d = tmem + kAtColS + (uint32_t)(g & 1) * kAtBN;
@@ -174,6 +198,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
             mma_ss(d, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
                    kd + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
           mma_commit(smem_u32(&s_full[g & 1]));
+          mma_commit(smem_u32(&k_empty[s]));
           if (j == I.n_tiles - 1) mma_commit(smem_u32(q_empty));       // the Q buffer may be refilled
         };
         mbar_wait(smem_u32(q_full), n_item & 1, abort_flag);
@@ -183,13 +208,14 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           const int g = g0 + j, s = g % kAtStages;
           mbar_wait(smem_u32(&p_full[g & 1]), (g >> 1) & 1, abort_flag);
           if (j == 0) mbar_wait(smem_u32(o_free), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
+          mbar_wait(smem_u32(&v_full[s]), (g / kAtStages) & 1, abort_flag);
           tc_fence_after();
           const uint64_t vd = v_desc0 + (uint64_t)((s * kAtStage) >> 4);
           const uint32_t p_tmem = tmem + kAtColS + (uint32_t)(g & 1) * kAtBN;
 #pragma unroll
           for (int ks = 0; ks < kAtBN / 16; ++ks)
             mma_ts(tmem + kAtColO, p_tmem + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), idesc_pv, (j | ks) != 0);
-          mma_commit(smem_u32(&kv_empty[s]));
+          mma_commit(smem_u32(&v_empty[s]));
           mma_commit(smem_u32(pv_done));
           if (j == I.n_tiles - 1) mma_commit(smem_u32(o_final));
         }
@@ -221,19 +247,19 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         const int c0 = j * kAtBN;
         // raw scores stay unscaled: max commutes with the (positive) scale and the scale is folded into
         // the exponent's FMA.  Only tiles that reach past the tile's first row need the causal mask.
-        float mx = -INFINITY;
         if (c0 + kAtBN - 1 > I.q0) {
 #pragma unroll
-          for (int c = 0; c < 64; ++c) {
-            const float v = (c0 + c > grow) ? -INFINITY : __uint_as_float(sr[c]);
-            sr[c] = __float_as_uint(v);
-            mx = fmaxf(mx, v);
-          }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
+          for (int c = 0; c < 64; ++c)
+            if (c0 + c > grow) sr[c] = 0xFF800000u;                          // -inf
         }
-        mx *= a.scale_log2;
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};       // four independent chains
+#pragma unroll
+        for (int c = 0; c < 64; c += 8) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
+        }
+        float mx = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
         if (j == 0) {
           m_used = mx;                        // column 0 is visible to every row, so mx is finite
         } else {
@@ -276,7 +302,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         if (j == I.n_tiles - 1 && kv_end < c0 + kAtBN) {
           // ragged last tile: zero the V rows past the sequence's end (both 64-dim halves)
           const int s = g % kAtStages;
-          mbar_wait(smem_u32(&kv_full[s]), (g / kAtStages) & 1, abort_flag);
+          mbar_wait(smem_u32(&v_full[s]), (g / kAtStages) & 1, abort_flag);
           char* vz = st_s + (size_t)s * kAtStage + kAtTile;
           const int first = kv_end - c0;
           for (int u = (warp - 2) * 32 + lane; u < 2 * kAtBN * 8; u += 128) {
