@@ -153,10 +153,23 @@ def micro(args):
     torch.cuda.synchronize()
     ts = sorted(a.elapsed_time(b) for a, b in ev)
     med = ts[len(ts) // 2]
+    # the same launches back to back under one event pair: a launch that is shorter than the host's
+    # own call cost shows that cost in the per-launch figure above, not here once the queue is full
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    gate = torch.empty(1 << 28, dtype=torch.uint8, device=dev)
+    gate.zero_()                                              # keeps the device busy while the queue fills
+    a.record()
+    for i in range(args.steps):
+        calls[i % NL]()
+    b.record()
+    torch.cuda.synchronize()
+    queued = a.elapsed_time(b) / args.steps
     code, detail = ctx.device_status()
     rate = work / (med * 1e-3) / (1e9 if unit == "GB/s" else 1e12)
     print(json.dumps({"micro": args.micro, "workload": cfg.name, "median_us": med * 1e3, "min_us": ts[0] * 1e3,
                       "algorithmic_work": work, "rate": rate, "unit": unit, "launches": args.steps,
+                      "queued_us": queued * 1e3,
+                      "queued_rate": work / (queued * 1e-3) / (1e9 if unit == "GB/s" else 1e12),
                       "device_status": code}), flush=True)
     ctx.close()
 
