@@ -110,8 +110,9 @@ def micro(args):
                 ln.zero_()
                 ctx.compact_kv(src[2 * l], src[2 * l + 1], keep, t_src, kc[l], vc[l], ln, commit=True)
             out = torch.empty(B, cfg.n0, H, D, dtype=tdt, device=dev)
+            qs = [wl.device_normal(cfg, wl.S_Q, (B, H, cfg.cap, D), dev, sub=l) for l in range(NL)]
             work, unit = 2.0 * D * cfg.n0 * (cfg.n0 + 1) * H * B, "TFLOP/s"
-            calls = [lambda l=l: ctx.sparse_attn_prefill(kc[l], kc[l], vc[l], ln, cfg.n0, scale, out)
+            calls = [lambda l=l: ctx.sparse_attn_prefill(qs[l], kc[l], vc[l], ln, cfg.n0, scale, out)
                      for l in range(NL)]
     elif args.micro == "nocache":
         # one pass of decoding WITHOUT cache for one layer (Eq. 12): decide all N_OT generated tokens, rebuild the

@@ -3,6 +3,8 @@
 // bf16, head_dim 128.  Persistent CTAs, two per SM (one CTA's softmax overlaps the other's MMAs),
 // walk work items (sequence, head, 128-row query tile), longest tiles first; tensor memory, barriers
 // and the pipelines live across items, so an item's loads start while the previous one finishes.
+// Query tiles are aligned to the END of a sequence (rows [n-128(t+1), n-128t)), so the ragged tile is
+// the one at the top of the causal triangle, where it needs the fewest key tiles.
 //   warp 0    : TMA producer.  Q of an item (two 64-dim halves) as soon as the previous item's last
 //               Q K^T has read the Q buffer; 64-row K tiles and V tiles through two separate 2-slot
 //               rings (a K slot is free once its Q K^T has run, long before the V slot of the same
@@ -14,7 +16,9 @@
 //   warps 2-5 : softmax, one query row per thread, straight out of tensor memory.  The running
 //               maximum is only raised when it grows by more than 2^8 (then O is rescaled in tensor
 //               memory), so most tiles never touch O.  P (bf16) overwrites the first half of its
-//               own S buffer.  The same warps normalise O and store the output rows.
+//               own S buffer.  The same warps normalise O and store the output rows, staged
+//               through a small per-warp buffer so that each store instruction writes whole
+//               64-byte row segments.
 // Tensor memory: O 128 columns, S0 and S1 64 columns each (256 columns per CTA, 512 per SM).
 // Barrier phases are driven by running counters (tiles, K/V stages, items) that every role advances
 // identically.  Rows past a sequence's length are fetched with the tile (they are masked); in the
@@ -31,7 +35,8 @@ constexpr int kAtBM = 128, kAtBN = 64, kAtStages = 2, kAtThreads = 192;
 constexpr int kAtQBytes = 2 * kAtBM * 128;            // 32 KB: two [128 rows][64 dims] halves
 constexpr int kAtTile = 2 * kAtBN * 128;              // 16 KB: two [64 rows][64 dims] halves
 constexpr int kAtStage = 2 * kAtTile;                 // K tile + V tile
-constexpr size_t kAtSmem = kAtQBytes + kAtStages * kAtStage + 1024 + 256;
+constexpr int kAtOutStage = 4 * 2048;                 // per softmax warp: 32 rows x 32 columns of bf16 output
+constexpr size_t kAtSmem = kAtQBytes + kAtStages * kAtStage + kAtOutStage + 1024 + 256;
 constexpr uint32_t kAtColO = 0, kAtColS = 128;        // tensor-memory columns: O | S0 | S1
 constexpr float kRescaleStep = 8.0f;                  // log2 units by which the maximum may lag
 
@@ -57,20 +62,21 @@ struct AtArgs {
   float scale_log2;
 };
 
-// Work item -> (b, h, query tile); the last query tiles (the longest) come first.  Returns false for
-// an item that lies past its sequence's end.
-struct AtItem { int b, h, q0, n, n_tiles, row_base; };
+// Work item -> (b, h, query tile).  Tile t counts from the sequence's end (the longest first): it owns
+// rows [q_hi - 128, q_hi) with q_hi = n - 128 t; the tile at the top is clipped to start at row 0 (it
+// loads rows [0, 128) and owns the first q_hi of them).  Returns false for a tile the sequence lacks.
+struct AtItem { int b, h, q0, q_hi, n, n_tiles, row_base; };
 __device__ __forceinline__ bool at_item(const AtArgs& a, int item, AtItem& I) {
   const int bh_count = a.B * a.H;
-  const int qt = a.q_tiles - 1 - item / bh_count;
-  const int bh = item - (item / bh_count) * bh_count;
+  const int t = item / bh_count;
+  const int bh = item - t * bh_count;
   I.b = bh / a.H;
   I.h = bh - I.b * a.H;
   I.n = min(max(a.cache_len[I.b], 0), min(a.cap, a.n_max));
-  I.q0 = qt * kAtBM;
-  if (I.q0 >= I.n) return false;
-  const int kv_end = min(I.n, I.q0 + kAtBM);                     // keys any row of this tile may see
-  I.n_tiles = (kv_end + kAtBN - 1) / kAtBN;
+  I.q_hi = I.n - t * kAtBM;
+  if (I.q_hi <= 0) return false;
+  I.q0 = max(I.q_hi - kAtBM, 0);
+  I.n_tiles = (I.q_hi + kAtBN - 1) / kAtBN;                       // keys any owned row may see: [0, q_hi)
   I.row_base = bh * a.cap;                                        // first row of this (b, h) in the caches
   return true;
 }
@@ -83,16 +89,16 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
   char* st_s = smem + kAtQBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(st_s + kAtStages * kAtStage);
   uint64_t* q_full = bars;                 // [1] per item: Q has landed
-  uint64_t* k_full = bars + 1;             // [2] per K-slot use
-  uint64_t* k_empty = bars + 3;            // [2] the slot's Q K^T has completed
-  uint64_t* v_full = bars + 5;             // [2] per V-slot use
-  uint64_t* v_empty = bars + 7;            // [2] the slot's P V has completed
-  uint64_t* s_full = bars + 9;             // [2] per S-buffer use: Q K^T of a tile has completed
-  uint64_t* p_full = bars + 11;            // [2] per S-buffer use: P of a tile is in tensor memory (4 warps)
-  uint64_t* pv_done = bars + 13;           // [1] per tile: its P V has completed
-  uint64_t* o_final = bars + 14;           // [1] per item: its last P V has completed
-  uint64_t* q_empty = bars + 15;           // [1] per item: its last Q K^T has read the Q buffer
-  uint64_t* o_free = bars + 16;            // [1] per item: the epilogue has read O (4 warps)
+  // Tile g of a CTA's running count uses slot g & 1 of the K ring, the V ring, the S buffers and of
+  // every [2] barrier below, in phase (g >> 1) & 1.  A waiter is never two uses of a slot behind.
+  uint64_t* k_full = bars + 1;             // [2] K tile has landed
+  uint64_t* v_full = bars + 3;             // [2] V tile has landed
+  uint64_t* s_full = bars + 5;             // [2] Q K^T of the tile has completed: S is ready, the K slot is free
+  uint64_t* p_full = bars + 7;             // [2] P of the tile is in tensor memory (4 warps)
+  uint64_t* pv_done = bars + 9;            // [2] P V of the tile has completed: O is at rest, the V slot is free
+  uint64_t* q_empty = bars + 11;           // [1] per item: its last Q K^T has read the Q buffer
+  uint64_t* o_free = bars + 12;            // [1] per item: the epilogue has read O (4 warps)
+  char* o_stage = st_s + kAtStages * kAtStage + 256;
   __shared__ uint32_t sh_tmem;
   __shared__ int sh_abort;
   volatile int* abort_flag = &sh_abort;
@@ -104,14 +110,11 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     mbar_init(smem_u32(q_full), 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&k_full[i]), 1);
-      mbar_init(smem_u32(&k_empty[i]), 1);
       mbar_init(smem_u32(&v_full[i]), 1);
-      mbar_init(smem_u32(&v_empty[i]), 1);
       mbar_init(smem_u32(&s_full[i]), 1);
       mbar_init(smem_u32(&p_full[i]), 4);
+      mbar_init(smem_u32(&pv_done[i]), 1);
     }
-    mbar_init(smem_u32(pv_done), 1);
-    mbar_init(smem_u32(o_final), 1);
     mbar_init(smem_u32(q_empty), 1);
     mbar_init(smem_u32(o_free), 4);
     fence_mbar_init();
@@ -132,9 +135,10 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       int n_item = 0, gk = 0, gv = 0;                                  // items / K tiles / V tiles issued so far
       bool q_pending = false, ok = true;
       // tile g of this CTA's running count -> slot g & 1 of either ring
-      auto load_tile = [&](uint64_t* full, uint64_t* empty, const CUtensorMap* m, int g, int r, int off) {
+      // (`freed` completes when the MMAs that read the slot's previous tile have)
+      auto load_tile = [&](uint64_t* full, uint64_t* freed, const CUtensorMap* m, int g, int r, int off) {
         const int s = g & 1;
-        if (!mbar_wait(smem_u32(&empty[s]), ((g >> 1) & 1) ^ 1, abort_flag)) return false;
+        if (g >= 2 && !mbar_wait(smem_u32(&freed[s]), ((g >> 1) & 1) ^ 1, abort_flag)) return false;
         const uint32_t fb = smem_u32(&full[s]);
         mbar_expect_tx(fb, kAtTile);
         char* st = st_s + (size_t)s * kAtStage + off;
@@ -152,15 +156,15 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         q_pending = true;
         ++n_item;
         // same order as the MMA warp consumes them: K(0), then K(j+1) before V(j)
-        ok = load_tile(k_full, k_empty, mk, gk, I.row_base, 0);
+        ok = load_tile(k_full, s_full, mk, gk, I.row_base, 0);
         if (ok) ++gk;
         for (int j = 0; j < I.n_tiles && ok; ++j) {
           if (j + 1 < I.n_tiles) {
-            ok = load_tile(k_full, k_empty, mk, gk, I.row_base + (j + 1) * kAtBN, 0);
+            ok = load_tile(k_full, s_full, mk, gk, I.row_base + (j + 1) * kAtBN, 0);
             if (!ok) break;
             ++gk;
           }
-          ok = load_tile(v_full, v_empty, mv, gv, I.row_base + j * kAtBN, kAtTile);
+          ok = load_tile(v_full, pv_done, mv, gv, I.row_base + j * kAtBN, kAtTile);
           if (ok) ++gv;
         }
       }
@@ -198,7 +202,6 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
             mma_ss(d, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
                    kd + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
           mma_commit(smem_u32(&s_full[g & 1]));
-          mma_commit(smem_u32(&k_empty[s]));
           if (j == I.n_tiles - 1) mma_commit(smem_u32(q_empty));       // the Q buffer may be refilled
         };
         mbar_wait(smem_u32(q_full), n_item & 1, abort_flag);
@@ -215,9 +218,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
 #pragma unroll
           for (int ks = 0; ks < kAtBN / 16; ++ks)
             mma_ts(tmem + kAtColO, p_tmem + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), idesc_pv, (j | ks) != 0);
-          mma_commit(smem_u32(&v_empty[s]));
-          mma_commit(smem_u32(pv_done));
-          if (j == I.n_tiles - 1) mma_commit(smem_u32(o_final));
+          mma_commit(smem_u32(&pv_done[g & 1]));
         }
         g0 += I.n_tiles;
         ++n_item;
@@ -233,7 +234,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       AtItem I;
       if (!at_item(a, item, I)) continue;
       const int grow = I.q0 + row;                                     // row within the sequence
-      const int kv_end = min(I.n, I.q0 + kAtBM);
+      const int kv_end = I.q_hi;
       float m_used = -INFINITY, l_run = 0.f;
       for (int j = 0; j < I.n_tiles; ++j) {
         const int g = g0 + j, sb = g & 1;
@@ -265,9 +266,8 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         } else {
           const bool need = mx > m_used + kRescaleStep;
           if (__any_sync(0xffffffffu, need)) {
-            // O must be at rest: the P V of the previous tile.  (At this point that phase is either
-            // running or just completed, never further along, so the parity is unambiguous.)
-            mbar_wait(smem_u32(pv_done), (g - 1) & 1, abort_flag);
+            // O must be at rest: the P V of the previous tile
+            mbar_wait(smem_u32(&pv_done[(g - 1) & 1]), ((g - 1) >> 1) & 1, abort_flag);
             tc_fence_after();
             const float corr = need ? fast_exp2(m_used - mx) : 1.0f;
             if (need) m_used = mx;
@@ -299,8 +299,9 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         l_run += l0 + l1;
         tmem_st32(s_addr, pw);                                             // P overwrites its own S buffer
         tmem_st_wait();
-        if (j == I.n_tiles - 1 && kv_end < c0 + kAtBN) {
-          // ragged last tile: zero the V rows past the sequence's end (both 64-dim halves)
+        if (j == I.n_tiles - 1 && kv_end == I.n && kv_end < c0 + kAtBN) {
+          // ragged last tile of the sequence: zero the V rows past its end (both 64-dim halves); past
+          // the end of an inner query tile the rows are the sequence's own and P is 0 there
           const int s = g % kAtStages;
           mbar_wait(smem_u32(&v_full[s]), (g / kAtStages) & 1, abort_flag);
           char* vz = st_s + (size_t)s * kAtStage + kAtTile;
@@ -316,11 +317,15 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&p_full[sb]));
       }
-      // ---- epilogue: O / l -> bf16 -> out[b][row][h][:]
-      mbar_wait(smem_u32(o_final), n_item & 1, abort_flag);
+      // ---- epilogue: O / l -> bf16 -> out[b][row][h][:], 32 columns at a time through the warp's
+      // staging buffer (16-byte units XOR-swizzled by row pair: no bank conflicts either way)
+      const int gl = g0 + I.n_tiles - 1;
+      mbar_wait(smem_u32(&pv_done[gl & 1]), (gl >> 1) & 1, abort_flag);
       tc_fence_after();
       const float inv = 1.0f / l_run;
-      __nv_bfloat16* orow = a.out + (((size_t)I.b * a.n_max + grow) * a.H + I.h) * 128;
+      char* so = o_stage + (warp - 2) * 2048;
+      __nv_bfloat16* otile = a.out + (((size_t)I.b * a.n_max + I.q0 + quad * 32) * a.H + I.h) * 128;
+      const int rows_here = I.q_hi - (I.q0 + quad * 32);               // owned rows among this warp's 32
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
         uint32_t o[32];
@@ -331,19 +336,25 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(o_free));
         }
-        if (grow < I.n) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint4 w;
-            __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
-            __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
-            __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
-            w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
-            w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
-            *reinterpret_cast<uint4*>(orow + cc * 32 + i) = w;
-          }
+        for (int u = 0; u < 4; ++u) {
+          uint4 w;
+          __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[8 * u]) * inv, __uint_as_float(o[8 * u + 1]) * inv);
+          __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 2]) * inv, __uint_as_float(o[8 * u + 3]) * inv);
+          __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 4]) * inv, __uint_as_float(o[8 * u + 5]) * inv);
+          __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
+          w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
+          w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
+          *reinterpret_cast<uint4*>(so + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
         }
+        __syncwarp();
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+          const int r = it * 8 + (lane >> 2), u = lane & 3;
+          const uint4 w = *reinterpret_cast<const uint4*>(so + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
+          if (r < rows_here) *reinterpret_cast<uint4*>(otile + (size_t)r * a.H * 128 + cc * 32 + u * 8) = w;
+        }
+        __syncwarp();
       }
       g0 += I.n_tiles;
       ++n_item;
