@@ -54,6 +54,31 @@ __device__ __forceinline__ float fmax3(float x, float y, float z) {
   return r;
 }
 
+// two fp32 lanes in one 64-bit register: fused multiply-add and add on both at once
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t x, uint64_t y, uint64_t z) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(x), "l"(y), "l"(z));
+  return r;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t x, uint64_t y) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(x), "l"(y));
+  return r;
+}
+__device__ __forceinline__ uint64_t fmul2(uint64_t x, uint64_t y) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(x), "l"(y));
+  return r;
+}
+
 struct AtMaps { alignas(64) unsigned char q[128]; alignas(64) unsigned char k[128]; alignas(64) unsigned char v[128]; };
 
 struct AtArgs {
@@ -234,6 +259,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       AtItem I;
       if (!at_item(a, item, I)) continue;
       const int grow = I.q0 + row;                                     // row within the sequence
+      const int r0 = I.q0 + quad * 32;                                 // this warp's first row
       const int kv_end = I.q_hi;
       float m_used = -INFINITY, l_run = 0.f;
       for (int j = 0; j < I.n_tiles; ++j) {
@@ -241,62 +267,77 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         mbar_wait(smem_u32(&s_full[sb]), (g >> 1) & 1, abort_flag);
         tc_fence_after();
         const uint32_t s_addr = tmem + lane_off + kAtColS + (uint32_t)sb * kAtBN;
-        uint32_t sr[64];
-        tmem_ld32(s_addr, sr);
-        tmem_ld32(s_addr + 32, sr + 32);
-        tmem_ld_wait();
         const int c0 = j * kAtBN;
-        // raw scores stay unscaled: max commutes with the (positive) scale and the scale is folded into
-        // the exponent's FMA.  Only tiles that reach past the tile's first row need the causal mask.
-        if (c0 + kAtBN - 1 > I.q0) {
-#pragma unroll
-          for (int c = 0; c < 64; ++c)
-            if (c0 + c > grow) sr[c] = 0xFF800000u;                          // -inf
-        }
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};       // four independent chains
-#pragma unroll
-        for (int c = 0; c < 64; c += 8) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-            mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
-        }
-        float mx = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-        if (j == 0) {
-          m_used = mx;                        // column 0 is visible to every row, so mx is finite
-        } else {
-          const bool need = mx > m_used + kRescaleStep;
-          if (__any_sync(0xffffffffu, need)) {
-            // O must be at rest: the P V of the previous tile
-            mbar_wait(smem_u32(&pv_done[(g - 1) & 1]), ((g - 1) >> 1) & 1, abort_flag);
-            tc_fence_after();
-            const float corr = need ? fast_exp2(m_used - mx) : 1.0f;
-            if (need) m_used = mx;
-            l_run *= corr;
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-              uint32_t o[32];
-              tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
-              tmem_ld_wait();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
-              tmem_st32(tmem + lane_off + kAtColO + cc * 32, o);
-            }
-            tmem_st_wait();
-          }
-        }
         uint32_t pw[32];
-        const float neg_m = -m_used;
-        float l0 = 0.f, l1 = 0.f;
+        if (c0 > r0 + 31) {
+          // no row of this warp sees a key of this tile: P = 0, nothing else to do
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c]), a.scale_log2, neg_m));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), a.scale_log2, neg_m));
-          l0 += p0;
-          l1 += p1;
-          __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-          pw[c] = *reinterpret_cast<uint32_t*>(&pk);
+          for (int c = 0; c < 32; ++c) pw[c] = 0u;
+        } else {
+          uint32_t sr[64];
+          tmem_ld32(s_addr, sr);
+          tmem_ld32(s_addr + 32, sr + 32);
+          tmem_ld_wait();
+          // raw scores stay unscaled: max commutes with the (positive) scale and the scale is folded into
+          // the exponent's FMA.  Only a tile that reaches past the warp's first row needs the causal mask.
+          if (c0 + kAtBN - 1 > r0) {
+#pragma unroll
+            for (int c = 0; c < 64; ++c)
+              if (c0 + c > grow) sr[c] = 0xFF800000u;                        // -inf
+          }
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four independent chains
+#pragma unroll
+          for (int c = 0; c < 64; c += 8) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
+          }
+          float mx = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
+          if (j == 0) {
+            m_used = mx;                      // column 0 is visible to every row, so mx is finite
+          } else {
+            const bool need = mx > m_used + kRescaleStep;
+            if (__any_sync(0xffffffffu, need)) {
+              // O must be at rest: the P V of the previous tile
+              mbar_wait(smem_u32(&pv_done[(g - 1) & 1]), ((g - 1) >> 1) & 1, abort_flag);
+              tc_fence_after();
+              const float corr = need ? fast_exp2(m_used - mx) : 1.0f;
+              if (need) m_used = mx;
+              l_run *= corr;
+              const uint64_t corr2 = pack2(corr, corr);
+#pragma unroll
+              for (int cc = 0; cc < 4; ++cc) {
+                uint32_t o[32];
+                tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                  float x, y;
+                  unpack2(fmul2(pack2(__uint_as_float(o[i]), __uint_as_float(o[i + 1])), corr2), x, y);
+                  o[i] = __float_as_uint(x);
+                  o[i + 1] = __float_as_uint(y);
+                }
+                tmem_st32(tmem + lane_off + kAtColO + cc * 32, o);
+              }
+              tmem_st_wait();
+            }
+          }
+          const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nm2 = pack2(-m_used, -m_used);
+          uint64_t l2[2] = {0ull, 0ull};                                    // two chains of packed row sums
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            float p0, p1;
+            unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
+            p0 = fast_exp2(p0);
+            p1 = fast_exp2(p1);
+            l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
+            __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+            pw[c] = *reinterpret_cast<uint32_t*>(&pk);
+          }
+          float la, lb;
+          unpack2(fadd2(l2[0], l2[1]), la, lb);
+          l_run += la + lb;
         }
-        l_run += l0 + l1;
         tmem_st32(s_addr, pw);                                             // P overwrites its own S buffer
         tmem_st_wait();
         if (j == I.n_tiles - 1 && kv_end == I.n && kv_end < c0 + kAtBN) {
