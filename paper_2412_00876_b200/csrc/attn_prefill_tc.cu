@@ -1,29 +1,38 @@
 // Prefill attention over the reduced set on the tensor cores (Eq. 1 applied to S^{P*}):
 // row i of a sequence's compact context attends rows 0..i of the same context.
-// bf16, head_dim 128.  Persistent CTAs, two per SM (one CTA's softmax overlaps the other's MMAs),
-// walk work items (sequence, head, 128-row query tile), longest tiles first; tensor memory, barriers
-// and the pipelines live across items, so an item's loads start while the previous one finishes.
-// Query tiles are aligned to the END of a sequence (rows [n-128(t+1), n-128t)), so the ragged tile is
-// the one at the top of the causal triangle, where it needs the fewest key tiles.
-//   warp 0    : TMA producer.  Q of an item (two 64-dim halves) as soon as the previous item's last
-//               Q K^T has read the Q buffer; 64-row K tiles and V tiles through two separate 2-slot
-//               rings (a K slot is free once its Q K^T has run, long before the V slot of the same
-//               tile, so the next K is in flight a whole softmax earlier), all with the 128-byte swizzle;
-//   warp 1    : tensor-memory allocation and the single MMA-issuing thread:
-//               S = Q K^T (128 x 64, K-major operands from shared memory) into one of two S buffers,
-//               O += P V (P read from tensor memory, V as an MN-major shared-memory operand);
-//               the next tile's Q K^T is issued before this tile's P V so it runs during the softmax;
-//   warps 2-5 : softmax, one query row per thread, straight out of tensor memory.  The running
-//               maximum is only raised when it grows by more than 2^8 (then O is rescaled in tensor
-//               memory), so most tiles never touch O.  P (bf16) overwrites the first half of its
-//               own S buffer.  The same warps normalise O and store the output rows, staged
-//               through a small per-warp buffer so that each store instruction writes whole
-//               64-byte row segments.
-// Tensor memory: O 128 columns, S0 and S1 64 columns each (256 columns per CTA, 512 per SM).
-// Barrier phases are driven by running counters (tiles, K/V stages, items) that every role advances
-// identically.  Rows past a sequence's length are fetched with the tile (they are masked); in the
-// last tile the surplus V rows are zeroed in shared memory first, since 0 * x must stay 0 for any
-// bit pattern.  Every wait is bounded (pipeline.cuh); an abort leaves DL_ERR_TIMEOUT in the status word.
+// bf16, head_dim 128.  One persistent CTA per SM walks work items (sequence, head, PAIR of 128-row
+// query tiles), longest first.  The two query tiles of a pair run as two lanes, A (the later rows)
+// and B (the 128 rows before them): each lane has its own Q buffers, its own score / output
+// accumulators in tensor memory, its own MMA-issuing thread and its own four softmax warps, and both
+// read the same K and V tiles, which are fetched once per pair into a ring shared by the lanes.
+// While one lane's softmax warps work on a score tile the tensor pipe runs the other lane's MMAs.
+// Pairs are aligned to the END of a sequence (rows [n-256(p+1), n-256p)), so the ragged pair is the
+// one at the top of the causal triangle, where it needs the fewest keys; lane B of a pair that has
+// 128 rows or fewer does not exist and the lane moves on to the next item on its own.
+//   warp 8     : TMA producer (one lane), a polling loop over three cursors: the K/V ring (tiles of
+//                128 keys, K and V alternating, three slots of 32 KB) and the Q loads of either lane
+//                (two slots per lane, so an item's Q is in flight while the previous item computes).
+//   warps 9,10 : the MMA-issuing thread of lane A / lane B:
+//                S = Q K^T (128 x N, K-major operands from shared memory), O += P V (P read from
+//                tensor memory, V as an MN-major shared-memory operand), then the next tile's Q K^T.
+//                Full tiles use N = 128 keys; a lane's last tile uses N = keys left rounded up to 16,
+//                in both products, so the tensor pipe does not multiply by padding.
+//   warps 0-3 / 4-7 : softmax of lane A / B, one query row per thread, straight out of tensor memory
+//                in two passes (row maximum, then exponentials).  32-column chunks that no row of the
+//                warp may see (above the causal diagonal) are skipped.  The running maximum is only
+//                raised when it grows by more than 2^8 (then O is rescaled in tensor memory), so most
+//                tiles never touch O.  P (bf16) overwrites the first half of S.  The same warps
+//                normalise O and write the output: 32 x 32 blocks staged in the item's own Q buffer
+//                (free once its last Q K^T has run) and sent with TMA stores; a clipped tile at the
+//                top of a sequence, whose surplus rows belong to the next tile, is written with
+//                predicated stores instead.  The Q slot returns to the producer once those stores
+//                have read it.
+//   warp 11    : tensor-memory allocation (all 512 columns: O_A | S_A | O_B | S_B).
+// Barrier phases are driven by running counters (ring tiles, a lane's tiles, a lane's items) that every
+// role advances identically.  Rows past a sequence's length are fetched with the tile (they are
+// masked); where the 16-row rounding of the last tile reaches past the sequence's end, those V rows
+// are zeroed in shared memory first, since 0 * x must stay 0 for any bit pattern.  Every wait is
+// bounded (pipeline.cuh); an abort leaves DL_ERR_TIMEOUT in the status word.
 #include <algorithm>
 
 #include "common.cuh"
@@ -31,13 +40,12 @@
 
 namespace dl {
 
-constexpr int kAtBM = 128, kAtBN = 64, kAtStages = 2, kAtThreads = 192;
-constexpr int kAtQBytes = 2 * kAtBM * 128;            // 32 KB: two [128 rows][64 dims] halves
-constexpr int kAtTile = 2 * kAtBN * 128;              // 16 KB: two [64 rows][64 dims] halves
-constexpr int kAtStage = 2 * kAtTile;                 // K tile + V tile
-constexpr int kAtOutStage = 4 * 2048;                 // per softmax warp: 32 rows x 32 columns of bf16 output
-constexpr size_t kAtSmem = kAtQBytes + kAtStages * kAtStage + kAtOutStage + 1024 + 256;
-constexpr uint32_t kAtColO = 0, kAtColS = 128;        // tensor-memory columns: O | S0 | S1
+constexpr int kAtBM = 128, kAtBN = 128, kAtThreads = 384, kAtRing = 3;
+constexpr int kAtTile = 2 * 128 * 128;                // 32 KB: two [128 rows][64 dims] halves
+constexpr int kAtOffRing = 4 * kAtTile;               // Q: [lane][slot] tiles first
+constexpr int kAtOffBar = kAtOffRing + kAtRing * kAtTile;
+constexpr size_t kAtSmem = kAtOffBar + 512;           // 229888 bytes: one CTA per SM
+constexpr uint32_t kAtColO = 0, kAtColS = 128, kAtLaneCols = 256;   // tensor-memory columns of one lane: O | S
 constexpr float kRescaleStep = 8.0f;                  // log2 units by which the maximum may lag
 
 // 2^x on the special-function unit (x <= 0 here; -inf gives 0)
@@ -79,304 +87,447 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t x, uint64_t y) {
   return r;
 }
 
-struct AtMaps { alignas(64) unsigned char q[128]; alignas(64) unsigned char k[128]; alignas(64) unsigned char v[128]; };
+struct AtMaps {
+  alignas(64) unsigned char q[128]; alignas(64) unsigned char k[128];
+  alignas(64) unsigned char v[128]; alignas(64) unsigned char o[128];
+};
 
 struct AtArgs {
   const int32_t* cache_len; __nv_bfloat16* out; DeviceStatus* status;
-  int32_t B, H, cap, n_max, q_tiles;
+  int32_t B, H, cap, n_max, q_pairs;
   float scale_log2;
 };
 
-// Work item -> (b, h, query tile).  Tile t counts from the sequence's end (the longest first): it owns
-// rows [q_hi - 128, q_hi) with q_hi = n - 128 t; the tile at the top is clipped to start at row 0 (it
-// loads rows [0, 128) and owns the first q_hi of them).  Returns false for a tile the sequence lacks.
-struct AtItem { int b, h, q0, q_hi, n, n_tiles, row_base; };
-__device__ __forceinline__ bool at_item(const AtArgs& a, int item, AtItem& I) {
-  const int bh_count = a.B * a.H;
-  const int t = item / bh_count;
-  const int bh = item - t * bh_count;
-  I.b = bh / a.H;
-  I.h = bh - I.b * a.H;
-  I.n = min(max(a.cache_len[I.b], 0), min(a.cap, a.n_max));
-  I.q_hi = I.n - t * kAtBM;
-  if (I.q_hi <= 0) return false;
-  I.q0 = max(I.q_hi - kAtBM, 0);
-  I.n_tiles = (I.q_hi + kAtBN - 1) / kAtBN;                       // keys any owned row may see: [0, q_hi)
-  I.row_base = bh * a.cap;                                        // first row of this (b, h) in the caches
-  return true;
+// Work item -> (b, h, pair p of query tiles).  Pair p counts from the sequence's end: it covers rows
+// [q_hi - 256, q_hi) with q_hi = n - 256 p, clipped at row 0; its keys are [0, q_hi) in n_kv tiles.
+struct AtItem { int b, h, q_hi, n, n_kv, row_base; };
+
+// One lane's share of an item: rows [q0, q_hi) are owned (the Q tile is loaded from row q0, 128 rows;
+// a tile clipped at the top of the sequence loads rows [0, 128) and owns the first q_hi of them),
+// keys [0, q_hi) in n_tiles tiles.
+struct AtLane { int q0, q_hi, n_tiles; bool exists; };
+__device__ __forceinline__ AtLane at_lane(const AtItem& I, int lane_id) {
+  AtLane L;
+  L.q_hi = I.q_hi - lane_id * kAtBM;
+  L.exists = L.q_hi > 0;
+  L.q0 = max(L.q_hi - kAtBM, 0);
+  L.n_tiles = (L.q_hi + kAtBN - 1) / kAtBN;
+  return L;
+}
+// keys of tile j that a lane's MMAs cover: all 128, or what is left of [0, q_hi) rounded up to 16
+__device__ __forceinline__ int at_cols(const AtLane& L, int j) {
+  return min(kAtBN, (L.q_hi - j * kAtBN + 15) & ~15);
 }
 
-__global__ void __launch_bounds__(kAtThreads, 2)
+// Walks the items of this CTA in the order every role uses; the length of the NEXT item's sequence is
+// requested one item early, so its latency never sits in front of a role's first wait.
+struct AtWalker {
+  const AtArgs& a;
+  int item, items, bh_count, len_nx;
+  __device__ __forceinline__ int len_of(int it) const { return __ldg(a.cache_len + (it % bh_count) / a.H); }
+  __device__ __forceinline__ explicit AtWalker(const AtArgs& a_) : a(a_) {
+    bh_count = a.B * a.H;
+    items = bh_count * a.q_pairs;
+    item = (int)blockIdx.x - (int)gridDim.x;
+    len_nx = (int)blockIdx.x < items ? len_of(blockIdx.x) : 0;
+  }
+  // Advances to the next item that exists (a sequence of 256 p rows or fewer has no pair p).
+  __device__ __forceinline__ bool next(AtItem& I) {
+    for (;;) {
+      item += (int)gridDim.x;
+      if (item >= items) return false;
+      const int len = len_nx;
+      const int nx = item + (int)gridDim.x;
+      if (nx < items) len_nx = len_of(nx);
+      const int p = item / bh_count;
+      const int bh = item - p * bh_count;
+      I.b = bh / a.H;
+      I.h = bh - I.b * a.H;
+      I.n = min(max(len, 0), min(a.cap, a.n_max));
+      I.q_hi = I.n - p * 2 * kAtBM;
+      if (I.q_hi <= 0) continue;
+      I.n_kv = (I.q_hi + kAtBN - 1) / kAtBN;
+      I.row_base = bh * a.cap;                                      // first row of this (b, h) in the caches
+      return true;
+    }
+  }
+};
+
+__global__ void __launch_bounds__(kAtThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
-  extern __shared__ char smem_raw[];
-  char* smem = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  char* q_s = smem;
-  char* st_s = smem + kAtQBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(st_s + kAtStages * kAtStage);
-  uint64_t* q_full = bars;                 // [1] per item: Q has landed
-  // Tile g of a CTA's running count uses slot g & 1 of the K ring, the V ring, the S buffers and of
-  // every [2] barrier below, in phase (g >> 1) & 1.  A waiter is never two uses of a slot behind.
-  uint64_t* k_full = bars + 1;             // [2] K tile has landed
-  uint64_t* v_full = bars + 3;             // [2] V tile has landed
-  uint64_t* s_full = bars + 5;             // [2] Q K^T of the tile has completed: S is ready, the K slot is free
-  uint64_t* p_full = bars + 7;             // [2] P of the tile is in tensor memory (4 warps)
-  uint64_t* pv_done = bars + 9;            // [2] P V of the tile has completed: O is at rest, the V slot is free
-  uint64_t* q_empty = bars + 11;           // [1] per item: its last Q K^T has read the Q buffer
-  uint64_t* o_free = bars + 12;            // [1] per item: the epilogue has read O (4 warps)
-  char* o_stage = st_s + kAtStages * kAtStage + 256;
-  __shared__ uint32_t sh_tmem;
-  __shared__ int sh_abort;
-  volatile int* abort_flag = &sh_abort;
+  extern __shared__ __align__(1024) char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int items = a.B * a.H * a.q_tiles;
+  if (smem_u32(smem) & 1023u) {                        // the swizzled tiles need 1024-byte alignment
+    if (tid == 0) report_status(a.status, DL_ERR_ALIGNMENT, -1);
+    return;
+  }
+  char* ring_s = smem + kAtOffRing;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kAtOffBar);
+  // Ring tile T of this CTA (running count over its items; K and V of key tile j of an item are tiles
+  // base + 2j and base + 2j + 1) lives in slot T % 3 and completes phase (T / 3) & 1 of that slot's
+  // `full` barrier; lane X's MMAs that read it complete a phase of the slot's `free_X` barrier.
+  // A lane's own barriers: its k-th tile completes phase k & 1 of s_full / p_full / pv_done; its i-th
+  // item completes phase i & 1 of o_free and phase (i >> 1) & 1 of q_full / q_done of Q slot i & 1.
+  auto ring_full = [&](int s) { return smem_u32(bars + s); };
+  auto ring_free = [&](int x, int s) { return smem_u32(bars + 3 + 3 * x + s); };
+  auto q_full = [&](int x, int s) { return smem_u32(bars + 9 + 2 * x + s); };    // Q tile has landed
+  auto q_done = [&](int x, int s) { return smem_u32(bars + 13 + 2 * x + s); };   // Q slot may be refilled (4 warps)
+  auto s_full = [&](int x) { return smem_u32(bars + 17 + x); };   // Q K^T has completed: S ready
+  auto p_full = [&](int x) { return smem_u32(bars + 19 + x); };   // P is in tensor memory (4 warps)
+  auto pv_done = [&](int x) { return smem_u32(bars + 21 + x); };  // P V has completed: O at rest
+  auto o_free = [&](int x) { return smem_u32(bars + 23 + x); };   // the epilogue has read O (4 warps)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
 
   if (tid == 0) {
-    sh_abort = 0;
-    mbar_init(smem_u32(q_full), 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&k_full[i]), 1);
-      mbar_init(smem_u32(&v_full[i]), 1);
-      mbar_init(smem_u32(&s_full[i]), 1);
-      mbar_init(smem_u32(&p_full[i]), 4);
-      mbar_init(smem_u32(&pv_done[i]), 1);
+    *abort_flag = 0;
+    for (int s = 0; s < kAtRing; ++s) {
+      mbar_init(ring_full(s), 1);
+      mbar_init(ring_free(0, s), 1);
+      mbar_init(ring_free(1, s), 1);
     }
-    mbar_init(smem_u32(q_empty), 1);
-    mbar_init(smem_u32(o_free), 4);
+    for (int x = 0; x < 2; ++x) {
+      for (int s = 0; s < 2; ++s) { mbar_init(q_full(x, s), 1); mbar_init(q_done(x, s), 4); }
+      mbar_init(s_full(x), 1);
+      mbar_init(p_full(x), 4);
+      mbar_init(pv_done(x), 1);
+      mbar_init(o_free(x), 4);
+    }
     fence_mbar_init();
   }
-  if (warp == 1) { tmem_alloc(smem_u32(&sh_tmem), 256); tmem_relinquish(); }
+  if (warp == 11) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = sh_tmem;
+  const uint32_t tmem = *tmem_slot;
 
-  if (warp == 0) {
+  if (warp == 8) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(maps.q);
       const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(maps.k);
       const CUtensorMap* mv = reinterpret_cast<const CUtensorMap*>(maps.v);
       tma_prefetch_desc(mq); tma_prefetch_desc(mk); tma_prefetch_desc(mv);
-      int n_item = 0, gk = 0, gv = 0;                                  // items / K tiles / V tiles issued so far
-      bool q_pending = false, ok = true;
-      // tile g of this CTA's running count -> slot g & 1 of either ring
-      // (`freed` completes when the MMAs that read the slot's previous tile have)
-      auto load_tile = [&](uint64_t* full, uint64_t* freed, const CUtensorMap* m, int g, int r, int off) {
-        const int s = g & 1;
-        if (g >= 2 && !mbar_wait(smem_u32(&freed[s]), ((g >> 1) & 1) ^ 1, abort_flag)) return false;
-        const uint32_t fb = smem_u32(&full[s]);
-        mbar_expect_tx(fb, kAtTile);
-        char* st = st_s + (size_t)s * kAtStage + off;
-        tma_load_2d(smem_u32(st), m, 0, r, fb);
-        tma_load_2d(smem_u32(st + kAtBN * 128), m, 64, r, fb);
-        return true;
-      };
-      for (int item = blockIdx.x; item < items && ok && !*abort_flag; item += gridDim.x) {
-        AtItem I;
-        if (!at_item(a, item, I)) continue;
-        if (!mbar_wait(smem_u32(q_empty), (n_item & 1) ^ 1, abort_flag)) break;
-        mbar_expect_tx(smem_u32(q_full), kAtQBytes);
-        tma_load_2d(smem_u32(q_s), mq, 0, I.row_base + I.q0, smem_u32(q_full));
-        tma_load_2d(smem_u32(q_s + kAtBM * 128), mq, 64, I.row_base + I.q0, smem_u32(q_full));
-        q_pending = true;
-        ++n_item;
-        // same order as the MMA warp consumes them: K(0), then K(j+1) before V(j)
-        ok = load_tile(k_full, s_full, mk, gk, I.row_base, 0);
-        if (ok) ++gk;
-        for (int j = 0; j < I.n_tiles && ok; ++j) {
-          if (j + 1 < I.n_tiles) {
-            ok = load_tile(k_full, s_full, mk, gk, I.row_base + (j + 1) * kAtBN, 0);
-            if (!ok) break;
-            ++gk;
+      // cursor of the ring
+      AtWalker Wr(a);
+      AtItem Ir;
+      bool hr = Wr.next(Ir);
+      int T = 0, jr = 0;                       // ring tiles issued so far / tile index within Ir (K, V alternating)
+      uint32_t free_par[2] = {0u, 0u};         // bit s: parity of the next phase of ring_free(x, s) to wait for
+      uint32_t prev_b = 0u;                    // bit s: the tile now in slot s is read by lane B too
+      // cursors of the Q loads
+      AtWalker Wq0(a), Wq1(a);
+      AtItem Iq[2];
+      bool hq[2];
+      int nq[2] = {0, 0};                      // Q loads issued so far per lane
+      hq[0] = Wq0.next(Iq[0]);
+      hq[1] = Wq1.next(Iq[1]);
+      while (hq[1] && !at_lane(Iq[1], 1).exists) hq[1] = Wq1.next(Iq[1]);
+      int idle = 0;
+      while ((hr || hq[0] || hq[1]) && !*abort_flag) {
+        bool prog = false;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          if (!hq[x]) continue;
+          const int s = nq[x] & 1;
+          // the slot's previous item (two items back) must have finished its epilogue
+          if (nq[x] >= 2 && !mbar_test(q_done(x, s), ((nq[x] - 2) >> 1) & 1)) continue;
+          const AtLane L = at_lane(Iq[x], x);
+          char* dst = smem + (2 * x + s) * kAtTile;
+          mbar_expect_tx(q_full(x, s), kAtTile);
+          tma_load_2d(smem_u32(dst), mq, 0, Iq[x].row_base + L.q0, q_full(x, s));
+          tma_load_2d(smem_u32(dst + kAtBM * 128), mq, 64, Iq[x].row_base + L.q0, q_full(x, s));
+          ++nq[x];
+          if (x == 0) {
+            hq[0] = Wq0.next(Iq[0]);
+          } else {
+            hq[1] = Wq1.next(Iq[1]);
+            while (hq[1] && !at_lane(Iq[1], 1).exists) hq[1] = Wq1.next(Iq[1]);
           }
-          ok = load_tile(v_full, pv_done, mv, gv, I.row_base + j * kAtBN, kAtTile);
-          if (ok) ++gv;
+          prog = true;
+        }
+        if (hr) {
+          const int s = T % kAtRing;
+          bool slot_free = true;
+          if (T >= kAtRing) {
+            slot_free = mbar_test(ring_free(0, s), (free_par[0] >> s) & 1u);
+            if (slot_free && ((prev_b >> s) & 1u)) slot_free = mbar_test(ring_free(1, s), (free_par[1] >> s) & 1u);
+          }
+          if (slot_free) {
+            if (T >= kAtRing) {
+              free_par[0] ^= 1u << s;
+              if ((prev_b >> s) & 1u) free_par[1] ^= 1u << s;
+            }
+            const int j = jr >> 1;
+            const AtLane LB = at_lane(Ir, 1);
+            const bool b_reads = LB.exists && j < LB.n_tiles;
+            prev_b = (prev_b & ~(1u << s)) | ((b_reads ? 1u : 0u) << s);
+            char* dst = ring_s + s * kAtTile;
+            const CUtensorMap* m = (jr & 1) ? mv : mk;
+            const int r = Ir.row_base + j * kAtBN;
+            mbar_expect_tx(ring_full(s), kAtTile);
+            tma_load_2d(smem_u32(dst), m, 0, r, ring_full(s));
+            tma_load_2d(smem_u32(dst + kAtBN * 128), m, 64, r, ring_full(s));
+            ++T;
+            if (++jr == 2 * Ir.n_kv) { jr = 0; hr = Wr.next(Ir); }
+            prog = true;
+          }
+        }
+        if (prog) {
+          idle = 0;
+        } else if (++idle > kSpinLimitBusy) {
+          *abort_flag = 1;
         }
       }
       if (*abort_flag) {
         // every copy that was issued must land before the CTA's shared memory is released
         report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
-        if (q_pending)
-          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(q_full), (n_item - 1) & 1); ++i) __nanosleep(40);
-        for (int j = max(0, gk - 2); j < gk; ++j)
-          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&k_full[j & 1]), (j >> 1) & 1); ++i) __nanosleep(40);
-        for (int j = max(0, gv - 2); j < gv; ++j)
-          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&v_full[j & 1]), (j >> 1) & 1); ++i) __nanosleep(40);
+        for (int t = max(0, T - kAtRing); t < T; ++t)
+          for (int i = 0; i < kSpinLimit && !mbar_try_wait(ring_full(t % kAtRing), (t / kAtRing) & 1); ++i) __nanosleep(40);
+        for (int x = 0; x < 2; ++x)
+          for (int t = max(0, nq[x] - 2); t < nq[x]; ++t)
+            for (int i = 0; i < kSpinLimit && !mbar_try_wait(q_full(x, t & 1), (t >> 1) & 1); ++i) __nanosleep(40);
       }
     }
-  } else if (warp == 1) {
-    // ---------------------------------------------------------------- MMA issuer
+  } else if (warp == 9 || warp == 10) {
+    // ---------------------------------------------------------------- MMA issuer of one lane
     if (lane == 0) {
-      const uint32_t idesc_qk = idesc_bf16(kAtBM, kAtBN);
-      const uint32_t idesc_pv = idesc_bf16(kAtBM, 128, 0, 1);        // B (= V) is MN-major
-      const uint64_t q_desc = smem_desc_sw128(smem_u32(q_s));
-      const uint64_t k_desc0 = smem_desc_sw128(smem_u32(st_s));
-      const uint64_t v_desc0 = smem_desc_sw128_mn(smem_u32(st_s) + kAtTile, kAtBN * 128);
-      int n_item = 0, g0 = 0;                                          // items / tiles before this item
-      for (int item = blockIdx.x; item < items; item += gridDim.x) {
-        AtItem I;
-        if (!at_item(a, item, I)) continue;
+      const int x = warp - 9;
+      const uint32_t t_o = tmem + x * kAtLaneCols + kAtColO, t_s = tmem + x * kAtLaneCols + kAtColS;
+      const uint32_t idesc_pv = idesc_bf16(kAtBM, 128, 0, 1);          // B (= V) is MN-major
+      AtWalker W(a);
+      AtItem I;
+      int n_item = 0, g0 = 0, T0 = 0;                 // this lane's items / tiles so far; ring tiles before this item
+      while (W.next(I)) {
+        const AtLane L = at_lane(I, x);
+        if (!L.exists) { T0 += 2 * I.n_kv; continue; }
+        const int qs = n_item & 1;
+        const uint64_t q_desc = smem_desc_sw128(smem_u32(smem + (2 * x + qs) * kAtTile));
         auto issue_qk = [&](int j) {
-          const int g = g0 + j, s = g % kAtStages;
-          mbar_wait(smem_u32(&k_full[s]), (g / kAtStages) & 1, abort_flag);
+          const int T = T0 + 2 * j, s = T % kAtRing;
+          mbar_wait_spin(ring_full(s), (T / kAtRing) & 1, abort_flag);
           tc_fence_after();
-          const uint64_t kd = k_desc0 + (uint64_t)((s * kAtStage) >> 4);
-          const uint32_t d = tmem + kAtColS + (uint32_t)(g & 1) * kAtBN;
+          const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile));
+          const uint32_t idesc_qk = idesc_bf16(kAtBM, (uint32_t)at_cols(L, j));
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
-            mma_ss(d, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
-                   kd + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
-          mma_commit(smem_u32(&s_full[g & 1]));
-          if (j == I.n_tiles - 1) mma_commit(smem_u32(q_empty));       // the Q buffer may be refilled
+            mma_ss(t_s, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
+                   k_desc + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
+          mma_commit(s_full(x));
+          mma_commit(ring_free(x, s));
         };
-        mbar_wait(smem_u32(q_full), n_item & 1, abort_flag);
+        mbar_wait_spin(q_full(x, qs), (n_item >> 1) & 1, abort_flag);
         issue_qk(0);
-        for (int j = 0; j < I.n_tiles; ++j) {
-          if (j + 1 < I.n_tiles) issue_qk(j + 1);
-          const int g = g0 + j, s = g % kAtStages;
-          mbar_wait(smem_u32(&p_full[g & 1]), (g >> 1) & 1, abort_flag);
-          if (j == 0) mbar_wait(smem_u32(o_free), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
-          mbar_wait(smem_u32(&v_full[s]), (g / kAtStages) & 1, abort_flag);
+        for (int j = 0; j < L.n_tiles; ++j) {
+          const int g = g0 + j;
+          const int T = T0 + 2 * j + 1, s = T % kAtRing;
+          mbar_wait_spin(p_full(x), g & 1, abort_flag);
+          if (j == 0) mbar_wait_spin(o_free(x), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
+          mbar_wait_spin(ring_full(s), (T / kAtRing) & 1, abort_flag);
           tc_fence_after();
-          const uint64_t vd = v_desc0 + (uint64_t)((s * kAtStage) >> 4);
-          const uint32_t p_tmem = tmem + kAtColS + (uint32_t)(g & 1) * kAtBN;
-#pragma unroll
-          for (int ks = 0; ks < kAtBN / 16; ++ks)
-            mma_ts(tmem + kAtColO, p_tmem + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), idesc_pv, (j | ks) != 0);
-          mma_commit(smem_u32(&pv_done[g & 1]));
+          const uint64_t v_desc = smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128);
+          const int ksteps = at_cols(L, j) >> 4;
+          for (int ks = 0; ks < ksteps; ++ks)
+            mma_ts(t_o, t_s + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv, (j | ks) != 0);
+          mma_commit(pv_done(x));
+          mma_commit(ring_free(x, s));
+          if (j + 1 < L.n_tiles) issue_qk(j + 1);                      // overwrites P: in order behind the P V
         }
-        g0 += I.n_tiles;
+        g0 += L.n_tiles;
         ++n_item;
+        T0 += 2 * I.n_kv;
       }
     }
-  } else {
-    // ---------------------------------------------------------------- softmax / epilogue warps
+  } else if (warp < 8) {
+    // ---------------------------------------------------------------- softmax / epilogue warps of one lane
+    const int x = warp >> 2;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                                  // row within the query tile
     const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
-    int n_item = 0, g0 = 0;
-    for (int item = blockIdx.x; item < items; item += gridDim.x) {
-      AtItem I;
-      if (!at_item(a, item, I)) continue;
-      const int grow = I.q0 + row;                                     // row within the sequence
-      const int r0 = I.q0 + quad * 32;                                 // this warp's first row
-      const int kv_end = I.q_hi;
+    const uint32_t s_addr = tmem + lane_off + x * kAtLaneCols + kAtColS;
+    const uint32_t o_addr = tmem + lane_off + x * kAtLaneCols + kAtColO;
+    const CUtensorMap* mo = reinterpret_cast<const CUtensorMap*>(maps.o);
+    AtWalker W(a);
+    AtItem I;
+    int n_item = 0, g0 = 0, T0 = 0;
+    int q_slot_held = -1;                                              // Q slot whose staged stores are still in flight
+    while (W.next(I)) {
+      const AtLane L = at_lane(I, x);
+      if (!L.exists) { T0 += 2 * I.n_kv; continue; }
+      const int grow = L.q0 + row;                                     // row within the sequence
+      const int r0 = L.q0 + quad * 32;                                 // this warp's first row
       float m_used = -INFINITY, l_run = 0.f;
-      for (int j = 0; j < I.n_tiles; ++j) {
-        const int g = g0 + j, sb = g & 1;
-        mbar_wait(smem_u32(&s_full[sb]), (g >> 1) & 1, abort_flag);
-        tc_fence_after();
-        const uint32_t s_addr = tmem + lane_off + kAtColS + (uint32_t)sb * kAtBN;
+      for (int j = 0; j < L.n_tiles; ++j) {
+        const int g = g0 + j;
         const int c0 = j * kAtBN;
-        uint32_t pw[32];
-        if (c0 > r0 + 31) {
-          // no row of this warp sees a key of this tile: P = 0, nothing else to do
+        // 32-column chunks of this tile that some row of the warp may see
+        const int n_ch = min(4, (min(L.q_hi, r0 + 32) - c0 + 31) >> 5);
+        mbar_wait_spin(s_full(x), g & 1, abort_flag);
+        tc_fence_after();
+        // ---- pass 1: row maximum of the raw scores (max commutes with the positive scale)
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
 #pragma unroll
-          for (int c = 0; c < 32; ++c) pw[c] = 0u;
-        } else {
-          uint32_t sr[64];
-          tmem_ld32(s_addr, sr);
-          tmem_ld32(s_addr + 32, sr + 32);
-          tmem_ld_wait();
-          // raw scores stay unscaled: max commutes with the (positive) scale and the scale is folded into
-          // the exponent's FMA.  Only a tile that reaches past the warp's first row needs the causal mask.
-          if (c0 + kAtBN - 1 > r0) {
+        for (int hf = 0; hf < 2; ++hf) {
+          if (n_ch > 2 * hf) {
+            uint32_t sr[64];
+            tmem_ld32(s_addr + 64 * hf, sr);
+            if (n_ch > 2 * hf + 1) tmem_ld32(s_addr + 64 * hf + 32, sr + 32);
+            tmem_ld_wait();
+            const int lim = n_ch > 2 * hf + 1 ? 64 : 32;
+            const int vis = grow - (c0 + 64 * hf);                     // columns 0..vis of this half are visible
+            if (c0 + 64 * hf + lim - 1 > r0) {
 #pragma unroll
-            for (int c = 0; c < 64; ++c)
-              if (c0 + c > grow) sr[c] = 0xFF800000u;                        // -inf
-          }
-          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four independent chains
+              for (int c = 0; c < 64; ++c)
+                if (c > vis) sr[c] = 0xFF800000u;                      // -inf
+            }
 #pragma unroll
-          for (int c = 0; c < 64; c += 8) {
+            for (int c = 0; c < 32; c += 8) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-              mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
-          }
-          float mx = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-          if (j == 0) {
-            m_used = mx;                      // column 0 is visible to every row, so mx is finite
-          } else {
-            const bool need = mx > m_used + kRescaleStep;
-            if (__any_sync(0xffffffffu, need)) {
-              // O must be at rest: the P V of the previous tile
-              mbar_wait(smem_u32(&pv_done[(g - 1) & 1]), ((g - 1) >> 1) & 1, abort_flag);
-              tc_fence_after();
-              const float corr = need ? fast_exp2(m_used - mx) : 1.0f;
-              if (need) m_used = mx;
-              l_run *= corr;
-              const uint64_t corr2 = pack2(corr, corr);
+              for (int u = 0; u < 4; ++u)
+                mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
+            }
+            if (lim == 64) {
 #pragma unroll
-              for (int cc = 0; cc < 4; ++cc) {
-                uint32_t o[32];
-                tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
-                tmem_ld_wait();
+              for (int c = 32; c < 64; c += 8) {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                  float x, y;
-                  unpack2(fmul2(pack2(__uint_as_float(o[i]), __uint_as_float(o[i + 1])), corr2), x, y);
-                  o[i] = __float_as_uint(x);
-                  o[i + 1] = __float_as_uint(y);
-                }
-                tmem_st32(tmem + lane_off + kAtColO + cc * 32, o);
+                for (int u = 0; u < 4; ++u)
+                  mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
               }
-              tmem_st_wait();
             }
           }
-          const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nm2 = pack2(-m_used, -m_used);
-          uint64_t l2[2] = {0ull, 0ull};                                    // two chains of packed row sums
+        }
+        const float mx = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
+        if (j == 0) {
+          m_used = mx;                        // column 0 is visible to every row, so mx is finite
+        } else {
+          const bool need = mx > m_used + kRescaleStep;
+          if (__any_sync(0xffffffffu, need)) {
+            // O must be at rest: the P V of the previous tile (it completed before this tile's Q K^T)
+            mbar_wait_spin(pv_done(x), (g - 1) & 1, abort_flag);
+            tc_fence_after();
+            const float corr = need ? fast_exp2(m_used - mx) : 1.0f;
+            if (need) m_used = mx;
+            l_run *= corr;
+            const uint64_t corr2 = pack2(corr, corr);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            float p0, p1;
-            unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
-            p0 = fast_exp2(p0);
-            p1 = fast_exp2(p1);
-            l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
-            __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-            pw[c] = *reinterpret_cast<uint32_t*>(&pk);
+            for (int cc = 0; cc < 4; ++cc) {
+              uint32_t o[32];
+              tmem_ld32(o_addr + cc * 32, o);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                float y0, y1;
+                unpack2(fmul2(pack2(__uint_as_float(o[i]), __uint_as_float(o[i + 1])), corr2), y0, y1);
+                o[i] = __float_as_uint(y0);
+                o[i + 1] = __float_as_uint(y1);
+              }
+              tmem_st32(o_addr + cc * 32, o);
+            }
+            tmem_st_wait();
           }
+        }
+        // ---- pass 2: P = 2^(s * scale - m), packed to bf16 over the first half of S
+        const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nm2 = pack2(-m_used, -m_used);
+        uint64_t l2[2] = {0ull, 0ull};                                  // two chains of packed row sums
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t pw[32];
+          if (n_ch > 2 * hf) {
+            uint32_t sr[64];
+            tmem_ld32(s_addr + 64 * hf, sr);
+            if (n_ch > 2 * hf + 1) tmem_ld32(s_addr + 64 * hf + 32, sr + 32);
+            tmem_ld_wait();
+            const int lim = n_ch > 2 * hf + 1 ? 64 : 32;
+            const int vis = grow - (c0 + 64 * hf);
+            if (c0 + 64 * hf + lim - 1 > r0) {
+#pragma unroll
+              for (int c = 0; c < 64; ++c)
+                if (c > vis) sr[c] = 0xFF800000u;
+            }
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+              float p0, p1;
+              unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
+              p0 = fast_exp2(p0);
+              p1 = fast_exp2(p1);
+              l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
+              __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+              pw[c] = *reinterpret_cast<uint32_t*>(&pk);
+            }
+            if (lim == 64) {
+#pragma unroll
+              for (int c = 16; c < 32; ++c) {
+                float p0, p1;
+                unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
+                p0 = fast_exp2(p0);
+                p1 = fast_exp2(p1);
+                l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
+                __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                pw[c] = *reinterpret_cast<uint32_t*>(&pk);
+              }
+            } else {
+#pragma unroll
+              for (int c = 16; c < 32; ++c) pw[c] = 0u;
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) pw[c] = 0u;
+          }
+          tmem_st32(s_addr + 32 * hf, pw);                             // P half hf: columns 32 hf .. 32 hf + 31
+        }
+        {
           float la, lb;
           unpack2(fadd2(l2[0], l2[1]), la, lb);
           l_run += la + lb;
         }
-        tmem_st32(s_addr, pw);                                             // P overwrites its own S buffer
         tmem_st_wait();
-        if (j == I.n_tiles - 1 && kv_end == I.n && kv_end < c0 + kAtBN) {
-          // ragged last tile of the sequence: zero the V rows past its end (both 64-dim halves); past
-          // the end of an inner query tile the rows are the sequence's own and P is 0 there
-          const int s = g % kAtStages;
-          mbar_wait(smem_u32(&v_full[s]), (g / kAtStages) & 1, abort_flag);
-          char* vz = st_s + (size_t)s * kAtStage + kAtTile;
-          const int first = kv_end - c0;
-          for (int u = (warp - 2) * 32 + lane; u < 2 * kAtBN * 8; u += 128) {
-            const int r = (u >> 3) & (kAtBN - 1);
-            if (r >= first)
-              *reinterpret_cast<uint4*>(vz + (u >> 9) * (kAtBN * 128) + r * 128 + (u & 7) * 16) = make_uint4(0, 0, 0, 0);
+        if (j == L.n_tiles - 1 && L.q_hi == I.n) {
+          // last tile of the sequence (only lane A of pair 0 gets here): the P V covers keys up to the next
+          // multiple of 16; zero the V rows between the sequence's end and that bound (both 64-dim halves).
+          // Other query tiles need nothing: rows past their end are the sequence's own and P is 0 there.
+          const int valid = I.n - c0, pad = at_cols(L, j) - valid;
+          if (pad > 0) {
+            const int T = T0 + 2 * j + 1, s = T % kAtRing;
+            mbar_wait_spin(ring_full(s), (T / kAtRing) & 1, abort_flag);
+            char* v_s = ring_s + s * kAtTile;
+            for (int u = quad * 32 + lane; u < pad * 16; u += 128) {
+              const int r = valid + (u >> 4);
+              *reinterpret_cast<uint4*>(v_s + ((u >> 3) & 1) * (kAtBN * 128) + r * 128 + (u & 7) * 16) = make_uint4(0, 0, 0, 0);
+            }
+            fence_proxy_async();
           }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&p_full[sb]));
+        if (lane == 0) mbar_arrive(p_full(x));
+        if (q_slot_held >= 0) {
+          // the previous item's staged output has long been read: hand its Q slot back to the producer
+          if (lane == 0) { bulk_wait_read<0>(); mbar_arrive(q_done(x, q_slot_held)); }
+          q_slot_held = -1;
+        }
       }
-      // ---- epilogue: O / l -> bf16 -> out[b][row][h][:], 32 columns at a time through the warp's
-      // staging buffer (16-byte units XOR-swizzled by row pair: no bank conflicts either way)
-      const int gl = g0 + I.n_tiles - 1;
-      mbar_wait(smem_u32(&pv_done[gl & 1]), (gl >> 1) & 1, abort_flag);
+      // ---- epilogue: O / l -> bf16 -> out[b][row][h][:], 32 columns at a time, staged in this warp's 8 KB of
+      // the item's Q slot (16-byte units XOR-swizzled by row pair: the 64-byte swizzle of the tensor map)
+      const int gl = g0 + L.n_tiles - 1;
+      mbar_wait_spin(pv_done(x), gl & 1, abort_flag);
       tc_fence_after();
       const float inv = 1.0f / l_run;
-      char* so = o_stage + (warp - 2) * 2048;
-      __nv_bfloat16* otile = a.out + (((size_t)I.b * a.n_max + I.q0 + quad * 32) * a.H + I.h) * 128;
-      const int rows_here = I.q_hi - (I.q0 + quad * 32);               // owned rows among this warp's 32
+      const int rows_here = L.q_hi - r0;                               // owned rows among this warp's 32
+      const bool whole = rows_here >= 32;                              // warp-uniform
+      const int qs = n_item & 1;
+      char* so = smem + (2 * x + qs) * kAtTile + quad * 8192;
+      __nv_bfloat16* otile = a.out + (((size_t)I.b * a.n_max + r0) * a.H + I.h) * 128;
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
         uint32_t o[32];
-        tmem_ld32(tmem + lane_off + kAtColO + cc * 32, o);
+        tmem_ld32(o_addr + cc * 32, o);
         tmem_ld_wait();
         if (cc == 3) {                                   // O is in registers: the next item may overwrite it
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(o_free));
+          if (lane == 0) mbar_arrive(o_free(x));
         }
+        char* sb = so + cc * 2048;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           uint4 w;
@@ -386,25 +537,35 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
           w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
           w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
-          *reinterpret_cast<uint4*>(so + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
+          *reinterpret_cast<uint4*>(sb + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
         }
-        __syncwarp();
+        if (whole) {
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) tma_store_4d(mo, smem_u32(sb), cc * 32, I.h, r0, I.b);
+        } else {
+          __syncwarp();
 #pragma unroll
-        for (int it = 0; it < 4; ++it) {
-          const int r = it * 8 + (lane >> 2), u = lane & 3;
-          const uint4 w = *reinterpret_cast<const uint4*>(so + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
-          if (r < rows_here) *reinterpret_cast<uint4*>(otile + (size_t)r * a.H * 128 + cc * 32 + u * 8) = w;
+          for (int it = 0; it < 4; ++it) {
+            const int r = it * 8 + (lane >> 2), u = lane & 3;
+            const uint4 w = *reinterpret_cast<const uint4*>(sb + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
+            if (r < rows_here) *reinterpret_cast<uint4*>(otile + (size_t)r * a.H * 128 + cc * 32 + u * 8) = w;
+          }
         }
-        __syncwarp();
       }
-      g0 += I.n_tiles;
+      if (lane == 0) bulk_commit();
+      __syncwarp();
+      q_slot_held = qs;
+      g0 += L.n_tiles;
       ++n_item;
+      T0 += 2 * I.n_kv;
     }
+    if (q_slot_held >= 0 && lane == 0) { bulk_wait_read<0>(); mbar_arrive(q_done(x, q_slot_held)); }
     if (*abort_flag && row == 0) report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 256); }
+  if (warp == 11) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
 bool attn_prefill_tc_supported(const dl_ctx* ctx) {
@@ -422,15 +583,20 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
   AtMaps maps;
   const uint64_t dims[2] = {128ull, (uint64_t)rows};
   const uint64_t strides[1] = {256ull};
-  const uint32_t box_q[2] = {64u, (uint32_t)kAtBM};
-  const uint32_t box_kv[2] = {64u, (uint32_t)kAtBN};
-  if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.q), q, 2, dims, strides, box_q) ||
-      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.k), k_cache, 2, dims, strides, box_kv) ||
-      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.v), v_cache, 2, dims, strides, box_kv))
+  const uint32_t box[2] = {64u, 128u};
+  // out [B][n_max][H][128]: 32 rows x 32 columns of one head per store
+  const uint64_t dims_o[4] = {128ull, (uint64_t)d.n_heads, (uint64_t)n_max, (uint64_t)B};
+  const uint64_t strides_o[3] = {256ull, 256ull * d.n_heads, 256ull * d.n_heads * n_max};
+  const uint32_t box_o[4] = {32u, 1u, 32u, 1u};
+  if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.q), q, 2, dims, strides, box) ||
+      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.k), k_cache, 2, dims, strides, box) ||
+      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.v), v_cache, 2, dims, strides, box) ||
+      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.o), out, 4, dims_o, strides_o, box_o,
+                       CU_TENSOR_MAP_SWIZZLE_64B))
     return cudaErrorInvalidValue;
   AtArgs a;
   a.cache_len = cache_len; a.out = static_cast<__nv_bfloat16*>(out); a.status = ctx->ws.base ? ctx->ws.status : nullptr;
-  a.B = B; a.H = d.n_heads; a.cap = cap; a.n_max = n_max; a.q_tiles = (n_max + kAtBM - 1) / kAtBM;
+  a.B = B; a.H = d.n_heads; a.cap = cap; a.n_max = n_max; a.q_pairs = (n_max + 2 * kAtBM - 1) / (2 * kAtBM);
   a.scale_log2 = scale * 1.4426950408889634f;
   static int attr_set[64];
   if (!attr_set[ctx->device & 63]) {
@@ -438,9 +604,9 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
     if (e != cudaSuccess) return e;
     attr_set[ctx->device & 63] = 1;
   }
-  const long long items = (long long)B * d.n_heads * a.q_tiles;
+  const long long items = (long long)B * d.n_heads * a.q_pairs;
   if (items >= (1LL << 31)) return cudaErrorInvalidValue;
-  const int grid = (int)std::min<long long>(items, 2LL * ctx->sm_count);
+  const int grid = (int)std::min<long long>(items, (long long)ctx->sm_count);
   attn_prefill_tc_kernel<<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
   return cudaGetLastError();
 }

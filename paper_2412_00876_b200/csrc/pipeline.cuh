@@ -8,6 +8,7 @@
 namespace dl {
 
 constexpr int kSpinLimit = 1 << 22;
+constexpr int kSpinLimitBusy = 1 << 21;     // polls of the sleepless wait (each try_wait may itself suspend)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -32,6 +33,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// One poll that never suspends the thread (for a role that watches several barriers in turn).
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false (and raises *abort) when the bound is hit or another warp aborted.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
   if (mbar_try_wait(bar, parity)) return !*abort;            // fast path: the phase is already complete
@@ -39,6 +50,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (*abort) return false;
     if (mbar_try_wait(bar, parity)) return true;
     if (i > 32) __nanosleep(40);
+  }
+  *abort = 1;
+  return false;
+}
+// The same bound without the sleep between polls, for hand-offs inside a pipeline whose stages are a
+// few hundred cycles long (try_wait itself suspends the thread for a hardware-chosen time).
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int* abort) {
+  if (mbar_try_wait(bar, parity)) return !*abort;
+  for (int i = 0; i < kSpinLimitBusy; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63) == 63 && *abort) return false;
   }
   *abort = 1;
   return false;
