@@ -14,12 +14,14 @@
 //                (two slots per lane, so an item's Q is in flight while the previous item computes).
 //   warps 9,10 : the MMA-issuing thread of lane A / lane B:
 //                S = Q K^T (128 x N, K-major operands from shared memory), O += P V (P read from
-//                tensor memory, V as an MN-major shared-memory operand), then the next tile's Q K^T.
+//                tensor memory, V as an MN-major shared-memory operand), then the next tile's Q K^T,
+//                issued as one block under a lock so that the two lanes alternate on the tensor pipe.
 //                Full tiles use N = 128 keys; a lane's last tile uses N = keys left rounded up to 16,
 //                in both products, so the tensor pipe does not multiply by padding.
 //   warps 0-3 / 4-7 : softmax of lane A / B, one query row per thread, straight out of tensor memory
-//                in two passes (row maximum, then exponentials).  32-column chunks that no row of the
-//                warp may see (above the causal diagonal) are skipped.  The running maximum is only
+//                with the whole row of the tile held in registers (these warps take the registers the
+//                other warps give back).  32-column chunks that no row of the warp may see (above the
+//                causal diagonal) are skipped.  The running maximum is only
 //                raised when it grows by more than 2^8 (then O is rescaled in tensor memory), so most
 //                tiles never touch O.  P (bf16) overwrites the first half of S.  The same warps
 //                normalise O and write the output: 32 x 32 blocks staged in the item's own Q buffer
@@ -119,39 +121,66 @@ __device__ __forceinline__ int at_cols(const AtLane& L, int j) {
   return min(kAtBN, (L.q_hi - j * kAtBN + 15) & ~15);
 }
 
-// Walks the items of this CTA in the order every role uses; the length of the NEXT item's sequence is
-// requested one item early, so its latency never sits in front of a role's first wait.
+// A load the compiler may not sink towards its use (the point is to have it in flight early).
+__device__ __forceinline__ int ld_early(const int32_t* p) {
+  int v;
+  asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+
+// Walks the items of this CTA (item = p * B * H + b * H + h, stepping by the grid size) in the order
+// every role uses.  The position is kept as (p, b, h) and advanced by additions; the length of the
+// NEXT item's sequence is requested one item early, so its latency never sits in front of a role's
+// first wait.
 struct AtWalker {
   const AtArgs& a;
-  int item, items, bh_count, len_nx;
-  __device__ __forceinline__ int len_of(int it) const { return __ldg(a.cache_len + (it % bh_count) / a.H); }
+  int p, b, h, len, db, dh;
   __device__ __forceinline__ explicit AtWalker(const AtArgs& a_) : a(a_) {
-    bh_count = a.B * a.H;
-    items = bh_count * a.q_pairs;
-    item = (int)blockIdx.x - (int)gridDim.x;
-    len_nx = (int)blockIdx.x < items ? len_of(blockIdx.x) : 0;
+    const int bh_count = a.B * a.H;
+    p = (int)blockIdx.x / bh_count;
+    const int bh = (int)blockIdx.x - p * bh_count;
+    b = bh / a.H;
+    h = bh - b * a.H;
+    db = (int)gridDim.x / a.H;
+    dh = (int)gridDim.x - db * a.H;
+    len = p < a.q_pairs ? ld_early(a.cache_len + b) : 0;
   }
   // Advances to the next item that exists (a sequence of 256 p rows or fewer has no pair p).
   __device__ __forceinline__ bool next(AtItem& I) {
     for (;;) {
-      item += (int)gridDim.x;
-      if (item >= items) return false;
-      const int len = len_nx;
-      const int nx = item + (int)gridDim.x;
-      if (nx < items) len_nx = len_of(nx);
-      const int p = item / bh_count;
-      const int bh = item - p * bh_count;
-      I.b = bh / a.H;
-      I.h = bh - I.b * a.H;
-      I.n = min(max(len, 0), min(a.cap, a.n_max));
-      I.q_hi = I.n - p * 2 * kAtBM;
+      if (p >= a.q_pairs) return false;
+      const int cp = p, cb = b, ch = h, clen = len;
+      h += dh;
+      b += db;
+      if (h >= a.H) { h -= a.H; ++b; }
+      while (b >= a.B) { b -= a.B; ++p; }
+      if (p < a.q_pairs) len = ld_early(a.cache_len + b);
+      I.b = cb;
+      I.h = ch;
+      I.n = min(max(clen, 0), min(a.cap, a.n_max));
+      I.q_hi = I.n - cp * 2 * kAtBM;
       if (I.q_hi <= 0) continue;
       I.n_kv = (I.q_hi + kAtBN - 1) / kAtBN;
-      I.row_base = bh * a.cap;                                      // first row of this (b, h) in the caches
+      I.row_base = (cb * a.H + ch) * a.cap;                         // first row of this (b, h) in the caches
       return true;
     }
   }
 };
+
+// The two MMA-issuing threads take turns: a lane issues a whole block (P V, then the next Q K^T) before
+// the other lane's block is queued, so the lanes run half a period apart and one lane's softmax has
+// the other lane's MMAs to hide behind.  Held only while issuing, never across a wait.
+__device__ __forceinline__ void pipe_lock(int* l, volatile int* abort) {
+  for (int i = 0; atomicCAS(l, 0, 1) != 0; ++i)
+    if (i > kSpinLimitBusy) { *abort = 1; return; }
+}
+__device__ __forceinline__ void pipe_unlock(int* l) { atomicExch(l, 0); }
+
+// Register budget per role (the kernel starts every thread at 168): the producer / MMA warps give
+// registers back, the softmax warps take them to hold a whole score row.
+constexpr int kAtRegsSmall = 72, kAtRegsSoftmax = 216;
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
@@ -178,9 +207,11 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
   auto o_free = [&](int x) { return smem_u32(bars + 23 + x); };   // the epilogue has read O (4 warps)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
+  int* pipe_turn = reinterpret_cast<int*>(bars + 34);
 
   if (tid == 0) {
     *abort_flag = 0;
+    *pipe_turn = 0;
     for (int s = 0; s < kAtRing; ++s) {
       mbar_init(ring_full(s), 1);
       mbar_init(ring_free(0, s), 1);
@@ -203,6 +234,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
 
   if (warp == 8) {
     // ---------------------------------------------------------------- TMA producer
+    reg_dec<kAtRegsSmall>();
     if (lane == 0) {
       const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(maps.q);
       const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(maps.k);
@@ -211,15 +243,15 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       // cursor of the ring
       AtWalker Wr(a);
       AtItem Ir;
-      bool hr = Wr.next(Ir);
       int T = 0, jr = 0;                       // ring tiles issued so far / tile index within Ir (K, V alternating)
       uint32_t free_par[2] = {0u, 0u};         // bit s: parity of the next phase of ring_free(x, s) to wait for
       uint32_t prev_b = 0u;                    // bit s: the tile now in slot s is read by lane B too
       // cursors of the Q loads
-      AtWalker Wq0(a), Wq1(a);
+      AtWalker Wq0 = Wr, Wq1 = Wr;
       AtItem Iq[2];
       bool hq[2];
       int nq[2] = {0, 0};                      // Q loads issued so far per lane
+      bool hr = Wr.next(Ir);
       hq[0] = Wq0.next(Iq[0]);
       hq[1] = Wq1.next(Iq[1]);
       while (hq[1] && !at_lane(Iq[1], 1).exists) hq[1] = Wq1.next(Iq[1]);
@@ -291,6 +323,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     }
   } else if (warp == 9 || warp == 10) {
     // ---------------------------------------------------------------- MMA issuer of one lane
+    reg_dec<kAtRegsSmall>();
     if (lane == 0) {
       const int x = warp - 9;
       const uint32_t t_o = tmem + x * kAtLaneCols + kAtColO, t_s = tmem + x * kAtLaneCols + kAtColS;
@@ -303,10 +336,9 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         if (!L.exists) { T0 += 2 * I.n_kv; continue; }
         const int qs = n_item & 1;
         const uint64_t q_desc = smem_desc_sw128(smem_u32(smem + (2 * x + qs) * kAtTile));
+        auto wait_ring = [&](int T) { mbar_wait_spin(ring_full(T % kAtRing), (T / kAtRing) & 1, abort_flag); };
         auto issue_qk = [&](int j) {
-          const int T = T0 + 2 * j, s = T % kAtRing;
-          mbar_wait_spin(ring_full(s), (T / kAtRing) & 1, abort_flag);
-          tc_fence_after();
+          const int s = (T0 + 2 * j) % kAtRing;
           const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile));
           const uint32_t idesc_qk = idesc_bf16(kAtBM, (uint32_t)at_cols(L, j));
 #pragma unroll
@@ -317,21 +349,29 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           mma_commit(ring_free(x, s));
         };
         mbar_wait_spin(q_full(x, qs), (n_item >> 1) & 1, abort_flag);
+        wait_ring(T0);
+        tc_fence_after();
+        pipe_lock(pipe_turn, abort_flag);
         issue_qk(0);
+        pipe_unlock(pipe_turn);
         for (int j = 0; j < L.n_tiles; ++j) {
           const int g = g0 + j;
           const int T = T0 + 2 * j + 1, s = T % kAtRing;
-          mbar_wait_spin(p_full(x), g & 1, abort_flag);
+          // operands first (they land long before), then the softmax's hand-over
+          wait_ring(T);
+          if (j + 1 < L.n_tiles) wait_ring(T + 1);
           if (j == 0) mbar_wait_spin(o_free(x), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
-          mbar_wait_spin(ring_full(s), (T / kAtRing) & 1, abort_flag);
+          mbar_wait_spin(p_full(x), g & 1, abort_flag);
           tc_fence_after();
           const uint64_t v_desc = smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128);
           const int ksteps = at_cols(L, j) >> 4;
+          pipe_lock(pipe_turn, abort_flag);
           for (int ks = 0; ks < ksteps; ++ks)
             mma_ts(t_o, t_s + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv, (j | ks) != 0);
           mma_commit(pv_done(x));
           mma_commit(ring_free(x, s));
           if (j + 1 < L.n_tiles) issue_qk(j + 1);                      // overwrites P: in order behind the P V
+          pipe_unlock(pipe_turn);
         }
         g0 += L.n_tiles;
         ++n_item;
@@ -340,6 +380,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     }
   } else if (warp < 8) {
     // ---------------------------------------------------------------- softmax / epilogue warps of one lane
+    reg_inc<kAtRegsSoftmax>();
     const int x = warp >> 2;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                                  // row within the query tile
@@ -364,37 +405,31 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         const int n_ch = min(4, (min(L.q_hi, r0 + 32) - c0 + 31) >> 5);
         mbar_wait_spin(s_full(x), g & 1, abort_flag);
         tc_fence_after();
-        // ---- pass 1: row maximum of the raw scores (max commutes with the positive scale)
+        // ---- the row's scores of this tile (chunks no row of the warp sees stay at -inf)
+        uint32_t sr[128];
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          if (n_ch > cc) {
+            tmem_ld32(s_addr + 32 * cc, sr + 32 * cc);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) sr[32 * cc + c] = 0xFF800000u;  // -inf
+          }
+        }
+        tmem_ld_wait();
+        if (c0 + 32 * n_ch - 1 > r0) {                                  // the tile reaches past the warp's first row
+          const int vis = grow - c0;                                   // columns 0..vis are visible to this row
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (c > vis) sr[c] = 0xFF800000u;
+        }
+        // ---- row maximum of the raw scores (max commutes with the positive scale)
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          if (n_ch > 2 * hf) {
-            uint32_t sr[64];
-            tmem_ld32(s_addr + 64 * hf, sr);
-            if (n_ch > 2 * hf + 1) tmem_ld32(s_addr + 64 * hf + 32, sr + 32);
-            tmem_ld_wait();
-            const int lim = n_ch > 2 * hf + 1 ? 64 : 32;
-            const int vis = grow - (c0 + 64 * hf);                     // columns 0..vis of this half are visible
-            if (c0 + 64 * hf + lim - 1 > r0) {
+        for (int c = 0; c < 128; c += 8) {
 #pragma unroll
-              for (int c = 0; c < 64; ++c)
-                if (c > vis) sr[c] = 0xFF800000u;                      // -inf
-            }
-#pragma unroll
-            for (int c = 0; c < 32; c += 8) {
-#pragma unroll
-              for (int u = 0; u < 4; ++u)
-                mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
-            }
-            if (lim == 64) {
-#pragma unroll
-              for (int c = 32; c < 64; c += 8) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                  mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
-              }
-            }
-          }
+          for (int u = 0; u < 4; ++u)
+            mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
         }
         const float mx = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
         if (j == 0) {
@@ -426,52 +461,31 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
             tmem_st_wait();
           }
         }
-        // ---- pass 2: P = 2^(s * scale - m), packed to bf16 over the first half of S
+        // ---- P = 2^(s * scale - m), packed to bf16 over the first half of S
         const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nm2 = pack2(-m_used, -m_used);
         uint64_t l2[2] = {0ull, 0ull};                                  // two chains of packed row sums
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
           uint32_t pw[32];
-          if (n_ch > 2 * hf) {
-            uint32_t sr[64];
-            tmem_ld32(s_addr + 64 * hf, sr);
-            if (n_ch > 2 * hf + 1) tmem_ld32(s_addr + 64 * hf + 32, sr + 32);
-            tmem_ld_wait();
-            const int lim = n_ch > 2 * hf + 1 ? 64 : 32;
-            const int vis = grow - (c0 + 64 * hf);
-            if (c0 + 64 * hf + lim - 1 > r0) {
 #pragma unroll
-              for (int c = 0; c < 64; ++c)
-                if (c > vis) sr[c] = 0xFF800000u;
-            }
+          for (int cq = 0; cq < 2; ++cq) {
+            const int cc = 2 * hf + cq;
+            if (n_ch > cc) {
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
-              float p0, p1;
-              unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
-              p0 = fast_exp2(p0);
-              p1 = fast_exp2(p1);
-              l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
-              __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-              pw[c] = *reinterpret_cast<uint32_t*>(&pk);
-            }
-            if (lim == 64) {
-#pragma unroll
-              for (int c = 16; c < 32; ++c) {
+              for (int c = 0; c < 16; ++c) {
                 float p0, p1;
-                unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
+                unpack2(ffma2(pack2(__uint_as_float(sr[32 * cc + 2 * c]), __uint_as_float(sr[32 * cc + 2 * c + 1])), sc2, nm2),
+                        p0, p1);
                 p0 = fast_exp2(p0);
                 p1 = fast_exp2(p1);
                 l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
                 __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                pw[c] = *reinterpret_cast<uint32_t*>(&pk);
+                pw[16 * cq + c] = *reinterpret_cast<uint32_t*>(&pk);
               }
             } else {
 #pragma unroll
-              for (int c = 16; c < 32; ++c) pw[c] = 0u;
+              for (int c = 0; c < 16; ++c) pw[16 * cq + c] = 0u;
             }
-          } else {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) pw[c] = 0u;
           }
           tmem_st32(s_addr + 32 * hf, pw);                             // P half hf: columns 32 hf .. 32 hf + 31
         }
@@ -539,16 +553,22 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
           *reinterpret_cast<uint4*>(sb + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
         }
-        if (whole) {
-          fence_proxy_async();
-          __syncwarp();
-          if (lane == 0) tma_store_4d(mo, smem_u32(sb), cc * 32, I.h, r0, I.b);
-        } else {
-          __syncwarp();
+      }
+      if (whole) {
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) tma_store_4d(mo, smem_u32(so + cc * 2048), cc * 32, I.h, r0, I.b);
+        }
+      } else {
+        __syncwarp();
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
 #pragma unroll
           for (int it = 0; it < 4; ++it) {
             const int r = it * 8 + (lane >> 2), u = lane & 3;
-            const uint4 w = *reinterpret_cast<const uint4*>(sb + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
+            const uint4 w = *reinterpret_cast<const uint4*>(so + cc * 2048 + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
             if (r < rows_here) *reinterpret_cast<uint4*>(otile + (size_t)r * a.H * 128 + cc * 32 + u * 8) = w;
           }
         }
@@ -562,6 +582,8 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     }
     if (q_slot_held >= 0 && lane == 0) { bulk_wait_read<0>(); mbar_arrive(q_done(x, q_slot_held)); }
     if (*abort_flag && row == 0) report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
+  } else {
+    reg_dec<kAtRegsSmall>();                             // warp 11: same budget as the rest of its warpgroup
   }
   tc_fence_before();
   __syncthreads();
