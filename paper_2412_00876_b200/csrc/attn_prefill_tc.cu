@@ -19,11 +19,11 @@
 //                Full tiles use N = 128 keys; a lane's last tile uses N = keys left rounded up to 16,
 //                in both products, so the tensor pipe does not multiply by padding.
 //   warps 0-3 / 4-7 : softmax of lane A / B, one query row per thread, straight out of tensor memory
-//                with the whole row of the tile held in registers (these warps take the registers the
-//                other warps give back).  32-column chunks that no row of the warp may see (above the
-//                causal diagonal) are skipped.  The running maximum is only
-//                raised when it grows by more than 2^8 (then O is rescaled in tensor memory), so most
-//                tiles never touch O.  P (bf16) overwrites the first half of S.  The same warps
+//                in one pass of 32-column chunks (the next chunk's load in flight meanwhile; these warps
+//                take the registers the other warps give back).  Chunks that no row of the warp may see
+//                (above the causal diagonal) are skipped.  The running maximum is only raised when the
+//                tile's maximum exceeds it by more than 2^8 (then O is rescaled in tensor memory and the
+//                tile redone), so most tiles never touch O.  P (bf16) overwrites the first half of S.  The same warps
 //                normalise O and write the output: 32 x 32 blocks staged in the item's own Q buffer
 //                (free once its last Q K^T has run) and sent with TMA stores; a clipped tile at the
 //                top of a sequence, whose surplus rows belong to the next tile, is written with
@@ -405,43 +405,72 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         const int n_ch = min(4, (min(L.q_hi, r0 + 32) - c0 + 31) >> 5);
         mbar_wait_spin(s_full(x), g & 1, abort_flag);
         tc_fence_after();
-        // ---- the row's scores of this tile (chunks no row of the warp sees stay at -inf)
-        uint32_t sr[128];
+        // ---- one pass over the tile in 32-column chunks, the next chunk's load in flight while this one is
+        // worked on.  Exponentials are taken against the maximum the row already uses (the first chunk's
+        // own maximum on an item's first tile); the tile's true maximum is tracked alongside, and only if
+        // it turns out more than 2^8 above the one used is the tile done again after rescaling O.
+        uint32_t pw[64];                                                // P of the row, bf16 pairs
+        const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2);
+        const int vis = grow - c0;                                      // columns 0..vis are visible to this row
+        float mx_tile;
+        bool first_try = true;
+        for (;;) {
+          uint32_t buf[2][32];
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}; // four independent chains
+          uint64_t l2[2] = {0ull, 0ull};                                // two chains of packed row sums
+          if (n_ch > 0) tmem_ld32(s_addr, buf[0]);
+          tmem_ld_wait();
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          if (n_ch > cc) {
-            tmem_ld32(s_addr + 32 * cc, sr + 32 * cc);
-          } else {
+          for (int cc = 0; cc < 4; ++cc) {
+            uint32_t* sr = buf[cc & 1];
+            if (n_ch > cc) {
+              if (n_ch > cc + 1) tmem_ld32(s_addr + 32 * (cc + 1), buf[(cc + 1) & 1]);
+              if (c0 + 32 * cc + 31 > r0) {                             // the chunk reaches past the warp's first row
 #pragma unroll
-            for (int c = 0; c < 32; ++c) sr[32 * cc + c] = 0xFF800000u;  // -inf
+                for (int c = 0; c < 32; ++c)
+                  if (32 * cc + c > vis) sr[c] = 0xFF800000u;           // -inf
+              }
+#pragma unroll
+              for (int c = 0; c < 32; c += 8) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                  mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
+              }
+              if (cc == 0 && j == 0 && first_try)                       // column 0 is visible to every row: finite
+                m_used = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
+              const uint64_t nm2 = pack2(-m_used, -m_used);
+#pragma unroll
+              for (int c = 0; c < 16; ++c) {
+                float p0, p1;
+                unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
+                p0 = fast_exp2(p0);
+                p1 = fast_exp2(p1);
+                l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
+                __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                pw[16 * cc + c] = *reinterpret_cast<uint32_t*>(&pk);
+              }
+              tmem_ld_wait();
+            } else {
+#pragma unroll
+              for (int c = 0; c < 16; ++c) pw[16 * cc + c] = 0u;
+            }
           }
-        }
-        tmem_ld_wait();
-        if (c0 + 32 * n_ch - 1 > r0) {                                  // the tile reaches past the warp's first row
-          const int vis = grow - c0;                                   // columns 0..vis are visible to this row
-#pragma unroll
-          for (int c = 0; c < 128; ++c)
-            if (c > vis) sr[c] = 0xFF800000u;
-        }
-        // ---- row maximum of the raw scores (max commutes with the positive scale)
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
-#pragma unroll
-        for (int c = 0; c < 128; c += 8) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-            mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
-        }
-        const float mx = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-        if (j == 0) {
-          m_used = mx;                        // column 0 is visible to every row, so mx is finite
-        } else {
-          const bool need = mx > m_used + kRescaleStep;
-          if (__any_sync(0xffffffffu, need)) {
+          mx_tile = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
+          const bool need = mx_tile > m_used + kRescaleStep;
+          if (!__any_sync(0xffffffffu, need)) {
+            float la, lb;
+            unpack2(fadd2(l2[0], l2[1]), la, lb);
+            l_run += la + lb;
+            break;
+          }
+          // rare: raise the maximum (rescaling what O and the row sum hold so far), then redo the tile
+          first_try = false;
+          const float corr = need ? fast_exp2(m_used - mx_tile) : 1.0f;
+          if (need) m_used = mx_tile;
+          if (j > 0) {
             // O must be at rest: the P V of the previous tile (it completed before this tile's Q K^T)
             mbar_wait_spin(pv_done(x), (g - 1) & 1, abort_flag);
             tc_fence_after();
-            const float corr = need ? fast_exp2(m_used - mx) : 1.0f;
-            if (need) m_used = mx;
             l_run *= corr;
             const uint64_t corr2 = pack2(corr, corr);
 #pragma unroll
@@ -461,39 +490,8 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
             tmem_st_wait();
           }
         }
-        // ---- P = 2^(s * scale - m), packed to bf16 over the first half of S
-        const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nm2 = pack2(-m_used, -m_used);
-        uint64_t l2[2] = {0ull, 0ull};                                  // two chains of packed row sums
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          uint32_t pw[32];
-#pragma unroll
-          for (int cq = 0; cq < 2; ++cq) {
-            const int cc = 2 * hf + cq;
-            if (n_ch > cc) {
-#pragma unroll
-              for (int c = 0; c < 16; ++c) {
-                float p0, p1;
-                unpack2(ffma2(pack2(__uint_as_float(sr[32 * cc + 2 * c]), __uint_as_float(sr[32 * cc + 2 * c + 1])), sc2, nm2),
-                        p0, p1);
-                p0 = fast_exp2(p0);
-                p1 = fast_exp2(p1);
-                l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
-                __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                pw[16 * cq + c] = *reinterpret_cast<uint32_t*>(&pk);
-              }
-            } else {
-#pragma unroll
-              for (int c = 0; c < 16; ++c) pw[16 * cq + c] = 0u;
-            }
-          }
-          tmem_st32(s_addr + 32 * hf, pw);                             // P half hf: columns 32 hf .. 32 hf + 31
-        }
-        {
-          float la, lb;
-          unpack2(fadd2(l2[0], l2[1]), la, lb);
-          l_run += la + lb;
-        }
+        tmem_st32(s_addr, pw);                                         // P (bf16) over the first half of S
+        tmem_st32(s_addr + 32, pw + 32);
         tmem_st_wait();
         if (j == L.n_tiles - 1 && L.q_hi == I.n) {
           // last tile of the sequence (only lane A of pair 0 gets here): the P V covers keys up to the next
