@@ -14,8 +14,8 @@
 //                (two slots per lane, so an item's Q is in flight while the previous item computes).
 //   warps 9,10 : the MMA-issuing thread of lane A / lane B:
 //                S = Q K^T (128 x N, K-major operands from shared memory), O += P V (P read from
-//                tensor memory, V as an MN-major shared-memory operand), then the next tile's Q K^T,
-//                issued as one block under a lock so that the two lanes alternate on the tensor pipe.
+//                tensor memory, V as an MN-major shared-memory operand), then the next tile's Q K^T;
+//                completion signals follow the block, the softmax's first.
 //                Full tiles use N = 128 keys; a lane's last tile uses N = keys left rounded up to 16,
 //                in both products, so the tensor pipe does not multiply by padding.
 //   warps 0-3 / 4-7 : softmax of lane A / B, one query row per thread, straight out of tensor memory
@@ -167,14 +167,21 @@ struct AtWalker {
   }
 };
 
-// The two MMA-issuing threads take turns: a lane issues a whole block (P V, then the next Q K^T) before
-// the other lane's block is queued, so the lanes run half a period apart and one lane's softmax has
-// the other lane's MMAs to hide behind.  Held only while issuing, never across a wait.
+// Whether the two MMA-issuing threads take turns (a lane issues a whole block, P V then the next
+// Q K^T, before the other lane's block is queued).  Measured both ways: with turns the lanes run half a
+// period apart, one lane's softmax hiding behind the other's MMAs, but a single thread cannot keep the
+// tensor pipe fed (a chain of eight dependent MMAs costs its issuer ~200 cycles of latency on top of
+// 8 x 64, and each completion signal ~90 more) and a softmax warp alone on its scheduler does not
+// overlap its exponentials with its arithmetic.  Without turns the lanes fall into step: both issue
+// at once (the pipe interleaves the two chains at full rate) and both softmax at once (two warps per
+// scheduler interleave).  The second is 3-7 % faster on the shapes at hand, so it is the default.
+constexpr bool kAtTakeTurns = false;
 __device__ __forceinline__ void pipe_lock(int* l, volatile int* abort) {
+  if (!kAtTakeTurns) return;
   for (int i = 0; atomicCAS(l, 0, 1) != 0; ++i)
     if (i > kSpinLimitBusy) { *abort = 1; return; }
 }
-__device__ __forceinline__ void pipe_unlock(int* l) { atomicExch(l, 0); }
+__device__ __forceinline__ void pipe_unlock(int* l) { if (kAtTakeTurns) atomicExch(l, 0); }
 
 // Register budget per role (the kernel starts every thread at 168): the producer / MMA warps give
 // registers back, the softmax warps take them to hold a whole score row.
@@ -345,8 +352,13 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           for (int ks = 0; ks < 8; ++ks)
             mma_ss(t_s, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
                    k_desc + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
-          mma_commit(s_full(x));
-          mma_commit(ring_free(x, s));
+        };
+        // Completion signals are issued after the lock is released (each one holds the issuing thread
+        // for about as long as an MMA, and the other lane's block can run meanwhile); a commit covers
+        // every MMA this thread has issued so far.
+        auto commit_qk = [&](int j) {
+          mma_commit(s_full(x));                                       // first: the softmax warps wait on it
+          mma_commit(ring_free(x, (T0 + 2 * j) % kAtRing));
         };
         mbar_wait_spin(q_full(x, qs), (n_item >> 1) & 1, abort_flag);
         wait_ring(T0);
@@ -354,6 +366,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         pipe_lock(pipe_turn, abort_flag);
         issue_qk(0);
         pipe_unlock(pipe_turn);
+        commit_qk(0);
         for (int j = 0; j < L.n_tiles; ++j) {
           const int g = g0 + j;
           const int T = T0 + 2 * j + 1, s = T % kAtRing;
@@ -368,10 +381,11 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           pipe_lock(pipe_turn, abort_flag);
           for (int ks = 0; ks < ksteps; ++ks)
             mma_ts(t_o, t_s + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv, (j | ks) != 0);
-          mma_commit(pv_done(x));
-          mma_commit(ring_free(x, s));
           if (j + 1 < L.n_tiles) issue_qk(j + 1);                      // overwrites P: in order behind the P V
           pipe_unlock(pipe_turn);
+          if (j + 1 < L.n_tiles) commit_qk(j + 1);
+          mma_commit(pv_done(x));
+          mma_commit(ring_free(x, s));
         }
         g0 += L.n_tiles;
         ++n_item;
@@ -529,27 +543,32 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       const int qs = n_item & 1;
       char* so = smem + (2 * x + qs) * kAtTile + quad * 8192;
       __nv_bfloat16* otile = a.out + (((size_t)I.b * a.n_max + r0) * a.H + I.h) * 128;
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t o[32];
-        tmem_ld32(o_addr + cc * 32, o);
+      {
+        uint32_t ob[2][32];                              // the next 32 columns load while these are converted
+        tmem_ld32(o_addr, ob[0]);
         tmem_ld_wait();
-        if (cc == 3) {                                   // O is in registers: the next item may overwrite it
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(o_free(x));
-        }
-        char* sb = so + cc * 2048;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          uint4 w;
-          __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[8 * u]) * inv, __uint_as_float(o[8 * u + 1]) * inv);
-          __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 2]) * inv, __uint_as_float(o[8 * u + 3]) * inv);
-          __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 4]) * inv, __uint_as_float(o[8 * u + 5]) * inv);
-          __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
-          w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
-          w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
-          *reinterpret_cast<uint4*>(sb + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
+        for (int cc = 0; cc < 4; ++cc) {
+          const uint32_t* o = ob[cc & 1];
+          if (cc < 3) tmem_ld32(o_addr + (cc + 1) * 32, ob[(cc + 1) & 1]);
+          char* sb = so + cc * 2048;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            uint4 w;
+            __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[8 * u]) * inv, __uint_as_float(o[8 * u + 1]) * inv);
+            __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 2]) * inv, __uint_as_float(o[8 * u + 3]) * inv);
+            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 4]) * inv, __uint_as_float(o[8 * u + 5]) * inv);
+            __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
+            w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
+            w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
+            *reinterpret_cast<uint4*>(sb + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
+          }
+          if (cc < 3) tmem_ld_wait();
+          if (cc == 2) {                                 // all of O is in registers: the next item may overwrite it
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(o_free(x));
+          }
         }
       }
       if (whole) {
