@@ -208,16 +208,15 @@ def test_decode_attention_other_types():
 
 
 # ------------------------------------------------------------------------------ prefill attention
-@pytest.mark.parametrize("dtype,H,D,lens", [("f32", 8, 64, [68]), ("bf16", 4, 128, [208, 1, 130, 64]),
-                                             ("bf16", 2, 128, [832, 300, 129, 128, 127, 65, 0]),
-                                             ("bf16", 2, 64, [33, 100]), ("f32", 2, 128, [40, 7])])
-def test_prefill_attention(dtype, H, D, lens):
+def _prefill_case(dtype, H, D, lens, amp=1.0):
     from paper_2412_00876_b200 import binding as dl
     B, cap = len(lens), (max(lens) + 63) // 64 * 64
     cfg = wl.CONFIGS[2]
     q = wl.host_normal(cfg, wl.S_Q, (B, H, cap, D), dtype=dtype)
     k = wl.host_normal(cfg, wl.S_K, (B, H, cap, D), dtype=dtype)
     v = wl.host_normal(cfg, wl.S_V, (B, H, cap, D), dtype=dtype)
+    if amp != 1.0:                               # power of two: stays exactly representable
+        q, k = q * amp, k * amp
     scale = 1 / np.sqrt(D)
     n_max = max(lens)
     for impl in (1, 2):
@@ -234,12 +233,34 @@ def test_prefill_attention(dtype, H, D, lens):
         except dl.DlError as e:
             assert impl == 2 and e.code == dl.DL_ERR_UNSUPPORTED and not (dtype == "bf16" and D == 128)
             continue
+        assert ctx.device_status()[0] == 0
         got = wl.from_torch(out)
         for b in range(B):
             n = lens[b]
             ref = np.stack([orc.attention_prefill_compact(q[b, h], k[b, h], v[b, h], n, scale) for h in range(H)], 1)
-            pc.check_att(got[b, :n], ref, f"prefill impl {impl} seq {b}")
+            pc.check_att(got[b, :n], ref, f"prefill impl {impl} seq {b} (n={n})")
             assert np.all(got[b, n:] == 7.0)                  # rows past the length are not written
+
+
+@pytest.mark.parametrize("dtype,H,D,lens", [("f32", 8, 64, [68]), ("bf16", 4, 128, [208, 1, 130, 64]),
+                                             ("bf16", 2, 128, [832, 300, 129, 128, 127, 65, 0]),
+                                             ("bf16", 2, 64, [33, 100]), ("f32", 2, 128, [40, 7])])
+def test_prefill_attention(dtype, H, D, lens):
+    _prefill_case(dtype, H, D, lens)
+
+
+def test_prefill_attention_tile_pair_boundaries():
+    """Lengths on and around the 128-row query tiles, the 256-row tile pairs and the 16-key steps of the
+    tensor-core kernel (a pair whose earlier tile is missing, clipped or full; last key tiles of 1..16 keys)."""
+    _prefill_case("bf16", 2, 128, [256, 257, 255, 272, 240, 384, 385, 383])
+    _prefill_case("bf16", 1, 128, [513, 512, 511, 16, 17, 15, 144, 145, 2])
+    _prefill_case("bf16", 3, 128, [640])
+
+
+def test_prefill_attention_large_scores():
+    """Scores whose row maximum keeps growing by far more than 2^8 from one key tile to the next: the
+    tensor-core kernel has to rescale its accumulator and redo tiles (its rare path)."""
+    _prefill_case("bf16", 2, 128, [600, 300, 129], amp=4.0)
 
 
 def test_prefill_attention_large_grid_is_reproducible():
