@@ -1,7 +1,7 @@
 // Prefill attention over the reduced set on the tensor cores (Eq. 1 applied to S^{P*}):
 // row i of a sequence's compact context attends rows 0..i of the same context.
 // bf16, head_dim 128.  One persistent CTA per SM walks work items (sequence, head, PAIR of 128-row
-// query tiles), longest first.  The two query tiles of a pair run as two lanes, A (the later rows)
+// query tiles), the pairs of a head side by side.  The two query tiles of a pair run as two lanes, A (the later rows)
 // and B (the 128 rows before them): each lane has its own Q buffers, its own score / output
 // accumulators in tensor memory, its own MMA-issuing thread and its own four softmax warps, and both
 // read the same K and V tiles, which are fetched once per pair into a ring shared by the lanes.
@@ -89,10 +89,14 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t x, uint64_t y) {
   return r;
 }
 
+// Tensor maps: Q, K and V each with boxes of 128, 64, 32 and 16 rows (index 0..3), so that a ragged
+// tile at the end of a sequence is fetched with the smallest box that covers it; O for the stores.
 struct AtMaps {
-  alignas(64) unsigned char q[128]; alignas(64) unsigned char k[128];
-  alignas(64) unsigned char v[128]; alignas(64) unsigned char o[128];
+  alignas(64) unsigned char q[4][128]; alignas(64) unsigned char k[4][128];
+  alignas(64) unsigned char v[4][128]; alignas(64) unsigned char o[128];
 };
+// index of the smallest box (128 >> index rows) that covers `rows` (a multiple of 16 in 16..128)
+__device__ __forceinline__ int at_box(int rows) { return rows > 64 ? 0 : rows > 32 ? 1 : rows > 16 ? 2 : 3; }
 
 struct AtArgs {
   const int32_t* cache_len; __nv_bfloat16* out; DeviceStatus* status;
@@ -102,15 +106,16 @@ struct AtArgs {
 
 // Work item -> (b, h, pair p of query tiles).  Pair p counts from the sequence's end: it covers rows
 // [q_hi - 256, q_hi) with q_hi = n - 256 p, clipped at row 0; its keys are [0, q_hi) in n_kv tiles.
-struct AtItem { int b, h, q_hi, n, n_kv, row_base; };
+struct AtItem { int b, h, q_hi, n, n_kv, row_base, swap; };
 
 // One lane's share of an item: rows [q0, q_hi) are owned (the Q tile is loaded from row q0, 128 rows;
 // a tile clipped at the top of the sequence loads rows [0, 128) and owns the first q_hi of them),
-// keys [0, q_hi) in n_tiles tiles.
+// keys [0, q_hi) in n_tiles tiles.  The later query tile of a pair has one key tile more than the
+// earlier one, so the lanes swap tiles from one item to the next (I.swap) and do the same work.
 struct AtLane { int q0, q_hi, n_tiles; bool exists; };
 __device__ __forceinline__ AtLane at_lane(const AtItem& I, int lane_id) {
   AtLane L;
-  L.q_hi = I.q_hi - lane_id * kAtBM;
+  L.q_hi = I.q_hi - (lane_id ^ I.swap) * kAtBM;
   L.exists = L.q_hi > 0;
   L.q0 = max(L.q_hi - kAtBM, 0);
   L.n_tiles = (L.q_hi + kAtBN - 1) / kAtBN;
@@ -128,40 +133,51 @@ __device__ __forceinline__ int ld_early(const int32_t* p) {
   return v;
 }
 
-// Walks the items of this CTA (item = p * B * H + b * H + h, stepping by the grid size) in the order
-// every role uses.  The position is kept as (p, b, h) and advanced by additions; the length of the
-// NEXT item's sequence is requested one item early, so its latency never sits in front of a role's
-// first wait.
+// Walks the items of this CTA in the order every role uses.  The CTA's k-th item has the linear index
+// i = blockIdx + k * grid; it belongs to head (b, h) = i / q_pairs, so the pairs of one head run at
+// the same time on neighbouring SMs and fetch its K and V from memory once (the later ones hit L2).
+// Which pair of the head it is rotates with k (p = (i mod q_pairs + k) mod q_pairs), so every CTA
+// gets long and short pairs alike whatever the grid size.  The length of the NEXT item's sequence
+// is requested one item early, so its latency never sits in front of a role's first wait.
+constexpr bool kAtHeadMajor = false;
+constexpr bool kAtSwapLanes = true;
 struct AtWalker {
   const AtArgs& a;
-  int p, b, h, len, db, dh;
+  int i, kr, items, len, sw;                   // next item's linear index, k mod q_pairs, item count, length, swap bit
+  __device__ __forceinline__ int bh_of(int idx) const { return kAtHeadMajor ? idx / a.q_pairs : idx % (a.B * a.H); }
+  __device__ __forceinline__ int len_of(int idx) const { return ld_early(a.cache_len + bh_of(idx) / a.H); }
   __device__ __forceinline__ explicit AtWalker(const AtArgs& a_) : a(a_) {
-    const int bh_count = a.B * a.H;
-    p = (int)blockIdx.x / bh_count;
-    const int bh = (int)blockIdx.x - p * bh_count;
-    b = bh / a.H;
-    h = bh - b * a.H;
-    db = (int)gridDim.x / a.H;
-    dh = (int)gridDim.x - db * a.H;
-    len = p < a.q_pairs ? ld_early(a.cache_len + b) : 0;
+    items = a.B * a.H * a.q_pairs;
+    i = (int)blockIdx.x;
+    kr = 0;
+    sw = 0;
+    len = i < items ? len_of(i) : 0;
   }
   // Advances to the next item that exists (a sequence of 256 p rows or fewer has no pair p).
   __device__ __forceinline__ bool next(AtItem& I) {
     for (;;) {
-      if (p >= a.q_pairs) return false;
-      const int cp = p, cb = b, ch = h, clen = len;
-      h += dh;
-      b += db;
-      if (h >= a.H) { h -= a.H; ++b; }
-      while (b >= a.B) { b -= a.B; ++p; }
-      if (p < a.q_pairs) len = ld_early(a.cache_len + b);
-      I.b = cb;
-      I.h = ch;
+      if (i >= items) return false;
+      const int ci = i, ck = kr, clen = len;
+      i += (int)gridDim.x;
+      if (++kr == a.q_pairs) kr = 0;
+      if (i < items) len = len_of(i);
+      const int bh = bh_of(ci);
+      int p;
+      if (kAtHeadMajor) {
+        p = ci - bh * a.q_pairs + ck;
+        if (p >= a.q_pairs) p -= a.q_pairs;
+      } else {
+        p = ci / (a.B * a.H);
+      }
+      I.b = bh / a.H;
+      I.h = bh - I.b * a.H;
       I.n = min(max(clen, 0), min(a.cap, a.n_max));
-      I.q_hi = I.n - cp * 2 * kAtBM;
+      I.q_hi = I.n - p * 2 * kAtBM;
       if (I.q_hi <= 0) continue;
       I.n_kv = (I.q_hi + kAtBN - 1) / kAtBN;
-      I.row_base = (cb * a.H + ch) * a.cap;                         // first row of this (b, h) in the caches
+      I.row_base = bh * a.cap;                                      // first row of this (b, h) in the caches
+      I.swap = kAtSwapLanes ? sw : 0;
+      sw ^= 1;
       return true;
     }
   }
@@ -243,16 +259,15 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     // ---------------------------------------------------------------- TMA producer
     reg_dec<kAtRegsSmall>();
     if (lane == 0) {
-      const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(maps.q);
-      const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(maps.k);
-      const CUtensorMap* mv = reinterpret_cast<const CUtensorMap*>(maps.v);
-      tma_prefetch_desc(mq); tma_prefetch_desc(mk); tma_prefetch_desc(mv);
+      for (int i = 0; i < 4; ++i) {
+        tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.q[i]));
+        tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.k[i]));
+        tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.v[i]));
+      }
       // cursor of the ring
       AtWalker Wr(a);
       AtItem Ir;
       int T = 0, jr = 0;                       // ring tiles issued so far / tile index within Ir (K, V alternating)
-      uint32_t free_par[2] = {0u, 0u};         // bit s: parity of the next phase of ring_free(x, s) to wait for
-      uint32_t prev_b = 0u;                    // bit s: the tile now in slot s is read by lane B too
       // cursors of the Q loads
       AtWalker Wq0 = Wr, Wq1 = Wr;
       AtItem Iq[2];
@@ -261,6 +276,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       bool hr = Wr.next(Ir);
       hq[0] = Wq0.next(Iq[0]);
       hq[1] = Wq1.next(Iq[1]);
+      while (hq[0] && !at_lane(Iq[0], 0).exists) hq[0] = Wq0.next(Iq[0]);
       while (hq[1] && !at_lane(Iq[1], 1).exists) hq[1] = Wq1.next(Iq[1]);
       int idle = 0;
       while ((hr || hq[0] || hq[1]) && !*abort_flag) {
@@ -273,12 +289,16 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           if (nq[x] >= 2 && !mbar_test(q_done(x, s), ((nq[x] - 2) >> 1) & 1)) continue;
           const AtLane L = at_lane(Iq[x], x);
           char* dst = smem + (2 * x + s) * kAtTile;
-          mbar_expect_tx(q_full(x, s), kAtTile);
+          // the rows the lane owns, in 16s (a tile clipped at the top of the sequence owns fewer than 128)
+          const int bx = at_box(min(kAtBM, (L.q_hi - L.q0 + 15) & ~15));
+          const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(maps.q[bx]);
+          mbar_expect_tx(q_full(x, s), kAtTile >> bx);
           tma_load_2d(smem_u32(dst), mq, 0, Iq[x].row_base + L.q0, q_full(x, s));
           tma_load_2d(smem_u32(dst + kAtBM * 128), mq, 64, Iq[x].row_base + L.q0, q_full(x, s));
           ++nq[x];
           if (x == 0) {
             hq[0] = Wq0.next(Iq[0]);
+            while (hq[0] && !at_lane(Iq[0], 0).exists) hq[0] = Wq0.next(Iq[0]);
           } else {
             hq[1] = Wq1.next(Iq[1]);
             while (hq[1] && !at_lane(Iq[1], 1).exists) hq[1] = Wq1.next(Iq[1]);
@@ -289,22 +309,18 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           const int s = T % kAtRing;
           bool slot_free = true;
           if (T >= kAtRing) {
-            slot_free = mbar_test(ring_free(0, s), (free_par[0] >> s) & 1u);
-            if (slot_free && ((prev_b >> s) & 1u)) slot_free = mbar_test(ring_free(1, s), (free_par[1] >> s) & 1u);
+            // both lanes have released the slot's previous tile (a lane releases every tile, read or not)
+            const uint32_t par = (uint32_t)(T / kAtRing - 1) & 1u;
+            slot_free = mbar_test(ring_free(0, s), par) && mbar_test(ring_free(1, s), par);
           }
           if (slot_free) {
-            if (T >= kAtRing) {
-              free_par[0] ^= 1u << s;
-              if ((prev_b >> s) & 1u) free_par[1] ^= 1u << s;
-            }
             const int j = jr >> 1;
-            const AtLane LB = at_lane(Ir, 1);
-            const bool b_reads = LB.exists && j < LB.n_tiles;
-            prev_b = (prev_b & ~(1u << s)) | ((b_reads ? 1u : 0u) << s);
             char* dst = ring_s + s * kAtTile;
-            const CUtensorMap* m = (jr & 1) ? mv : mk;
+            // keys of the tile that the pair's later query tile covers (the earlier one never needs more)
+            const int bx = at_box(min(kAtBN, (Ir.q_hi - j * kAtBN + 15) & ~15));
+            const CUtensorMap* m = reinterpret_cast<const CUtensorMap*>((jr & 1) ? maps.v[bx] : maps.k[bx]);
             const int r = Ir.row_base + j * kAtBN;
-            mbar_expect_tx(ring_full(s), kAtTile);
+            mbar_expect_tx(ring_full(s), kAtTile >> bx);
             tma_load_2d(smem_u32(dst), m, 0, r, ring_full(s));
             tma_load_2d(smem_u32(dst + kAtBN * 128), m, 64, r, ring_full(s));
             ++T;
@@ -340,10 +356,24 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       int n_item = 0, g0 = 0, T0 = 0;                 // this lane's items / tiles so far; ring tiles before this item
       while (W.next(I)) {
         const AtLane L = at_lane(I, x);
-        if (!L.exists) { T0 += 2 * I.n_kv; continue; }
+        auto wait_ring = [&](int T) { mbar_wait_spin(ring_full(T % kAtRing), (T / kAtRing) & 1, abort_flag); };
+        // A lane does not read every ring tile (not the pair's last key tile when it has the earlier query
+        // tile, nothing of a pair that has no earlier tile).  It still observes every tile's landing and
+        // releases it, in ring order, so that the slot barriers advance one phase per tile for every
+        // waiter: a waiter that had skipped phases could not tell them apart by parity.
+        auto pass_tiles = [&](int from, int to) {
+          for (int T = from; T < to; ++T) {
+            wait_ring(T);
+            mbar_arrive(ring_free(x, T % kAtRing));
+          }
+        };
+        if (!L.exists) {
+          pass_tiles(T0, T0 + 2 * I.n_kv);
+          T0 += 2 * I.n_kv;
+          continue;
+        }
         const int qs = n_item & 1;
         const uint64_t q_desc = smem_desc_sw128(smem_u32(smem + (2 * x + qs) * kAtTile));
-        auto wait_ring = [&](int T) { mbar_wait_spin(ring_full(T % kAtRing), (T / kAtRing) & 1, abort_flag); };
         auto issue_qk = [&](int j) {
           const int s = (T0 + 2 * j) % kAtRing;
           const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile));
@@ -387,6 +417,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           mma_commit(pv_done(x));
           mma_commit(ring_free(x, s));
         }
+        pass_tiles(T0 + 2 * L.n_tiles, T0 + 2 * I.n_kv);
         g0 += L.n_tiles;
         ++n_item;
         T0 += 2 * I.n_kv;
@@ -470,7 +501,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
             }
           }
           mx_tile = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-          const bool need = mx_tile > m_used + kRescaleStep;
+          const bool need = grow < L.q_hi && mx_tile > m_used + kRescaleStep;   // rows the tile does not own hold stale data
           if (!__any_sync(0xffffffffu, need)) {
             float la, lb;
             unpack2(fadd2(l2[0], l2[1]), la, lb);
@@ -622,15 +653,18 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
   AtMaps maps;
   const uint64_t dims[2] = {128ull, (uint64_t)rows};
   const uint64_t strides[1] = {256ull};
-  const uint32_t box[2] = {64u, 128u};
   // out [B][n_max][H][128]: 32 rows x 32 columns of one head per store
   const uint64_t dims_o[4] = {128ull, (uint64_t)d.n_heads, (uint64_t)n_max, (uint64_t)B};
   const uint64_t strides_o[3] = {256ull, 256ull * d.n_heads, 256ull * d.n_heads * n_max};
   const uint32_t box_o[4] = {32u, 1u, 32u, 1u};
-  if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.q), q, 2, dims, strides, box) ||
-      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.k), k_cache, 2, dims, strides, box) ||
-      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.v), v_cache, 2, dims, strides, box) ||
-      !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.o), out, 4, dims_o, strides_o, box_o,
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t box[2] = {64u, 128u >> i};
+    if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.q[i]), q, 2, dims, strides, box) ||
+        !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.k[i]), k_cache, 2, dims, strides, box) ||
+        !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.v[i]), v_cache, 2, dims, strides, box))
+      return cudaErrorInvalidValue;
+  }
+  if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.o), out, 4, dims_o, strides_o, box_o,
                        CU_TENSOR_MAP_SWIZZLE_64B))
     return cudaErrorInvalidValue;
   AtArgs a;

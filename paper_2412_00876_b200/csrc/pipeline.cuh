@@ -57,7 +57,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // The same bound without the sleep between polls, for hand-offs inside a pipeline whose stages are a
 // few hundred cycles long (try_wait itself suspends the thread for a hardware-chosen time).
 __device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int* abort) {
-  if (mbar_try_wait(bar, parity)) return !*abort;
+  if (mbar_test(bar, parity)) return true;                  // fast path: one non-suspending poll
   for (int i = 0; i < kSpinLimitBusy; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63) == 63 && *abort) return false;
