@@ -16,9 +16,9 @@ int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_
   const int64_t o_status = take(sizeof(DeviceStatus));
   const int64_t o_pbase = take((int64_t)max_batch * 4);
   const int64_t o_pcount = take((int64_t)max_batch * 4);
-  const int64_t o_ticket = take((int64_t)max_batch * d.n_heads * 4);
+  const int64_t o_ticket = take((int64_t)2 * max_batch * d.n_heads * 4);
   const int32_t slots = (cap + kDecodeMinChunk - 1) / kDecodeMinChunk + 1;
-  const int64_t o_partial = take((int64_t)max_batch * d.n_heads * slots * (d.head_dim + 2) * 4);
+  const int64_t o_partial = take((int64_t)2 * max_batch * d.n_heads * slots * (d.head_dim + 2) * 4);
   const int32_t rows_pad = (max_rows + kPredRowTile - 1) / kPredRowTile * kPredRowTile;
   const int64_t o_ppart = take((int64_t)kPredMaxSplit * rows_pad * 4);
   const int64_t o_ptick = take((int64_t)(rows_pad / kPredRowTile + 1) * 4);
@@ -129,7 +129,7 @@ int32_t dl_set_workspace(dl_ctx* ctx, void* dev_ptr, int64_t bytes, int32_t max_
   workspace_layout(ctx->desc, max_batch, max_rows, cap, &ctx->ws);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemsetAsync(ctx->ws.status, 0, sizeof(DeviceStatus), s);
-  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.dec_ticket, 0, (size_t)max_batch * ctx->desc.n_heads * 4, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.dec_ticket, 0, (size_t)2 * max_batch * ctx->desc.n_heads * 4, s);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ctx->ws.pred_ticket, 0, (size_t)(ctx->ws.pred_rows_padded / kPredRowTile + 1) * 4, s);
   return cuda_status(ctx, e);
@@ -250,7 +250,7 @@ int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, 
 // caches and outputs are distinct tensors).
 static int32_t decode_layer(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
                             void* v_cache, const int32_t* cache_len, const uint8_t* keep, int32_t B,
-                            int32_t cap, float scale, void* out, bool overlap_prev, void* stream) {
+                            int32_t cap, float scale, void* out, bool overlap_prev, int scratch_set, void* stream) {
   if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
   if (B == 0) return DL_OK;
   if (!q_t || !k_t || !v_t || !k_cache || !v_cache || !cache_len || !out) return DL_ERR_INVALID_ARG;
@@ -261,13 +261,13 @@ static int32_t decode_layer(dl_ctx* ctx, const void* q_t, const void* k_t, const
   if (B > 2048) return DL_ERR_UNSUPPORTED;
   DeviceGuard g(ctx->device);
   return cuda_status(ctx, launch_attn_decode(ctx, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, B, cap,
-                                             scale, out, overlap_prev, static_cast<cudaStream_t>(stream)));
+                                             scale, out, overlap_prev, scratch_set, static_cast<cudaStream_t>(stream)));
 }
 
 int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
                               void* v_cache, const int32_t* cache_len, const uint8_t* keep, int32_t B,
                               int32_t cap, float scale, void* out, void* stream) {
-  return decode_layer(ctx, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, B, cap, scale, out, false, stream);
+  return decode_layer(ctx, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, B, cap, scale, out, false, 0, stream);
 }
 
 int32_t dl_decode_keep(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
@@ -326,7 +326,7 @@ int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, co
     // consecutive layers touch different caches and outputs, so layer l may start while layer l-1 drains
     const bool overlap = l > 0 && k_caches[l] != k_caches[l - 1] && v_caches[l] != v_caches[l - 1];
     int32_t st = decode_layer(ctx, ql, kl, vl, k_caches[l], v_caches[l], cache_len, keep, B, cap, scale, ol, overlap,
-                              stream);
+                              l & 1, stream);
     if (st != DL_OK) return st;
   }
   return DL_OK;

@@ -822,19 +822,27 @@ static int scratch_slots(const DecodeArgs& a) { return max_chunks(a) + 1; }
 cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t,
                                void* k_cache, void* v_cache, const int32_t* cache_len,
                                const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                               bool overlap_prev, cudaStream_t s) {
+                               bool overlap_prev, int scratch_set, cudaStream_t s) {
   if (B == 0) return cudaSuccess;
   if (B > kMaxDecodeBatch) return cudaErrorInvalidValue;
   const dl_model_desc& d = ctx->desc;
   DecodeArgs a;
   a.q = q; a.k_t = k_t; a.v_t = v_t; a.k_cache = k_cache; a.v_cache = v_cache;
   a.cache_len = cache_len; a.keep = keep; a.out = out;
-  a.partial = ctx->ws.dec_partial; a.ticket = ctx->ws.dec_ticket; a.status = ctx->ws.status;
+  a.status = ctx->ws.status;
   a.B = B; a.H = d.n_heads; a.cap = cap;
   pick_split(ctx, a);
   a.slots = ctx->ws.dec_slots;
-  // overlapping launches share the split scratch, so only unsplit launches may overlap
-  a.overlap = (overlap_prev && max_chunks(a) == 1) ? 1 : 0;
+  // the scratch of split sequences: two sets, so that a launch and the one that may overlap it differ
+  const size_t set = (size_t)(scratch_set & 1);
+  a.ticket = ctx->ws.dec_ticket + set * (size_t)ctx->ws.max_batch * d.n_heads;
+  a.partial = ctx->ws.dec_partial + set * (size_t)ctx->ws.max_batch * d.n_heads * ctx->ws.dec_slots * (d.head_dim + 2);
+  // A launch may overlap its predecessor if it is unsplit (no scratch), or if the grid fills every CTA
+  // slot of the GPU: then the predecessor's CTAs, which stay until the launch before them has completed,
+  // hold all the slots, and no launch can start before the one two back, which shares its scratch set,
+  // is done.
+  const long long full_grid = (long long)ctx->sm_count * kMmaCtas;
+  a.overlap = (overlap_prev && (max_chunks(a) == 1 || (long long)B * d.n_heads * max_chunks(a) >= full_grid)) ? 1 : 0;
   a.n_stages = 0;
   a.scale_log2 = scale * 1.4426950408889634f;
   if (d.dtype == DL_BF16) {

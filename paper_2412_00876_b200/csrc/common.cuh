@@ -45,8 +45,9 @@ struct Workspace {
   DeviceStatus* status = nullptr;
   int32_t* plan_base = nullptr;       // [max_batch] compaction: first destination row
   int32_t* plan_count = nullptr;      // [max_batch] compaction: rows to append (-1: skip sequence)
-  int32_t* dec_ticket = nullptr;      // [max_batch * H] decode: arrivals per (b,h); zero between launches
-  float* dec_partial = nullptr;       // [max_batch * H * dec_slots * (D + 2)]
+  // decode scratch, two sets: launches that overlap in time (consecutive layers of a stack) alternate
+  int32_t* dec_ticket = nullptr;      // [2][max_batch * H] arrivals per (b,h); zero between launches
+  float* dec_partial = nullptr;       // [2][max_batch * H * dec_slots * (D + 2)]
   int32_t dec_slots = 0;              // partial slots per (b,h)
   float* pred_partial = nullptr;      // [kPredMaxSplit][max_rows padded to kPredRowTile]
   int32_t* pred_ticket = nullptr;     // [row tiles]; zero between launches
@@ -117,7 +118,7 @@ cudaError_t launch_commit_len(const uint8_t* keep, int32_t B, int32_t cap, int32
 cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t,
                                void* k_cache, void* v_cache, const int32_t* cache_len,
                                const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                               bool overlap_prev, cudaStream_t s);
+                               bool overlap_prev, int scratch_set, cudaStream_t s);
 
 cudaError_t launch_predictor_simt(const dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows,
                                   float* score, cudaStream_t s);
