@@ -16,9 +16,9 @@ int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_
   const int64_t o_status = take(sizeof(DeviceStatus));
   const int64_t o_pbase = take((int64_t)max_batch * 4);
   const int64_t o_pcount = take((int64_t)max_batch * 4);
-  const int64_t o_ticket = take((int64_t)2 * max_batch * d.n_heads * 4);
+  const int64_t o_ticket = take((int64_t)kDecodeScratchSets * max_batch * d.n_heads * 4);
   const int32_t slots = (cap + kDecodeMinChunk - 1) / kDecodeMinChunk + 1;
-  const int64_t o_partial = take((int64_t)2 * max_batch * d.n_heads * slots * (d.head_dim + 2) * 4);
+  const int64_t o_partial = take((int64_t)kDecodeScratchSets * max_batch * d.n_heads * slots * (d.head_dim + 2) * 4);
   const int32_t rows_pad = (max_rows + kPredRowTile - 1) / kPredRowTile * kPredRowTile;
   const int64_t o_ppart = take((int64_t)kPredMaxSplit * rows_pad * 4);
   const int64_t o_ptick = take((int64_t)(rows_pad / kPredRowTile + 1) * 4);
@@ -129,7 +129,8 @@ int32_t dl_set_workspace(dl_ctx* ctx, void* dev_ptr, int64_t bytes, int32_t max_
   workspace_layout(ctx->desc, max_batch, max_rows, cap, &ctx->ws);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemsetAsync(ctx->ws.status, 0, sizeof(DeviceStatus), s);
-  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.dec_ticket, 0, (size_t)2 * max_batch * ctx->desc.n_heads * 4, s);
+  if (e == cudaSuccess)
+    e = cudaMemsetAsync(ctx->ws.dec_ticket, 0, (size_t)kDecodeScratchSets * max_batch * ctx->desc.n_heads * 4, s);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ctx->ws.pred_ticket, 0, (size_t)(ctx->ws.pred_rows_padded / kPredRowTile + 1) * 4, s);
   return cuda_status(ctx, e);
@@ -318,6 +319,7 @@ int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, co
   if (B == 0 || L == 0) return DL_OK;
   if (!k_caches || !v_caches || !q_t || !k_t || !v_t || !out) return DL_ERR_INVALID_ARG;
   const size_t layer_bytes = (size_t)B * ctx->desc.n_heads * ctx->desc.head_dim * elt_bytes(ctx);
+  ctx->opt.in_layer_stack = L > 1 ? 1 : 0;
   for (int32_t l = 0; l < L; ++l) {
     const char* ql = static_cast<const char*>(q_t) + l * layer_bytes;
     const char* kl = static_cast<const char*>(k_t) + l * layer_bytes;
@@ -326,9 +328,10 @@ int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, co
     // consecutive layers touch different caches and outputs, so layer l may start while layer l-1 drains
     const bool overlap = l > 0 && k_caches[l] != k_caches[l - 1] && v_caches[l] != v_caches[l - 1];
     int32_t st = decode_layer(ctx, ql, kl, vl, k_caches[l], v_caches[l], cache_len, keep, B, cap, scale, ol, overlap,
-                              l & 1, stream);
-    if (st != DL_OK) return st;
+                              l % kDecodeScratchSets, stream);
+    if (st != DL_OK) { ctx->opt.in_layer_stack = 0; return st; }
   }
+  ctx->opt.in_layer_stack = 0;
   return DL_OK;
 }
 

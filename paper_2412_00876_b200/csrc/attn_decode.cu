@@ -86,6 +86,7 @@ struct DecodeArgs {
   float* partial; int32_t* ticket; DeviceStatus* status;
   int32_t B, H, cap, chunk, per_bh, slots, n_stages;
   int32_t overlap;        // launched with programmatic stream serialisation (see launch_mma)
+  int32_t one_slot;       // host only: one CTA per SM (see launch_attn_decode)
   float scale_log2;
 };
 
@@ -782,7 +783,7 @@ static cudaError_t launch_mma(const dl_ctx* ctx, DecodeArgs& a, cudaStream_t s) 
     attr_set_for = (int)smem;
   }
   const long long max_items = (long long)a.B * a.H * max_chunks(a);
-  const int grid = (int)max(1LL, min((long long)ctx->sm_count * kMmaCtas, max_items));
+  const int grid = (int)max(1LL, min((long long)ctx->sm_count * (a.one_slot ? 1 : kMmaCtas), max_items));
   if (!a.overlap) {
     attn_decode_mma_kernel<<<grid, kMmaWarps * 32, smem, s>>>(maps, a);
     return cudaGetLastError();
@@ -833,16 +834,21 @@ cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t
   a.B = B; a.H = d.n_heads; a.cap = cap;
   pick_split(ctx, a);
   a.slots = ctx->ws.dec_slots;
-  // the scratch of split sequences: two sets, so that a launch and the one that may overlap it differ
-  const size_t set = (size_t)(scratch_set & 1);
+  // the scratch of split sequences: one of three sets, so that launches in flight together differ
+  const size_t set = (size_t)(scratch_set % kDecodeScratchSets);
   a.ticket = ctx->ws.dec_ticket + set * (size_t)ctx->ws.max_batch * d.n_heads;
   a.partial = ctx->ws.dec_partial + set * (size_t)ctx->ws.max_batch * d.n_heads * ctx->ws.dec_slots * (d.head_dim + 2);
-  // A launch may overlap its predecessor if it is unsplit (no scratch), or if the grid fills every CTA
-  // slot of the GPU: then the predecessor's CTAs, which stay until the launch before them has completed,
-  // hold all the slots, and no launch can start before the one two back, which shares its scratch set,
-  // is done.
-  const long long full_grid = (long long)ctx->sm_count * kMmaCtas;
-  a.overlap = (overlap_prev && (max_chunks(a) == 1 || (long long)B * d.n_heads * max_chunks(a) >= full_grid)) ? 1 : 0;
+  // Inside a layer stack a launch takes ONE CTA slot per SM (where the GPU has two): the next layer's
+  // launch, which may start as soon as this one has, takes the other, so two layers stream side by side
+  // and a layer's start-up and tail are covered by its neighbour's traffic.  How many layers can be in
+  // flight: a CTA of layer l+1 stays until layer l has completed (its grid-dependency wait), so the
+  // first sm_count CTAs to leave are layer l's; layer l+2 has started everywhere only once they have
+  // left, and layer l+3 cannot start before that.  So at most layers l, l+1, l+2 overlap: three scratch sets.
+  // Outside a stack, or with fewer items than SMs, a launch uses both slots and overlaps its predecessor
+  // only if it needs no scratch.
+  const bool mma_path = d.dtype == DL_BF16 && d.head_dim == 128 && ctx->tmap_encode && ctx->opt.decode_impl != 1;
+  a.one_slot = (mma_path && ctx->opt.in_layer_stack && (long long)B * d.n_heads * max_chunks(a) >= ctx->sm_count) ? 1 : 0;
+  a.overlap = (overlap_prev && (max_chunks(a) == 1 || a.one_slot)) ? 1 : 0;
   a.n_stages = 0;
   a.scale_log2 = scale * 1.4426950408889634f;
   if (d.dtype == DL_BF16) {
@@ -910,6 +916,7 @@ extern "C" int32_t dl_sparse_attn_decode_static(dl_ctx* ctx, const void* q_t, co
   a.B = B; a.H = d.n_heads; a.cap = cap;
   pick_split(ctx, a);
   a.overlap = 0;
+  a.one_slot = 0;
   const int slots = scratch_slots(a);
   // layout inside the array: tickets [B*H] int32 (256-byte padded) | partials [B*H*slots*(D+2)] float
   const size_t ticket_bytes = ((size_t)B * d.n_heads * sizeof(int32_t) + 255) & ~size_t(255);

@@ -34,6 +34,7 @@ __device__ __forceinline__ void report_status(DeviceStatus* st, int32_t code, lo
 // Workspace layout (all offsets 256-byte aligned).
 // ---------------------------------------------------------------------------------------
 constexpr int kDecodeMinChunk = 64;   // smallest rows-per-item the decode kernel may be asked for
+constexpr int kDecodeScratchSets = 3; // decode scratch sets (see Workspace)
 constexpr int kPredMaxSplit = 80;     // most unit tiles of the predictor's hidden layer
 constexpr int kPredRowTile = 128;     // rows per predictor row tile (tensor-core kernel)
 
@@ -45,9 +46,9 @@ struct Workspace {
   DeviceStatus* status = nullptr;
   int32_t* plan_base = nullptr;       // [max_batch] compaction: first destination row
   int32_t* plan_count = nullptr;      // [max_batch] compaction: rows to append (-1: skip sequence)
-  // decode scratch, two sets: launches that overlap in time (consecutive layers of a stack) alternate
-  int32_t* dec_ticket = nullptr;      // [2][max_batch * H] arrivals per (b,h); zero between launches
-  float* dec_partial = nullptr;       // [2][max_batch * H * dec_slots * (D + 2)]
+  // decode scratch, three sets: up to three consecutive layers of a stack are in flight at a time
+  int32_t* dec_ticket = nullptr;      // [3][max_batch * H] arrivals per (b,h); zero between launches
+  float* dec_partial = nullptr;       // [3][max_batch * H * dec_slots * (D + 2)]
   int32_t dec_slots = 0;              // partial slots per (b,h)
   float* pred_partial = nullptr;      // [kPredMaxSplit][max_rows padded to kPredRowTile]
   int32_t* pred_ticket = nullptr;     // [row tiles]; zero between launches
@@ -62,6 +63,7 @@ struct Options {
   int32_t prefill_attn_impl = 0;
   int32_t decode_chunk = 0;
   int32_t decode_impl = 0;
+  int32_t in_layer_stack = 0;          // set by the layer-stack call around its launches (not a user option)
 };
 
 }  // namespace dl
