@@ -39,10 +39,17 @@ def test_invalid_arguments_are_refused_with_codes():
     ctx.close()
 
 
-def test_layer_stack_equals_per_layer_calls_and_is_reproducible():
+@pytest.mark.parametrize("B,H,L,cap", [
+    (32, 32, 3, 512),      # 1024 (b,h) pairs: unsplit launches, two layers side by side
+    (8, 32, 8, 1024),      # 256 pairs: every sequence split in four, more layers than scratch sets
+    (2, 32, 5, 2048),      # 64 pairs: fewer items per chunk than SMs in places, split, both CTA slots
+])
+def test_layer_stack_equals_per_layer_calls_and_is_reproducible(B, H, L, cap):
+    """A stack of layers issued as one call (launches that overlap on the GPU, sharing the split scratch in
+    rotation) gives bit for bit what separate per-layer calls give, every time."""
     from paper_2412_00876_b200 import binding as dl
     cfg = wl.CONFIGS[3]
-    B, H, D, L, cap = 32, 32, 128, 3, 512                  # 1024 (b,h) pairs: unsplit, overlapped launches
+    D = 128
     ctx = dl.Context(256, H, D, 64, torch.bfloat16, 0, max_batch=B, max_rows=B, cap=cap)
     mk = lambda s, shape, sub=0: wl.device_normal(cfg, s, shape, DEV, sub=sub)
     q, kt, vt = mk(wl.S_DEC_Q, (L, B, H, D)), mk(wl.S_DEC_K, (L, B, H, D)), mk(wl.S_DEC_V, (L, B, H, D))
@@ -52,7 +59,7 @@ def test_layer_stack_equals_per_layer_calls_and_is_reproducible():
     keep = torch.from_numpy((np.arange(B) % 3 != 0).astype(np.uint8)).to(DEV)
     scale = 1 / np.sqrt(D)
     results = []
-    for mode in ("per-layer", "stack", "stack"):
+    for mode in ("per-layer", "stack", "stack", "stack", "stack"):
         kc, vc = [t.clone() for t in base_k], [t.clone() for t in base_v]
         out = torch.zeros(L, B, H, D, dtype=torch.bfloat16, device=DEV)
         if mode == "per-layer":
