@@ -425,6 +425,7 @@ def main():
                 "config": {"workload": cfg.name, "B_per_gpu": cfg.B, "layers": cfg.n_layers, "n_vis": cfg.n_vis,
                            "k_vis": cfg.k_vis, "n_text": cfg.n_text, "n_gen": cfg.n_gen, "keep_rate": cfg.keep_rate,
                            "parallelism": f"batch-shards x{world}", "decode_steps_from_cuda_graphs": use_graphs,
+                           "layer_stack": "q/k/v of all layers of a step are inputs; launches of consecutive layers overlap",
                            "l2": "inputs larger than L2 (caches tens of GB; input pools > 126 MB)"},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
                 "clocks": clocks}

@@ -225,6 +225,25 @@ int32_t dl_decode_step_host(dl_ctx* ctx, const dl_predictor* p_txt, const void* 
                             void* const* v_caches, int32_t cap, int32_t* cache_len, float scale,
                             void* stream);
 
+/* n_steps decode steps fed from HOST buffers as a pipeline (Eq. 6, once per step): while step t
+ * computes, the inputs of step t+1 are copied in and the results of step t-1 are copied out, on
+ * two copy streams the context owns (created at the first call, with the events that order them;
+ * no device memory is allocated).  Same results as n_steps calls of dl_decode_step_host.
+ *   x_host, q_host, k_host, v_host, out_host, keep_host: HOST arrays of n_steps host pointers (the
+ *   buffers pinned for full copy speed; keep_host or its entries may be NULL); stage_x dev
+ *   [2][B][hidden]; stage_q, stage_k, stage_v, stage_out dev [2][L][B][H][D]; logit_dev dev [2][B];
+ *   keep_dev dev [2][B]: two staging sets, used in turn.  The compute runs on `stream`, behind what the
+ *   caller queued there; returns after all three streams have been synchronised.  A failed step ends
+ *   the sequence: its status is returned once the queued work has drained. */
+int32_t dl_decode_steps_host(dl_ctx* ctx, const dl_predictor* p_txt, int32_t n_steps, int32_t B,
+                             float threshold, int32_t L, const void* const* x_host,
+                             const void* const* q_host, const void* const* k_host,
+                             const void* const* v_host, void* const* out_host,
+                             uint8_t* const* keep_host, void* stage_x, void* stage_q, void* stage_k,
+                             void* stage_v, void* stage_out, float* logit_dev, uint8_t* keep_dev,
+                             void* const* k_caches, void* const* v_caches, int32_t cap,
+                             int32_t* cache_len, float scale, void* stream);
+
 /* ---- decode attention without any allocation ------------------------------------------- */
 
 /* Size of the library's built-in scratch array (bytes). */

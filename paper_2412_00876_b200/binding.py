@@ -26,6 +26,7 @@ EXPORTS = [
     "dl_topk_from_scores", "dl_prefill_select", "dl_compact_kv", "dl_sparse_attn_prefill",
     "dl_sparse_attn_decode", "dl_decode_keep", "dl_commit_len", "dl_decode_step", "dl_decode_step_host",
     "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers", "dl_decode_nocache_select",
+    "dl_decode_steps_host",
 ]
 
 
@@ -77,6 +78,9 @@ def lib() -> C.CDLL:
                                      C.POINTER(vp), i32, vp, f32, vp, vp]),
             "dl_decode_step_host": (i32, [vp, P, vp, i32, f32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                           vp, vp, C.POINTER(vp), C.POINTER(vp), i32, vp, f32, vp]),
+            "dl_decode_steps_host": (i32, [vp, P, i32, i32, f32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
+                                           C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp, vp, vp, vp, vp, vp, vp,
+                                           C.POINTER(vp), C.POINTER(vp), i32, vp, f32, vp]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -255,6 +259,21 @@ class Context:
                                          _ptr(keep_out), L, _ptr(q_t), _ptr(k_t), _ptr(v_t), k_ptrs, v_ptrs, cap,
                                          _ptr(cache_len), float(scale), _ptr(out), _stream(stream)),
                     "dl_decode_step")
+
+    def decode_steps_host(self, p: Predictor, x_hosts, q_hosts, k_hosts, v_hosts, out_hosts, keep_hosts, stage_x,
+                          stage_q, stage_k, stage_v, stage_out, logit_dev, keep_dev, k_ptrs, v_ptrs, L, cap,
+                          cache_len, scale, threshold=0.0, stream=None):
+        """len(x_hosts) decode steps fed from (pinned) host tensors, copies pipelined against the compute;
+        the staging tensors hold two sets each (leading dimension 2)."""
+        n = len(x_hosts)
+        B = logit_dev.shape[-1]
+        arr = lambda ts: (C.c_void_p * n)(*[(t.data_ptr() if t is not None else None) for t in ts])
+        keep_arr = arr(keep_hosts) if keep_hosts is not None else None
+        self._check(lib().dl_decode_steps_host(
+            self._h, C.byref(p.desc), n, B, float(threshold), L, arr(x_hosts), arr(q_hosts), arr(k_hosts),
+            arr(v_hosts), arr(out_hosts), keep_arr, _ptr(stage_x), _ptr(stage_q), _ptr(stage_k), _ptr(stage_v),
+            _ptr(stage_out), _ptr(logit_dev), _ptr(keep_dev), k_ptrs, v_ptrs, cap, _ptr(cache_len), float(scale),
+            _stream(stream)), "dl_decode_steps_host")
 
     def decode_step_host(self, p: Predictor, x_host, q_host, k_host, v_host, out_host, keep_host, stage_x,
                          stage_q, stage_k, stage_v, stage_out, logit_dev, keep_dev, k_ptrs, v_ptrs, L, cap,

@@ -107,6 +107,17 @@ int32_t dl_create(dl_ctx** out, int32_t device, const dl_model_desc* desc) {
 }
 
 int32_t dl_destroy(dl_ctx* ctx) {
+  if (ctx) {
+    DeviceGuard g(ctx->device);
+    if (ctx->h2d_stream) cudaStreamDestroy(ctx->h2d_stream);
+    if (ctx->d2h_stream) cudaStreamDestroy(ctx->d2h_stream);
+    for (int i = 0; i < 2; ++i) {
+      if (ctx->ev_in[i]) cudaEventDestroy(ctx->ev_in[i]);
+      if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
+      if (ctx->ev_out[i]) cudaEventDestroy(ctx->ev_out[i]);
+    }
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  }
   delete ctx;
   return DL_OK;
 }
@@ -376,6 +387,78 @@ int32_t dl_decode_step_host(dl_ctx* ctx, const dl_predictor* p_txt, const void* 
   if (lb) e = cudaMemcpyAsync(out_host, stage_out, lb, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess && keep_host) e = cudaMemcpyAsync(keep_host, keep_dev, (size_t)B, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  return cuda_status(ctx, e);
+}
+
+// Copy streams and events of the pipelined host-fed decode: made once per context.
+static cudaError_t host_pipeline_setup(dl_ctx* ctx) {
+  if (ctx->h2d_stream) return cudaSuccess;
+  cudaError_t e = cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking);
+  for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+    e = cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+  return e;
+}
+
+int32_t dl_decode_steps_host(dl_ctx* ctx, const dl_predictor* p_txt, int32_t n_steps, int32_t B, float threshold,
+                             int32_t L, const void* const* x_host, const void* const* q_host,
+                             const void* const* k_host, const void* const* v_host, void* const* out_host,
+                             uint8_t* const* keep_host, void* stage_x, void* stage_q, void* stage_k, void* stage_v,
+                             void* stage_out, float* logit_dev, uint8_t* keep_dev, void* const* k_caches,
+                             void* const* v_caches, int32_t cap, int32_t* cache_len, float scale, void* stream) {
+  if (!ctx || n_steps < 0 || L < 0 || B < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || n_steps == 0) return DL_OK;
+  if (!x_host || !stage_x || !logit_dev || !keep_dev) return DL_ERR_INVALID_ARG;
+  if (L > 0 && (!q_host || !k_host || !v_host || !out_host || !stage_q || !stage_k || !stage_v || !stage_out))
+    return DL_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaError_t e = host_pipeline_setup(ctx);
+  if (e != cudaSuccess) return cuda_status(ctx, e);
+  cudaStream_t s = static_cast<cudaStream_t>(stream), sin = ctx->h2d_stream, sout = ctx->d2h_stream;
+  const size_t xb = (size_t)B * ctx->desc.hidden * elt_bytes(ctx);
+  const size_t lb = (size_t)L * B * ctx->desc.n_heads * ctx->desc.head_dim * elt_bytes(ctx);
+  // the copy streams start behind whatever the caller has queued on `stream`
+  e = cudaEventRecord(ctx->ev_fork, s);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(sin, ctx->ev_fork, 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(sout, ctx->ev_fork, 0);
+  int32_t st = DL_OK;
+  for (int32_t t = 0; t < n_steps && e == cudaSuccess && st == DL_OK; ++t) {
+    const int set = t & 1;
+    char* sx = static_cast<char*>(stage_x) + set * xb;
+    char* sq = static_cast<char*>(stage_q) + set * lb;
+    char* sk = static_cast<char*>(stage_k) + set * lb;
+    char* sv = static_cast<char*>(stage_v) + set * lb;
+    char* so = static_cast<char*>(stage_out) + set * lb;
+    // inputs of step t into staging set `set`, once step t-2 has finished computing from it
+    if (t >= 2) e = cudaStreamWaitEvent(sin, ctx->ev_done[set], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sx, x_host[t], xb, cudaMemcpyHostToDevice, sin);
+    if (e == cudaSuccess && lb) e = cudaMemcpyAsync(sq, q_host[t], lb, cudaMemcpyHostToDevice, sin);
+    if (e == cudaSuccess && lb) e = cudaMemcpyAsync(sk, k_host[t], lb, cudaMemcpyHostToDevice, sin);
+    if (e == cudaSuccess && lb) e = cudaMemcpyAsync(sv, v_host[t], lb, cudaMemcpyHostToDevice, sin);
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_in[set], sin);
+    // the step itself, once its inputs have landed and step t-2's results have left the output staging
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ctx->ev_in[set], 0);
+    if (e == cudaSuccess && t >= 2) e = cudaStreamWaitEvent(s, ctx->ev_out[set], 0);
+    if (e != cudaSuccess) break;
+    st = dl_decode_step(ctx, p_txt, sx, B, threshold, logit_dev + (size_t)set * B, keep_dev + (size_t)set * B, L, sq,
+                        sk, sv, k_caches, v_caches, cap, cache_len, scale, so, stream);
+    if (st != DL_OK) break;
+    e = cudaEventRecord(ctx->ev_done[set], s);
+    // results of step t back to the host
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(sout, ctx->ev_done[set], 0);
+    if (e == cudaSuccess && lb) e = cudaMemcpyAsync(out_host[t], so, lb, cudaMemcpyDeviceToHost, sout);
+    if (e == cudaSuccess && keep_host && keep_host[t])
+      e = cudaMemcpyAsync(keep_host[t], keep_dev + (size_t)set * B, (size_t)B, cudaMemcpyDeviceToHost, sout);
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_out[set], sout);
+  }
+  // everything that was queued is waited for, also after an error (the staging buffers are the caller's)
+  cudaError_t e1 = cudaStreamSynchronize(sin), e2 = cudaStreamSynchronize(s), e3 = cudaStreamSynchronize(sout);
+  if (st != DL_OK) return st;
+  if (e == cudaSuccess) e = e1 != cudaSuccess ? e1 : (e2 != cudaSuccess ? e2 : e3);
   return cuda_status(ctx, e);
 }
 

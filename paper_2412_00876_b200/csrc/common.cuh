@@ -77,6 +77,10 @@ struct dl_ctx {
   int32_t smem_optin = 0;
   cudaError_t last_cuda = cudaSuccess;
   void* tmap_encode = nullptr;        // cuTensorMapEncodeTiled, resolved at create
+  // copy streams and events of the pipelined host-fed decode (dl_decode_steps_host), created on first use
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+  cudaEvent_t ev_fork = nullptr;
   // tensor maps of cache tensors seen before (decode attention); see attn_decode.cu
   static constexpr int kMapCache = 256;
   struct MapEntry { const void* base = nullptr; long long rows = 0; unsigned char map[128]; };

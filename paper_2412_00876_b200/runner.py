@@ -177,8 +177,13 @@ class BatchRunner:
         self.h_prefill_out = torch.empty_like(self.prefill_out, device="cpu").pin_memory()
         self.h_dec_out = torch.empty_like(self.dec_out, device="cpu").pin_memory()
         self.h_keep = torch.empty(self.cfg.B, dtype=torch.uint8).pin_memory()
-        self.s_x = torch.empty_like(self.x_dec[0])
-        self.s_q, self.s_k, self.s_v = (torch.empty_like(self.q_dec[0]) for _ in range(3))
+        # two staging sets each: the pipelined host-fed decode copies step t+1 in while step t computes
+        two = lambda t: torch.empty((2,) + tuple(t.shape), dtype=t.dtype, device=t.device)
+        self.s_x = two(self.x_dec[0])
+        self.s_q, self.s_k, self.s_v, self.s_out = (two(self.q_dec[0]) for _ in range(4))
+        self.s_logit, self.s_keep = two(self.logit), two(self.keep_t)
+        self.h_dec_out2 = [torch.empty_like(self.dec_out, device="cpu").pin_memory() for _ in range(2)]
+        self.h_keep2 = [torch.empty(self.cfg.B, dtype=torch.uint8).pin_memory() for _ in range(2)]
         self.s_qsrc, self.s_ksrc, self.s_vsrc = (torch.empty_like(self.q_src[0]) for _ in range(3))
         self.s_xvis = torch.empty_like(self.x_vis)
 
@@ -207,15 +212,21 @@ class BatchRunner:
                                     self.prefill_out)
             self.h_prefill_out.copy_(self.prefill_out, non_blocking=True)
             d2h += self.prefill_out.numel() * self.prefill_out.element_size()
-        per_step_in = (self.s_x.numel() + 3 * self.s_q.numel()) * self.s_x.element_size()
+        per_step_in = (self.s_x[0].numel() + 3 * self.s_q[0].numel()) * self.s_x.element_size()
         per_step_out = self.dec_out.numel() * self.dec_out.element_size() + c.B
-        for t in range(c.n_gen):
-            i = t % self.step_pool
-            ctx.decode_step_host(self.p_txt, self.h_x_dec[i], self.h_q_dec[i], self.h_k_dec[i], self.h_v_dec[i],
-                                 self.h_dec_out, self.h_keep, self.s_x, self.s_q, self.s_k, self.s_v, self.dec_out,
-                                 self.logit, self.keep_t, self.kp, self.vp, L, self.cap, self.cache_len, self.scale)
-            h2d += per_step_in
-            d2h += per_step_out
+        # the decode steps as one pipelined host-fed call per chunk of steps (results land in two host
+        # buffers in turn: a consumer would read step t's while step t+1 computes)
+        chunk = 64
+        for t0 in range(0, c.n_gen, chunk):
+            steps = range(t0, min(c.n_gen, t0 + chunk))
+            pool = [t % self.step_pool for t in steps]
+            ctx.decode_steps_host(self.p_txt, [self.h_x_dec[i] for i in pool], [self.h_q_dec[i] for i in pool],
+                                  [self.h_k_dec[i] for i in pool], [self.h_v_dec[i] for i in pool],
+                                  [self.h_dec_out2[t & 1] for t in steps], [self.h_keep2[t & 1] for t in steps],
+                                  self.s_x, self.s_q, self.s_k, self.s_v, self.s_out, self.s_logit, self.s_keep,
+                                  self.kp, self.vp, L, self.cap, self.cache_len, self.scale)
+            h2d += per_step_in * len(steps)
+            d2h += per_step_out * len(steps)
         return h2d, d2h
 
     def close(self):

@@ -78,3 +78,51 @@ def test_layer_stack_equals_per_layer_calls_and_is_reproducible(B, H, L, cap):
             assert torch.equal(vc[l].view(torch.int16), ref[2][l].view(torch.int16))
     assert ctx.device_status()[0] == 0
     ctx.close()
+
+
+def test_pipelined_host_fed_steps_equal_single_host_steps():
+    """dl_decode_steps_host (copies of step t+1 and t-1 overlapping the compute of step t) leaves the same
+    caches, lengths, outputs and keep flags as one dl_decode_step_host call per step."""
+    from paper_2412_00876_b200 import binding as dl
+    cfg = wl.CONFIGS[2]
+    B, H, D, L, cap, hidden, ph, n_steps = 4, 4, 128, 3, 128, 256, 64, 7
+    rng = np.random.default_rng(5)
+    w1 = torch.from_numpy(rng.normal(0, 0.05, (ph, hidden)).astype(np.float32)).to(torch.bfloat16).to(DEV)
+    pd = dl.Predictor(w1, torch.zeros(ph, device=DEV), torch.from_numpy(rng.normal(0, 0.5, ph).astype(np.float32)).to(DEV), 0.0)
+    pin = lambda t: t.cpu().pin_memory()
+    xs = [pin(torch.randn(B, hidden).to(torch.bfloat16)) for _ in range(n_steps)]
+    qs, ks, vs = ([pin(torch.randn(L, B, H, D).to(torch.bfloat16)) for _ in range(n_steps)] for _ in range(3))
+    base_k = [torch.randn(B, H, cap, D, device=DEV).to(torch.bfloat16) for _ in range(L)]
+    base_v = [torch.randn(B, H, cap, D, device=DEV).to(torch.bfloat16) for _ in range(L)]
+    scale = 1 / np.sqrt(D)
+    results = []
+    for mode in ("single", "pipelined"):
+        ctx = dl.Context(hidden, H, D, ph, torch.bfloat16, 0, max_batch=B, max_rows=B, cap=cap)
+        kc, vc = [t.clone() for t in base_k], [t.clone() for t in base_v]
+        kp, vp = ctx.pointer_array(kc), ctx.pointer_array(vc)
+        ln = torch.tensor([5, 0, 60, 100], dtype=torch.int32, device=DEV)
+        outs = [pin(torch.zeros(L, B, H, D, dtype=torch.bfloat16)) for _ in range(n_steps)]
+        keeps = [pin(torch.zeros(B, dtype=torch.uint8)) for _ in range(n_steps)]
+        two = lambda *shape, dt=torch.bfloat16: torch.empty((2,) + shape, dtype=dt, device=DEV)
+        sx, sq, sk, sv, so = two(B, hidden), two(L, B, H, D), two(L, B, H, D), two(L, B, H, D), two(L, B, H, D)
+        lg, kd = two(B, dt=torch.float32), two(B, dt=torch.uint8)
+        if mode == "single":
+            for t in range(n_steps):
+                ctx.decode_step_host(pd, xs[t], qs[t], ks[t], vs[t], outs[t], keeps[t], sx[0], sq[0], sk[0], sv[0],
+                                     so[0], lg[0], kd[0], kp, vp, L, cap, ln, scale)
+        else:
+            ctx.decode_steps_host(pd, xs, qs, ks, vs, outs, keeps, sx, sq, sk, sv, so, lg, kd, kp, vp, L, cap, ln, scale)
+        torch.cuda.synchronize()
+        assert ctx.device_status()[0] == 0
+        results.append((outs, keeps, kc, vc, ln.cpu()))
+        ctx.close()
+    a, b = results
+    assert any(int(k.sum()) not in (0, B) for k in a[1]), "keep flags should vary"
+    for t in range(n_steps):
+        assert torch.equal(a[0][t].view(torch.int16), b[0][t].view(torch.int16)), f"step {t} output"
+        assert torch.equal(a[1][t], b[1][t])
+    for l in range(L):
+        assert torch.equal(a[2][l].view(torch.int16), b[2][l].view(torch.int16))
+        assert torch.equal(a[3][l].view(torch.int16), b[3][l].view(torch.int16))
+    assert torch.equal(a[4], b[4])
+
