@@ -782,6 +782,21 @@ static cudaError_t launch_mma(const dl_ctx* ctx, DecodeArgs& a, cudaStream_t s) 
     if (e != cudaSuccess) return e;
     attr_set_for = (int)smem;
   }
+  // The one-slot mode of a layer stack counts on exactly kMmaCtas CTAs of this kernel fitting an SM (that
+  // bounds how many layers can be in flight, hence how many scratch sets are needed): checked once per
+  // device and shared-memory size; otherwise a launch takes all slots and overlaps only when unsplit.
+  static int occ_for[64], occ_val[64];
+  if (occ_for[ctx->device & 63] != (int)smem) {
+    int nb = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, attn_decode_mma_kernel, kMmaWarps * 32, smem);
+    if (e != cudaSuccess) return e;
+    occ_val[ctx->device & 63] = nb;
+    occ_for[ctx->device & 63] = (int)smem;
+  }
+  if (a.one_slot && occ_val[ctx->device & 63] != kMmaCtas) {
+    a.one_slot = 0;
+    a.overlap = (a.overlap && max_chunks(a) == 1) ? 1 : 0;
+  }
   const long long max_items = (long long)a.B * a.H * max_chunks(a);
   const int grid = (int)max(1LL, min((long long)ctx->sm_count * (a.one_slot ? 1 : kMmaCtas), max_items));
   if (!a.overlap) {
