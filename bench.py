@@ -44,6 +44,8 @@ def parse():
     ap.add_argument("--micro-layers", type=int, default=2, help="layers of cache / source held in --micro mode")
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
     ap.add_argument("--decode-chunk", type=int, default=0, help="--micro decode: rows per work item (0: library's choice)")
+    ap.add_argument("--prefill-impl", type=int, default=0,
+                    help="--micro prefill/nocache: 0 library's choice, 2 whole 128-key tiles, 3 64-key half tiles")
     return ap.parse_args()
 
 
@@ -65,6 +67,8 @@ def micro(args):
     ctx = dl.Context(cfg.hidden, H, D, cfg.pred_hidden, tdt, 0, max_batch=B, max_rows=rows, cap=cfg.cap)
     if args.decode_chunk:
         ctx.set_option(dl.DL_OPT_DECODE_CHUNK, args.decode_chunk)
+    if args.prefill_impl:
+        ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, args.prefill_impl)
     scale = 1.0 / float(np.sqrt(D))
     i32 = dict(dtype=torch.int32, device=dev)
     work, unit, calls = 0.0, "GB/s", []

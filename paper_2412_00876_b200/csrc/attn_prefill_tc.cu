@@ -205,8 +205,16 @@ constexpr int kAtRegsSmall = 72, kAtRegsSoftmax = 216;
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
+// SUB = 1: a lane works on whole 128-key tiles (one S buffer; softmax and MMAs of a lane alternate).
+// SUB = 2: a lane works on 64-key half tiles with two S buffers of 64 columns, so the Q K^T of the next
+// half tile runs while the softmax works on this one.  An MMA of N = 64 costs the tensor pipe as much as
+// one of N = 128, so this trades pipe time (and twice the hand-overs) for overlap; measured, it loses:
+// 447 against 481 TFLOP/s at 832 rows, 373 against 401 at ~1650.  Kept selectable, not the default.
+template <int SUB>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
+  constexpr int Wd = kAtBN / SUB;                      // keys per sub-tile = columns of one S buffer
+  constexpr int NCH = Wd / 32;                         // 32-column chunks per sub-tile
   extern __shared__ __align__(1024) char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (smem_u32(smem) & 1023u) {                        // the swizzled tiles need 1024-byte alignment
@@ -218,16 +226,18 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
   // Ring tile T of this CTA (running count over its items; K and V of key tile j of an item are tiles
   // base + 2j and base + 2j + 1) lives in slot T % 3 and completes phase (T / 3) & 1 of that slot's
   // `full` barrier; lane X's MMAs that read it complete a phase of the slot's `free_X` barrier.
-  // A lane's own barriers: its k-th tile completes phase k & 1 of s_full / p_full / pv_done; its i-th
-  // item completes phase i & 1 of o_free and phase (i >> 1) & 1 of q_full / q_done of Q slot i & 1.
+  // A lane's own barriers: its g-th sub-tile (running count) uses S buffer g % SUB and completes phase
+  // (g / SUB) & 1 of that buffer's s_full / p_full / pv_done (per buffer, so that a waiter is never two
+  // phases behind: before sub-tile g's S is ready, the P V of g - SUB has completed); its i-th item completes
+  // phase i & 1 of o_free and phase (i >> 1) & 1 of q_full / q_done of Q slot i & 1.
   auto ring_full = [&](int s) { return smem_u32(bars + s); };
   auto ring_free = [&](int x, int s) { return smem_u32(bars + 3 + 3 * x + s); };
   auto q_full = [&](int x, int s) { return smem_u32(bars + 9 + 2 * x + s); };    // Q tile has landed
   auto q_done = [&](int x, int s) { return smem_u32(bars + 13 + 2 * x + s); };   // Q slot may be refilled (4 warps)
-  auto s_full = [&](int x) { return smem_u32(bars + 17 + x); };   // Q K^T has completed: S ready
-  auto p_full = [&](int x) { return smem_u32(bars + 19 + x); };   // P is in tensor memory (4 warps)
-  auto pv_done = [&](int x) { return smem_u32(bars + 21 + x); };  // P V has completed: O at rest
-  auto o_free = [&](int x) { return smem_u32(bars + 23 + x); };   // the epilogue has read O (4 warps)
+  auto s_full = [&](int x, int b) { return smem_u32(bars + 17 + 2 * x + b); };   // Q K^T has completed: S ready
+  auto p_full = [&](int x, int b) { return smem_u32(bars + 21 + 2 * x + b); };   // P is in tensor memory (4 warps)
+  auto pv_done = [&](int x, int b) { return smem_u32(bars + 25 + 2 * x + b); };  // P V has completed: O at rest
+  auto o_free = [&](int x) { return smem_u32(bars + 29 + x); };   // the epilogue has read O (4 warps)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
   int* pipe_turn = reinterpret_cast<int*>(bars + 34);
@@ -242,9 +252,11 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     }
     for (int x = 0; x < 2; ++x) {
       for (int s = 0; s < 2; ++s) { mbar_init(q_full(x, s), 1); mbar_init(q_done(x, s), 4); }
-      mbar_init(s_full(x), 1);
-      mbar_init(p_full(x), 4);
-      mbar_init(pv_done(x), 1);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(s_full(x, b), 1);
+        mbar_init(p_full(x, b), 4);
+        mbar_init(pv_done(x, b), 1);
+      }
       mbar_init(o_free(x), 4);
     }
     fence_mbar_init();
@@ -374,21 +386,25 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         }
         const int qs = n_item & 1;
         const uint64_t q_desc = smem_desc_sw128(smem_u32(smem + (2 * x + qs) * kAtTile));
-        auto issue_qk = [&](int j) {
-          const int s = (T0 + 2 * j) % kAtRing;
-          const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile));
-          const uint32_t idesc_qk = idesc_bf16(kAtBM, (uint32_t)at_cols(L, j));
+        // Sub-tile u of the item covers keys [u Wd, u Wd + sub_cols(u)): it is half u % SUB of ring tile
+        // pair u / SUB and uses S buffer (g0 + u) % SUB.
+        const int n_sub = (L.q_hi + Wd - 1) / Wd;
+        auto sub_cols = [&](int u) { return min(Wd, (L.q_hi - u * Wd + 15) & ~15); };
+        auto issue_qk = [&](int u) {
+          const int s = (T0 + 2 * (u / SUB)) % kAtRing;
+          const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile) + (u % SUB) * (Wd * 128));
+          const uint32_t idesc_qk = idesc_bf16(kAtBM, (uint32_t)sub_cols(u));
+          const uint32_t d = t_s + ((g0 + u) % SUB) * Wd;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
-            mma_ss(t_s, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
+            mma_ss(d, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
                    k_desc + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
         };
-        // Completion signals are issued after the lock is released (each one holds the issuing thread
-        // for about as long as an MMA, and the other lane's block can run meanwhile); a commit covers
-        // every MMA this thread has issued so far.
-        auto commit_qk = [&](int j) {
-          mma_commit(s_full(x));                                       // first: the softmax warps wait on it
-          mma_commit(ring_free(x, (T0 + 2 * j) % kAtRing));
+        // Completion signals: a commit covers every MMA this thread has issued so far.  The K tile is
+        // released by the Q K^T of its last sub-tile.
+        auto commit_qk = [&](int u) {
+          mma_commit(s_full(x, (g0 + u) % SUB));                       // first: the softmax warps wait on it
+          if (u % SUB == SUB - 1 || u == n_sub - 1) mma_commit(ring_free(x, (T0 + 2 * (u / SUB)) % kAtRing));
         };
         mbar_wait_spin(q_full(x, qs), (n_item >> 1) & 1, abort_flag);
         wait_ring(T0);
@@ -397,28 +413,34 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         issue_qk(0);
         pipe_unlock(pipe_turn);
         commit_qk(0);
-        for (int j = 0; j < L.n_tiles; ++j) {
-          const int g = g0 + j;
-          const int T = T0 + 2 * j + 1, s = T % kAtRing;
+        if (SUB == 2 && n_sub > 1) {                                   // the second S buffer: same K tile
+          issue_qk(1);
+          commit_qk(1);
+        }
+        for (int u = 0; u < n_sub; ++u) {
+          const int g = g0 + u, b = g % SUB;
+          const int T = T0 + 2 * (u / SUB) + 1, s = T % kAtRing;       // the V tile of this sub-tile
+          const int un = u + SUB;                                      // the sub-tile whose Q K^T reuses this S buffer
           // operands first (they land long before), then the softmax's hand-over
           wait_ring(T);
-          if (j + 1 < L.n_tiles) wait_ring(T + 1);
-          if (j == 0) mbar_wait_spin(o_free(x), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
-          mbar_wait_spin(p_full(x), g & 1, abort_flag);
+          if (un < n_sub) wait_ring(T0 + 2 * (un / SUB));
+          if (u == 0) mbar_wait_spin(o_free(x), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
+          mbar_wait_spin(p_full(x, b), (g / SUB) & 1, abort_flag);
           tc_fence_after();
-          const uint64_t v_desc = smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128);
-          const int ksteps = at_cols(L, j) >> 4;
+          const uint64_t v_desc =
+              smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128) + (uint64_t)(((u % SUB) * Wd * 128) >> 4);
+          const int ksteps = sub_cols(u) >> 4;
           pipe_lock(pipe_turn, abort_flag);
           for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(t_o, t_s + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv, (j | ks) != 0);
-          if (j + 1 < L.n_tiles) issue_qk(j + 1);                      // overwrites P: in order behind the P V
+            mma_ts(t_o, t_s + b * Wd + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv, (u | ks) != 0);
+          if (un < n_sub) issue_qk(un);                                // overwrites P: in order behind the P V
           pipe_unlock(pipe_turn);
-          if (j + 1 < L.n_tiles) commit_qk(j + 1);
-          mma_commit(pv_done(x));
-          mma_commit(ring_free(x, s));
+          if (un < n_sub) commit_qk(un);
+          mma_commit(pv_done(x, b));
+          if (u % SUB == SUB - 1 || u == n_sub - 1) mma_commit(ring_free(x, s));
         }
         pass_tiles(T0 + 2 * L.n_tiles, T0 + 2 * I.n_kv);
-        g0 += L.n_tiles;
+        g0 += n_sub;
         ++n_item;
         T0 += 2 * I.n_kv;
       }
@@ -443,18 +465,20 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       const int grow = L.q0 + row;                                     // row within the sequence
       const int r0 = L.q0 + quad * 32;                                 // this warp's first row
       float m_used = -INFINITY, l_run = 0.f;
-      for (int j = 0; j < L.n_tiles; ++j) {
-        const int g = g0 + j;
-        const int c0 = j * kAtBN;
-        // 32-column chunks of this tile that some row of the warp may see
-        const int n_ch = min(4, (min(L.q_hi, r0 + 32) - c0 + 31) >> 5);
-        mbar_wait_spin(s_full(x), g & 1, abort_flag);
+      const int n_sub = (L.q_hi + Wd - 1) / Wd;
+      for (int u = 0; u < n_sub; ++u) {
+        const int g = g0 + u, sbuf = g % SUB;
+        const int c0 = u * Wd;
+        const uint32_t sa = s_addr + sbuf * Wd;                         // this sub-tile's S buffer
+        // 32-column chunks of this sub-tile that some row of the warp may see
+        const int n_ch = min(NCH, (min(L.q_hi, r0 + 32) - c0 + 31) >> 5);
+        mbar_wait_spin(s_full(x, sbuf), (g / SUB) & 1, abort_flag);
         tc_fence_after();
         // ---- one pass over the tile in 32-column chunks, the next chunk's load in flight while this one is
         // worked on.  Exponentials are taken against the maximum the row already uses (the first chunk's
         // own maximum on an item's first tile); the tile's true maximum is tracked alongside, and only if
         // it turns out more than 2^8 above the one used is the tile done again after rescaling O.
-        uint32_t pw[64];                                                // P of the row, bf16 pairs
+        uint32_t pw[16 * NCH];                                          // P of the row, bf16 pairs
         const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2);
         const int vis = grow - c0;                                      // columns 0..vis are visible to this row
         float mx_tile;
@@ -463,13 +487,13 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           uint32_t buf[2][32];
           float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}; // four independent chains
           uint64_t l2[2] = {0ull, 0ull};                                // two chains of packed row sums
-          if (n_ch > 0) tmem_ld32(s_addr, buf[0]);
+          if (n_ch > 0) tmem_ld32(sa, buf[0]);
           tmem_ld_wait();
 #pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
+          for (int cc = 0; cc < NCH; ++cc) {
             uint32_t* sr = buf[cc & 1];
             if (n_ch > cc) {
-              if (n_ch > cc + 1) tmem_ld32(s_addr + 32 * (cc + 1), buf[(cc + 1) & 1]);
+              if (n_ch > cc + 1) tmem_ld32(sa + 32 * (cc + 1), buf[(cc + 1) & 1]);
               if (c0 + 32 * cc + 31 > r0) {                             // the chunk reaches past the warp's first row
 #pragma unroll
                 for (int c = 0; c < 32; ++c)
@@ -481,7 +505,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
                 for (int u = 0; u < 4; ++u)
                   mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
               }
-              if (cc == 0 && j == 0 && first_try)                       // column 0 is visible to every row: finite
+              if (cc == 0 && u == 0 && first_try)                       // column 0 is visible to every row: finite
                 m_used = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
               const uint64_t nm2 = pack2(-m_used, -m_used);
 #pragma unroll
@@ -512,9 +536,9 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           first_try = false;
           const float corr = need ? fast_exp2(m_used - mx_tile) : 1.0f;
           if (need) m_used = mx_tile;
-          if (j > 0) {
-            // O must be at rest: the P V of the previous tile (it completed before this tile's Q K^T)
-            mbar_wait_spin(pv_done(x), (g - 1) & 1, abort_flag);
+          if (u > 0) {
+            // O must be at rest: the P V of the previous sub-tile
+            mbar_wait_spin(pv_done(x, (g - 1) % SUB), ((g - 1) / SUB) & 1, abort_flag);
             tc_fence_after();
             l_run *= corr;
             const uint64_t corr2 = pack2(corr, corr);
@@ -535,14 +559,15 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
             tmem_st_wait();
           }
         }
-        tmem_st32(s_addr, pw);                                         // P (bf16) over the first half of S
-        tmem_st32(s_addr + 32, pw + 32);
+        tmem_st32(sa, pw);                                             // P (bf16) over the first half of its S buffer
+        if (NCH == 4) tmem_st32(sa + 32, pw + 32 * (NCH / 4));
         tmem_st_wait();
-        if (j == L.n_tiles - 1 && L.q_hi == I.n) {
+        if (u == n_sub - 1 && L.q_hi == I.n) {
           // last tile of the sequence (only lane A of pair 0 gets here): the P V covers keys up to the next
           // multiple of 16; zero the V rows between the sequence's end and that bound (both 64-dim halves).
           // Other query tiles need nothing: rows past their end are the sequence's own and P is 0 there.
-          const int valid = I.n - c0, pad = at_cols(L, j) - valid;
+          const int j = u / SUB;                                       // in rows of the 128-key ring tile
+          const int valid = I.n - j * kAtBN, pad = at_cols(L, j) - valid;
           if (pad > 0) {
             const int T = T0 + 2 * j + 1, s = T % kAtRing;
             mbar_wait_spin(ring_full(s), (T / kAtRing) & 1, abort_flag);
@@ -556,7 +581,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(p_full(x));
+        if (lane == 0) mbar_arrive(p_full(x, sbuf));
         if (q_slot_held >= 0) {
           // the previous item's staged output has long been read: hand its Q slot back to the producer
           if (lane == 0) { bulk_wait_read<0>(); mbar_arrive(q_done(x, q_slot_held)); }
@@ -565,8 +590,8 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       }
       // ---- epilogue: O / l -> bf16 -> out[b][row][h][:], 32 columns at a time, staged in this warp's 8 KB of
       // the item's Q slot (16-byte units XOR-swizzled by row pair: the 64-byte swizzle of the tensor map)
-      const int gl = g0 + L.n_tiles - 1;
-      mbar_wait_spin(pv_done(x), gl & 1, abort_flag);
+      const int gl = g0 + n_sub - 1;
+      mbar_wait_spin(pv_done(x, gl % SUB), (gl / SUB) & 1, abort_flag);   // MMAs complete in order: all of O is in
       tc_fence_after();
       const float inv = 1.0f / l_run;
       const int rows_here = L.q_hi - r0;                               // owned rows among this warp's 32
@@ -624,7 +649,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       if (lane == 0) bulk_commit();
       __syncwarp();
       q_slot_held = qs;
-      g0 += L.n_tiles;
+      g0 += n_sub;
       ++n_item;
       T0 += 2 * I.n_kv;
     }
@@ -673,14 +698,19 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
   a.scale_log2 = scale * 1.4426950408889634f;
   static int attr_set[64];
   if (!attr_set[ctx->device & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
+    cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attn_prefill_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
     if (e != cudaSuccess) return e;
     attr_set[ctx->device & 63] = 1;
   }
   const long long items = (long long)B * d.n_heads * a.q_pairs;
   if (items >= (1LL << 31)) return cudaErrorInvalidValue;
   const int grid = (int)std::min<long long>(items, (long long)ctx->sm_count);
-  attn_prefill_tc_kernel<<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
+  // half tiles (two S buffers per lane) only on request (option value 3)
+  const bool halves = ctx->opt.prefill_attn_impl == 3;
+  if (halves) attn_prefill_tc_kernel<2><<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
+  else attn_prefill_tc_kernel<1><<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
   return cudaGetLastError();
 }
 

@@ -219,7 +219,7 @@ def _prefill_case(dtype, H, D, lens, amp=1.0):
         q, k = q * amp, k * amp
     scale = 1 / np.sqrt(D)
     n_max = max(lens)
-    for impl in (1, 2):
+    for impl in (1, 2, 3):                       # CUDA cores; tensor cores on whole tiles / on half tiles
         ctx = _ctx(dtype, H, D, B=B, cap=cap)
         ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, impl)
         out = torch.full((B, n_max, H, D), 7.0, dtype=wl.torch_dtype(dtype), device=DEV)
@@ -231,7 +231,7 @@ def _prefill_case(dtype, H, D, lens, amp=1.0):
         try:
             ctx.sparse_attn_prefill(qd, kd, vd, torch.tensor(lens, dtype=torch.int32, device=DEV), n_max, scale, out)
         except dl.DlError as e:
-            assert impl == 2 and e.code == dl.DL_ERR_UNSUPPORTED and not (dtype == "bf16" and D == 128)
+            assert impl >= 2 and e.code == dl.DL_ERR_UNSUPPORTED and not (dtype == "bf16" and D == 128)
             continue
         assert ctx.device_status()[0] == 0
         got = wl.from_torch(out)
