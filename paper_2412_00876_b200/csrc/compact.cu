@@ -35,6 +35,9 @@ compact_plan_kernel(const uint8_t* __restrict__ keep, int32_t keep_cols, const i
                     int32_t cap, int32_t* __restrict__ cache_len, int32_t commit,
                     int32_t* __restrict__ plan_base, int32_t* __restrict__ plan_count, DeviceStatus* st) {
   __shared__ int sh[8];
+  // the copy kernel behind this one may start now: it ranks its tile's tokens first and waits for this
+  // kernel's results (grid-dependency wait) only before it needs them
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int b = blockIdx.x;
   int tb = t_src ? t_src[b] : t_max;
   tb = max(0, min(tb, t_max));
@@ -73,7 +76,6 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
   __shared__ int tile_kept;
 
   const int b = blockIdx.y;
-  if (plan_count[b] <= 0) return;
   int tb = t_src ? t_src[b] : t_max;
   tb = max(0, min(tb, t_max));
   const int t0 = blockIdx.x * kTileTokens;
@@ -97,6 +99,9 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
     if (threadIdx.x == 0) tile_kept = __popc(m);
   }
   __syncthreads();
+  // launched with programmatic stream serialisation: the plan of this call is complete from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (plan_count[b] <= 0) return;
   const int nk = tile_kept;
   const int dst0 = plan_base[b] + before;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -143,10 +148,16 @@ cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_s
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   dim3 grid((t_src_max + kTileTokens - 1) / kTileTokens, B);
-  compact_copy_kernel<<<grid, kCopyThreads, 0, s>>>(
-      (const uint4*)k_src, (const uint4*)v_src, keep, keep_cols, t_src, t_src_max, (uint4*)k_cache, (uint4*)v_cache,
-      cap, d.n_heads, row_units, piece_units, ctx->ws.plan_base, ctx->ws.plan_count);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = dim3(kCopyThreads); cfg.dynamicSmemBytes = 0; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, compact_copy_kernel, (const uint4*)k_src, (const uint4*)v_src, keep, (int32_t)keep_cols,
+                            t_src, (int32_t)t_src_max, (uint4*)k_cache, (uint4*)v_cache, (int32_t)cap, (int32_t)d.n_heads,
+                            (int32_t)row_units, (int32_t)piece_units, (const int32_t*)ctx->ws.plan_base,
+                            (const int32_t*)ctx->ws.plan_count);
 }
 
 __global__ void commit_len_kernel(const uint8_t* __restrict__ keep, int32_t B, int32_t cap,
