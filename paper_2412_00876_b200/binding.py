@@ -19,6 +19,7 @@ DL_OK = 0
 DL_ERR_INVALID_ARG, DL_ERR_ALIGNMENT, DL_ERR_UNSUPPORTED, DL_ERR_WORKSPACE = -1, -2, -3, -4
 DL_ERR_CUDA, DL_ERR_CAPACITY, DL_ERR_TIMEOUT, DL_WARN_NAN = -5, -6, -7, 1
 DL_OPT_PREDICTOR_IMPL, DL_OPT_PREFILL_ATTN_IMPL, DL_OPT_DECODE_CHUNK, DL_OPT_DECODE_IMPL = 1, 2, 3, 4
+DL_OPT_COMPACT_IMPL = 5
 
 EXPORTS = [
     "dl_create", "dl_destroy", "dl_workspace_bytes", "dl_set_workspace", "dl_set_option",

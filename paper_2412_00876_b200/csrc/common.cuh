@@ -63,6 +63,7 @@ struct Options {
   int32_t prefill_attn_impl = 0;
   int32_t decode_chunk = 0;
   int32_t decode_impl = 0;
+  int32_t compact_impl = 0;            // 0 auto, 1 register-staged copy kernel, 2 bulk-copy kernel
   int32_t in_layer_stack = 0;          // set by the layer-stack call around its launches (not a user option)
 };
 

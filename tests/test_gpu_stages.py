@@ -98,6 +98,40 @@ def test_compaction_bit_exact(dtype, H, D):
     assert ctx.device_status()[0] == 0
 
 
+@pytest.mark.parametrize("impl", [1, 2])
+def test_compaction_does_not_read_a_stale_plan(impl):
+    """The copy kernel starts while the plan kernel of the same call still runs.  With the workspace holding
+    a hostile old plan (count -1 = skip the sequence) a copy that read the plan too early would leave rows
+    unwritten: both copy kernels, several calls in a row, on a grid large enough to start early."""
+    from paper_2412_00876_b200 import binding as dl
+    B, T, H, D, nv, cap = 16, 704, 32, 128, 576, 768
+    ctx = dl.Context(4096, H, D, 1024, torch.bfloat16, 0, max_batch=B, max_rows=B * nv, cap=cap)
+    ctx.set_option(dl.DL_OPT_COMPACT_IMPL, impl)
+    g = torch.Generator(device=DEV).manual_seed(7)
+    ks = torch.randn(B, T, H, D, device=DEV, generator=g).to(torch.bfloat16)
+    vs = torch.randn(B, T, H, D, device=DEV, generator=g).to(torch.bfloat16)
+    keep = (torch.rand(B, nv, device=DEV, generator=g) < 0.25).to(torch.uint8)
+    t_src = torch.full((B,), T, dtype=torch.int32, device=DEV)
+    for rep in range(4):
+        ctx._ws.fill_(0xFF)                                  # every plan word reads -1 until rewritten
+        base = (ctx._ws.data_ptr() + 255) // 256 * 256       # same memory set up again: status and tickets zeroed
+        n = dl.lib().dl_workspace_bytes(ctx._h, B, B * nv, cap)
+        assert dl.lib().dl_set_workspace(ctx._h, base, n, B, B * nv, cap, None) == 0
+        kc = torch.zeros(B, H, cap, D, dtype=torch.bfloat16, device=DEV)
+        vc = torch.zeros(B, H, cap, D, dtype=torch.bfloat16, device=DEV)
+        ln = torch.zeros(B, dtype=torch.int32, device=DEV)
+        ctx.compact_kv(ks, vs, keep, t_src, kc, vc, ln, commit=True)
+        torch.cuda.synchronize()
+        for b in range(B):
+            rows = torch.cat([torch.nonzero(keep[b]).flatten(), torch.arange(nv, T, device=DEV)])
+            assert int(ln[b]) == rows.numel()
+            for src, got in ((ks, kc), (vs, vc)):
+                ref = src[b, rows].permute(1, 0, 2)
+                assert torch.equal(ref.view(torch.int16), got[b, :, : rows.numel()].view(torch.int16)), (rep, b)
+        assert ctx.device_status()[0] == 0
+    ctx.close()
+
+
 def test_compaction_keep_all_single_tensor_and_capacity():
     from paper_2412_00876_b200 import binding as dl
     B, T, H, D, cap = 2, 40, 4, 128, 48
