@@ -1,7 +1,7 @@
 // Prefill attention over the reduced set on the tensor cores (Eq. 1 applied to S^{P*}):
 // row i of a sequence's compact context attends rows 0..i of the same context.
 // bf16, head_dim 128.  One persistent CTA per SM walks work items (sequence, head, PAIR of 128-row
-// query tiles), the pairs of a head side by side.  The two query tiles of a pair run as two lanes, A (the later rows)
+// query tiles), longest pairs first.  The two query tiles of a pair run as two lanes, A (the later rows)
 // and B (the 128 rows before them): each lane has its own Q buffers, its own score / output
 // accumulators in tensor memory, its own MMA-issuing thread and its own four softmax warps, and both
 // read the same K and V tiles, which are fetched once per pair into a ring shared by the lanes.
@@ -133,49 +133,44 @@ __device__ __forceinline__ int ld_early(const int32_t* p) {
   return v;
 }
 
-// Walks the items of this CTA in the order every role uses.  The CTA's k-th item has the linear index
-// i = blockIdx + k * grid; it belongs to head (b, h) = i / q_pairs, so the pairs of one head run at
-// the same time on neighbouring SMs and fetch its K and V from memory once (the later ones hit L2).
-// Which pair of the head it is rotates with k (p = (i mod q_pairs + k) mod q_pairs), so every CTA
-// gets long and short pairs alike whatever the grid size.  The length of the NEXT item's sequence
-// is requested one item early, so its latency never sits in front of a role's first wait.
-constexpr bool kAtHeadMajor = false;
+// Walks the items of this CTA in the order every role uses: item = p * B * H + b * H + h, stepping by the
+// grid size, so all pairs 0 (the longest) come first.  The position is kept as (p, b, h) and advanced by
+// additions (a division per item and role is what an item's set-up cannot afford); the length of the NEXT
+// item's sequence is requested one item early, so its latency never sits in front of a role's first wait.
+// (Walking head by head instead, all pairs of a head side by side, halves the DRAM reads on long contexts
+// - K and V of a head are then fetched once - but measured 20-60 % slower: the kernel is not DRAM-bound.)
 constexpr bool kAtSwapLanes = true;
 struct AtWalker {
   const AtArgs& a;
-  int i, kr, items, len, sw;                   // next item's linear index, k mod q_pairs, item count, length, swap bit
-  __device__ __forceinline__ int bh_of(int idx) const { return kAtHeadMajor ? idx / a.q_pairs : idx % (a.B * a.H); }
-  __device__ __forceinline__ int len_of(int idx) const { return ld_early(a.cache_len + bh_of(idx) / a.H); }
+  int p, b, h, len, db, dh, sw;               // next item, its length (in flight), the step as (db, dh), swap bit
   __device__ __forceinline__ explicit AtWalker(const AtArgs& a_) : a(a_) {
-    items = a.B * a.H * a.q_pairs;
-    i = (int)blockIdx.x;
-    kr = 0;
+    const int bh_count = a.B * a.H;
+    p = (int)blockIdx.x / bh_count;
+    const int bh = (int)blockIdx.x - p * bh_count;
+    b = bh / a.H;
+    h = bh - b * a.H;
+    db = (int)gridDim.x / a.H;
+    dh = (int)gridDim.x - db * a.H;
     sw = 0;
-    len = i < items ? len_of(i) : 0;
+    len = p < a.q_pairs ? ld_early(a.cache_len + b) : 0;
   }
   // Advances to the next item that exists (a sequence of 256 p rows or fewer has no pair p).
   __device__ __forceinline__ bool next(AtItem& I) {
     for (;;) {
-      if (i >= items) return false;
-      const int ci = i, ck = kr, clen = len;
-      i += (int)gridDim.x;
-      if (++kr == a.q_pairs) kr = 0;
-      if (i < items) len = len_of(i);
-      const int bh = bh_of(ci);
-      int p;
-      if (kAtHeadMajor) {
-        p = ci - bh * a.q_pairs + ck;
-        if (p >= a.q_pairs) p -= a.q_pairs;
-      } else {
-        p = ci / (a.B * a.H);
-      }
-      I.b = bh / a.H;
-      I.h = bh - I.b * a.H;
+      if (p >= a.q_pairs) return false;
+      const int cp = p, cb = b, ch = h, clen = len;
+      h += dh;
+      b += db;
+      if (h >= a.H) { h -= a.H; ++b; }
+      while (b >= a.B) { b -= a.B; ++p; }
+      if (p < a.q_pairs) len = ld_early(a.cache_len + b);
+      I.b = cb;
+      I.h = ch;
       I.n = min(max(clen, 0), min(a.cap, a.n_max));
-      I.q_hi = I.n - p * 2 * kAtBM;
+      I.q_hi = I.n - cp * 2 * kAtBM;
       if (I.q_hi <= 0) continue;
       I.n_kv = (I.q_hi + kAtBN - 1) / kAtBN;
-      I.row_base = bh * a.cap;                                      // first row of this (b, h) in the caches
+      I.row_base = (cb * a.H + ch) * a.cap;                         // first row of this (b, h) in the caches
       I.swap = kAtSwapLanes ? sw : 0;
       sw ^= 1;
       return true;
@@ -425,7 +420,14 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           wait_ring(T);
           if (un < n_sub) wait_ring(T0 + 2 * (un / SUB));
           if (u == 0) mbar_wait_spin(o_free(x), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
-          mbar_wait_spin(p_full(x, b), (g / SUB) & 1, abort_flag);
+          // polled without suspending: the wake-up of a suspended wait costs this thread ~600 cycles per tile
+          {
+            const uint32_t pb = p_full(x, b), ph = (uint32_t)(g / SUB) & 1u;
+            int spins = 0;
+            while (!mbar_test(pb, ph)) {
+              if ((++spins & 1023) == 0 && (*abort_flag || spins > (kSpinLimitBusy << 4))) { *abort_flag = 1; break; }
+            }
+          }
           tc_fence_after();
           const uint64_t v_desc =
               smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128) + (uint64_t)(((u % SUB) * Wd * 128) >> 4);
