@@ -39,7 +39,7 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-every", type=int, default=64, help="decode steps between timed attention launches")
-    ap.add_argument("--micro", default="", choices=["", "decode", "predictor", "compact", "prefill", "nocache"],
+    ap.add_argument("--micro", default="", choices=["", "decode", "predictor", "select", "compact", "prefill", "nocache"],
                     help="time one stage alone on the config's shapes (small memory; used for ncu captures)")
     ap.add_argument("--micro-layers", type=int, default=2, help="layers of cache / source held in --micro mode")
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
@@ -94,6 +94,19 @@ def micro(args):
         out = torch.empty(rows, dtype=torch.float32, device=dev)
         work, unit = 2.0 * rows * cfg.hidden * cfg.pred_hidden, "TFLOP/s"
         calls = [lambda l=l: ctx.predictor_scores(pd, xs[l], out) for l in range(NL)]
+    elif args.micro == "select":
+        # the whole prefill selection of a batch as one call: predictor scores, then the k best per sequence
+        p = wl.make_predictor(cfg, "img")
+        pd = dl.Predictor(wl.to_torch(p.w1, cfg.dtype, dev), torch.from_numpy(p.b1).to(dev),
+                          torch.from_numpy(p.w2).to(dev), p.b2)
+        xs = [wl.device_normal(cfg, wl.S_X_VIS, (B, cfg.n_vis, cfg.hidden), dev, sub=i) for i in range(NL)]
+        n_vis = torch.full((B,), cfg.n_vis, **i32)
+        k_arr = torch.full((B,), cfg.k_vis, **i32)
+        score = torch.empty(B, cfg.n_vis, dtype=torch.float32, device=dev)
+        kept = torch.empty(B, cfg.k_vis, dtype=torch.int32, device=dev)
+        keepm = torch.empty(B, cfg.n_vis, dtype=torch.uint8, device=dev)
+        work, unit = 2.0 * rows * cfg.hidden * cfg.pred_hidden, "TFLOP/s"
+        calls = [lambda l=l: ctx.prefill_select(pd, xs[l], n_vis, k_arr, score, kept, keepm) for l in range(NL)]
     elif args.micro in ("compact", "prefill"):
         T = cfg.n_vis + cfg.n_text
         src = [wl.device_normal(cfg, wl.S_K, (B, T, H, D), dev, sub=i) for i in range(2 * NL)]
