@@ -84,16 +84,36 @@ topk_kernel(const float* __restrict__ score, const int32_t* __restrict__ n_vis,
         if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 0xff], 1);
       }
       __syncthreads();
-      if (tid == 0) {
-        int rem = sh_remaining;
-        int d = 255;
-        for (; d > 0; --d) {
-          int c = hist[d];
-          if (c >= rem) break;
-          rem -= c;
+      if (tid < 32) {
+        // the digit d with (keys in higher digits) < remaining <= (keys in digits >= d), found by one warp:
+        // lane l owns the eight digits 255 - 8l .. 248 - 8l, highest first
+        const int rem = sh_remaining;
+        int c[8], lane_total = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = hist[255 - 8 * tid - j]; lane_total += c[j]; }
+        int incl = lane_total;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          int v = __shfl_up_sync(0xffffffffu, incl, o);
+          if (tid >= o) incl += v;
         }
-        sh_remaining = rem;
-        sh_prefix = prefix | ((uint32_t)d << shift);
+        int above = incl - lane_total;                       // keys in the digits of lower lanes (higher digits)
+        const bool mine = above < rem && rem <= incl;
+        const unsigned who = __ballot_sync(0xffffffffu, mine);
+        if (who == 0u) {
+          // fewer keys than asked for cannot happen (remaining <= keys under the prefix); digit 0 as a guard
+          if (tid == 31) { sh_remaining = max(1, rem - (incl - c[7])); sh_prefix = prefix; }
+        } else if (mine) {
+          int d = 255 - 8 * tid, r = rem - above;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (c[j] >= r) break;
+            r -= c[j];
+            --d;
+          }
+          sh_remaining = r;
+          sh_prefix = prefix | ((uint32_t)d << shift);
+        }
       }
       mask |= 0xffu << shift;
       __syncthreads();
