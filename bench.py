@@ -45,7 +45,8 @@ def parse():
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
     ap.add_argument("--decode-chunk", type=int, default=0, help="--micro decode: rows per work item (0: library's choice)")
     ap.add_argument("--prefill-impl", type=int, default=0,
-                    help="--micro prefill/nocache: 0 library's choice, 2 whole 128-key tiles, 3 64-key half tiles")
+                    help="--micro prefill/nocache: 0 library's choice, 2 whole 128-key tiles, 3 64-key half tiles, "
+                         "4 P through shared memory")
     return ap.parse_args()
 
 
