@@ -47,6 +47,9 @@ def parse():
     ap.add_argument("--prefill-impl", type=int, default=0,
                     help="--micro prefill/nocache: 0 library's choice, 2 whole 128-key tiles, 3 64-key half tiles, "
                          "4 P through shared memory")
+    ap.add_argument("--compact-impl", type=int, default=0,
+                    help="--micro compact: 0 library's choice, 1 register-staged copy, 2 bulk copy by token tiles, "
+                         "3 bulk copy by even row ranges")
     return ap.parse_args()
 
 
@@ -70,6 +73,8 @@ def micro(args):
         ctx.set_option(dl.DL_OPT_DECODE_CHUNK, args.decode_chunk)
     if args.prefill_impl:
         ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, args.prefill_impl)
+    if args.compact_impl:
+        ctx.set_option(dl.DL_OPT_COMPACT_IMPL, args.compact_impl)
     scale = 1.0 / float(np.sqrt(D))
     i32 = dict(dtype=torch.int32, device=dev)
     work, unit, calls = 0.0, "GB/s", []

@@ -57,7 +57,9 @@ enum {
                                  * shared memory and the score buffer released early (auto: whole tiles) */
   DL_OPT_DECODE_CHUNK = 3,      /* cache rows per decode work item (0 = chosen by the library) */
   DL_OPT_DECODE_IMPL = 4,       /* 0 auto, 1 CUDA-core kernel, 2 tensor-core (mma.sync) kernel (bf16, D=128) */
-  DL_OPT_COMPACT_IMPL = 5       /* 0 auto, 1 register-staged copy kernel, 2 bulk-copy (TMA) kernel */
+  DL_OPT_COMPACT_IMPL = 5       /* 0 auto, 1 register-staged copy kernel, 2 bulk-copy (TMA) kernel by tiles of 32
+                                 * source tokens, 3 bulk-copy kernel over even ranges of kept rows with one tensor
+                                 * store per row (auto: 3 for up to 2048 sequences, else 2) */
 };
 
 typedef struct {

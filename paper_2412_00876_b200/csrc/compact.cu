@@ -8,9 +8,15 @@
 //   copy : per tile of 32 source tokens, rank the kept ones by a ballot scan on top of the
 //          count of kept tokens before the tile, then move each kept row with 16-byte loads
 //          and stores (a warp moves 512 contiguous source bytes per instruction).
-// Dropped rows are never read.
+// Dropped rows are never read.  The copy exists in three forms (DL_OPT_COMPACT_IMPL): register-staged by
+// token tiles, bulk (TMA) copies by token tiles, and bulk copies over even row ranges with one tensor
+// store per row, which is the one the library picks where it applies.
+#include <algorithm>
+#include <cstring>
+
 #include "common.cuh"
 #include "pipeline.cuh"
+#include "tc05.cuh"
 
 namespace dl {
 
@@ -253,6 +259,179 @@ compact_copy_bulk_kernel(const char* __restrict__ k_src, const char* __restrict_
   }
 }
 
+// The bulk copy again, with the work dealt evenly: the kept rows of the whole batch, in (sequence, rank)
+// order, are cut into one contiguous range per CTA (the tile kernel above gives a CTA 32 source tokens,
+// so a tile of text tokens, all kept, carries four times the rows of a tile of vision tokens at a 25 % keep
+// rate, and the CTAs that start last finish long after the rest).  A CTA reads the per-sequence row counts
+// of the plan, finds its range, and for each sequence the range touches ranks the sequence's mask once
+// (a block scan over 128 token segments) to list the tokens whose rank falls inside; its warps then move
+// those rows exactly as above, their two-buffer pipelines running on across lists.  Up to 2048 sequences.
+constexpr int kRowsList = 64;
+constexpr int kRowsMaxBatch = 2048;
+
+// Tensor maps of the two caches for the row stores (32-bit words, no swizzle).
+struct RowMaps { alignas(64) unsigned char k[128]; alignas(64) unsigned char v[128]; };
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+// cache [B*H][cap][piece] as words; box = (piece, 1 row, H heads): what one token row holds, head by head
+static bool encode_row_map(void* fn, void* out, const void* base, int piece_bytes, int cap, long long bh, int H) {
+  if (!fn || !base) return false;
+  if ((piece_bytes & 15) || piece_bytes / 4 > 256 || H > 256) return false;
+  cuuint64_t gd[3] = {(cuuint64_t)(piece_bytes / 4), (cuuint64_t)cap, (cuuint64_t)bh};
+  cuuint64_t gs[2] = {(cuuint64_t)piece_bytes, (cuuint64_t)piece_bytes * (cuuint64_t)cap};
+  cuuint32_t bx[3] = {(cuuint32_t)(piece_bytes / 4), 1u, (cuuint32_t)H};
+  cuuint32_t es[3] = {1u, 1u, 1u};
+  return reinterpret_cast<EncodeTiledFn>(fn)(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_UINT32, 3,
+                                             const_cast<void*>(base), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                             CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+__global__ void __launch_bounds__(kBulkWarps * 32)
+compact_copy_rows_kernel(const char* __restrict__ k_src, const char* __restrict__ v_src,
+                         const uint8_t* __restrict__ keep, int32_t keep_cols, const int32_t* __restrict__ t_src,
+                         int32_t t_max, char* __restrict__ k_cache, char* __restrict__ v_cache, int32_t cap, int32_t H,
+                         int32_t row_bytes, int32_t piece_bytes, int32_t B, const int32_t* plan_base,
+                         const int32_t* plan_count, DeviceStatus* st, const __grid_constant__ RowMaps maps,
+                         int32_t use_maps) {
+  extern __shared__ __align__(128) char rows_s[];
+  __shared__ uint64_t bars[kBulkWarps][2];
+  __shared__ int sh[kBulkWarps];
+  __shared__ int s_cnt[kRowsMaxBatch];
+  __shared__ int list_tok[kRowsList];
+  __shared__ int sh_abort;
+  volatile int* abort_flag = &sh_abort;
+  constexpr int kThreads = kBulkWarps * 32;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) sh_abort = 0;
+  if (lane == 0) {
+    mbar_init(smem_u32(&bars[warp][0]), 1);
+    mbar_init(smem_u32(&bars[warp][1]), 1);
+    fence_mbar_init();
+  }
+  // launched with programmatic stream serialisation: the plan of this call is complete from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  int part = 0;
+  for (int b = tid; b < B; b += kThreads) {
+    const int c = max(ld_plan(plan_count + b), 0);                    // -1: the sequence does not fit, skip it
+    s_cnt[b] = c;
+    part += c;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+  if (lane == 0) sh[warp] = part;
+  __syncthreads();
+  long long n_rows = 0;
+#pragma unroll
+  for (int w = 0; w < kBulkWarps; ++w) n_rows += sh[w];
+  const long long lo = n_rows * blockIdx.x / gridDim.x, hi = n_rows * (blockIdx.x + 1) / gridDim.x;
+  if (hi <= lo) return;
+
+  const int n_tensors = v_src ? 2 : 1;
+  char* buf = rows_s + (size_t)warp * 2 * row_bytes;
+  const size_t head_stride = (size_t)cap * piece_bytes;
+  int n_ld = 0;                                   // loads this warp has issued so far (the same in every lane)
+  bool ok = true;
+  long long off = 0;                              // rows of the sequences before b
+  for (int b = 0; b < B && off < hi && ok; ++b) {
+    const int cb = s_cnt[b];
+    const int ra = (int)max(lo - off, 0LL), rb = (int)min(hi - off, (long long)cb);
+    off += cb;
+    if (ra >= rb) continue;
+    int tb = t_src ? t_src[b] : t_max;
+    tb = max(0, min(tb, t_max));
+    const uint8_t* kp = keep ? keep + (size_t)b * keep_cols : nullptr;
+    const int base_row = ld_plan(plan_base + b);
+    const int seg = (tb + kThreads - 1) / kThreads, ts = min(tb, tid * seg), te = min(tb, ts + seg);
+    auto kept = [&](int i) { return kp == nullptr || i >= keep_cols || kp[i] != 0; };
+    for (int r0 = ra; r0 < rb && ok; r0 += kRowsList) {
+      const int r1 = min(rb, r0 + kRowsList);
+      // ---- tokens of ranks [r0, r1): block scan of the kept counts of 128 token segments
+      int cnt = 0;
+      for (int i = ts; i < te; ++i) cnt += kept(i);
+      int incl = cnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      __syncthreads();                            // the previous list and sh are no longer read
+      if (lane == 31) sh[warp] = incl;
+      __syncthreads();
+      int r = incl - cnt;
+      for (int w = 0; w < warp; ++w) r += sh[w];
+      if (r < r1 && r + cnt > r0) {
+        for (int i = ts; i < te; ++i)
+          if (kept(i)) {
+            if (r >= r0 && r < r1) list_tok[r - r0] = i;
+            ++r;
+          }
+      }
+      __syncthreads();
+      // ---- this warp's (row, tensor) jobs of the list: job = warp + idx * warps
+      const int total = (r1 - r0) * n_tensors;
+      const int my_jobs = total > warp ? (total - warp + kBulkWarps - 1) / kBulkWarps : 0;
+      const int dst0 = base_row + r0;
+      auto load = [&](int idx) {
+        const int job = warp + idx * kBulkWarps;
+        const int j = job / n_tensors, which = job - j * n_tensors;
+        const char* src = (which ? v_src : k_src) + ((size_t)b * t_max + list_tok[j]) * row_bytes;
+        const int g = n_ld + idx;
+        const uint32_t bar = smem_u32(&bars[warp][g & 1]);
+        mbar_expect_tx(bar, (uint32_t)row_bytes);
+        bulk_g2s(smem_u32(buf + (size_t)(g & 1) * row_bytes), src, (uint32_t)row_bytes, bar);
+      };
+      if (my_jobs > 0) {
+        // the buffer's previous row: every lane's stores of it must have read it before it is refilled
+        bulk_group_wait_read_all();
+        __syncwarp();
+        if (lane == 0) load(0);
+      }
+      int done = 0;
+      for (int idx = 0; idx < my_jobs; ++idx) {
+        if (idx + 1 < my_jobs) {
+          bulk_group_wait_read_all();
+          __syncwarp();
+          if (lane == 0) load(idx + 1);
+        }
+        const int g = n_ld + idx;
+        done = min(my_jobs, idx + 2);             // loads issued so far in this list
+        if (!mbar_wait(smem_u32(&bars[warp][g & 1]), (g >> 1) & 1, abort_flag)) { ok = false; break; }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const int job = warp + idx * kBulkWarps;
+        const int j = job / n_tensors, which = job - j * n_tensors;
+        char* dst = (which ? v_cache : k_cache) + (size_t)b * H * head_stride + (size_t)(dst0 + j) * piece_bytes;
+        const uint32_t src = smem_u32(buf + (size_t)(g & 1) * row_bytes);
+        if (use_maps) {
+          // the row's H head pieces as ONE tensor store: box (piece, 1 row, H heads) of the cache seen as
+          // [B*H][cap][piece]
+          if (lane == 0)
+            tma_store_3d(reinterpret_cast<const CUtensorMap*>(which ? maps.v : maps.k), src, 0, dst0 + j, b * H);
+        } else {
+          for (int h = lane; h < H; h += 32) bulk_s2g(dst + (size_t)h * head_stride, src + (uint32_t)(h * piece_bytes), (uint32_t)piece_bytes);
+        }
+        bulk_group_commit();
+      }
+      n_ld += ok ? my_jobs : done;
+      if (*abort_flag) ok = false;                // another warp gave up: leave together (the loop holds block barriers)
+      ok = __syncthreads_and(ok);
+    }
+  }
+  bulk_group_wait_read_all();                     // shared memory is read before the CTA ends
+  if (*abort_flag) {
+    // a load that was issued must land before the CTA's shared memory is released
+    if (lane == 0) {
+      report_status(st, DL_ERR_TIMEOUT, blockIdx.x);
+      for (int j = max(0, n_ld - 2); j < n_ld; ++j)
+        for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&bars[warp][j & 1]), (j >> 1) & 1); ++i) __nanosleep(40);
+    }
+  }
+}
+
 cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
                            int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
                            void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, cudaStream_t s) {
@@ -280,10 +459,31 @@ cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_s
     int& set_for = attr_set[ctx->device & 63];
     if (set_for < (int)bulk_smem) {
       e = cudaFuncSetAttribute(compact_copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk_smem);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(compact_copy_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk_smem);
       if (e != cudaSuccess) return e;
       set_for = (int)bulk_smem;
     }
     cfg.blockDim = dim3(kBulkWarps * 32); cfg.dynamicSmemBytes = bulk_smem;
+    if (ctx->opt.compact_impl != 2 && B <= kRowsMaxBatch) {
+      // evenly dealt rows: as many CTAs as fit the GPU at once, fewer when the batch has few rows
+      const size_t per_cta = bulk_smem + 10 * 1024;
+      const long long resident = (long long)ctx->sm_count * std::max<size_t>(1, (size_t)ctx->smem_optin / per_cta);
+      const long long by_rows = ((long long)B * t_src_max + 7) / 8;
+      cfg.gridDim = dim3((unsigned)std::max(1LL, std::min(resident, by_rows)));
+      // one tensor store per row where the row buffers are 128-byte aligned and the maps can be made
+      RowMaps maps;
+      memset(&maps, 0, sizeof(maps));
+      const int piece_bytes = piece_units * 16;
+      int32_t use_maps = (row_bytes % 128 == 0) &&
+                         encode_row_map(ctx->tmap_encode, maps.k, k_cache, piece_bytes, cap, (long long)B * d.n_heads, d.n_heads) &&
+                         (!v_src || encode_row_map(ctx->tmap_encode, maps.v, v_cache, piece_bytes, cap, (long long)B * d.n_heads, d.n_heads));
+      return cudaLaunchKernelEx(&cfg, compact_copy_rows_kernel, (const char*)k_src, (const char*)v_src, keep,
+                                (int32_t)keep_cols, t_src, (int32_t)t_src_max, (char*)k_cache, (char*)v_cache,
+                                (int32_t)cap, (int32_t)d.n_heads, (int32_t)row_bytes, (int32_t)piece_bytes,
+                                (int32_t)B, (const int32_t*)ctx->ws.plan_base, (const int32_t*)ctx->ws.plan_count,
+                                ctx->ws.status, maps, use_maps);
+    }
     return cudaLaunchKernelEx(&cfg, compact_copy_bulk_kernel, (const char*)k_src, (const char*)v_src, keep,
                               (int32_t)keep_cols, t_src, (int32_t)t_src_max, (char*)k_cache, (char*)v_cache, (int32_t)cap,
                               (int32_t)d.n_heads, (int32_t)row_bytes, (int32_t)(piece_units * 16),

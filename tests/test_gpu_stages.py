@@ -63,12 +63,15 @@ def test_topk_paper_rate():
 
 
 # ------------------------------------------------------------------------------ compaction
+@pytest.mark.parametrize("impl", [0, 1, 2, 3])      # library's choice; register-staged; bulk copy by tiles / by even row ranges
 @pytest.mark.parametrize("dtype,H,D", [("bf16", 32, 128), ("f32", 8, 64), ("bf16", 3, 64), ("f32", 2, 128)])
-def test_compaction_bit_exact(dtype, H, D):
+def test_compaction_bit_exact(dtype, H, D, impl):
+    from paper_2412_00876_b200 import binding as dl
     rng = np.random.default_rng(2)
     B, T, nv, cap = 3, 150, 110, 256
     cfg = wl.CONFIGS[1]
     ctx = _ctx(dtype, H, D, B=B, cap=cap)
+    ctx.set_option(dl.DL_OPT_COMPACT_IMPL, impl)
     ks = wl.host_normal(cfg, wl.S_K, (B, T, H, D), dtype=dtype)
     vs = wl.host_normal(cfg, wl.S_V, (B, T, H, D), dtype=dtype)
     keep = (rng.random((B, nv)) < 0.3).astype(np.uint8)
@@ -98,7 +101,7 @@ def test_compaction_bit_exact(dtype, H, D):
     assert ctx.device_status()[0] == 0
 
 
-@pytest.mark.parametrize("impl", [1, 2])
+@pytest.mark.parametrize("impl", [1, 2, 3])
 def test_compaction_does_not_read_a_stale_plan(impl):
     """The copy kernel starts while the plan kernel of the same call still runs.  With the workspace holding
     a hostile old plan (count -1 = skip the sequence) a copy that read the plan too early would leave rows
