@@ -73,9 +73,13 @@ def selection_flips(s_ref: np.ndarray, keep_gpu: np.ndarray, k: int):
 
 
 def run_chained(cid: int, n_decode: int | None = None, B: int | None = None, L: int | None = None,
-                ragged: bool = False, options: dict | None = None, device: int = 0, verbose: bool = False):
+                ragged: bool = False, options: dict | None = None, device: int = 0, verbose: bool = False,
+                shape: dict | None = None, txt_keep_rate: float | None = None):
+    """`shape` overrides fields of the configuration (n_vis, k_vis, n_text, ...); `txt_keep_rate` moves the decode
+    predictor's second-layer bias so that about that share of this run's generated tokens gets a positive logit
+    (the bias is an input of both implementations; it is taken from the oracle's logits of the same rows)."""
     cfg = wl.CONFIGS[cid]
-    kw = {}
+    kw = dict(shape or {})
     if B is not None:
         kw["B"] = B
     if L is not None:
@@ -105,6 +109,9 @@ def run_chained(cid: int, n_decode: int | None = None, B: int | None = None, L: 
         k_arr[1] = min(cfg.k_vis, n_vis[1]) // 2
     t_src = (cfg.n_vis + n_text).astype(np.int32)
     x_dec = wl.host_normal(cfg, wl.S_X_TXT, (cfg.n_gen, B, cfg.hidden))
+    if txt_keep_rate is not None:
+        z0 = orc.predictor_logits(x_dec.reshape(-1, cfg.hidden), p_txt.w1, p_txt.b1, p_txt.w2, 0.0)
+        p_txt = wl.make_predictor(cfg, "txt", b2=float(-np.quantile(z0, 1.0 - txt_keep_rate)))
     q_dec = wl.host_normal(cfg, wl.S_DEC_Q, (cfg.n_gen, L, B, H, D))
     k_dec = wl.host_normal(cfg, wl.S_DEC_K, (cfg.n_gen, L, B, H, D))
     v_dec = wl.host_normal(cfg, wl.S_DEC_V, (cfg.n_gen, L, B, H, D))
