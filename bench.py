@@ -434,7 +434,9 @@ def main():
         barrier()
         ms = max_over_ranks(max(a.elapsed_time(b), (time.perf_counter() - t0) * 1e3)) / k2
         e2e = {"value": world * cfg.B * cfg.n_gen / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": k2, "ms_per_step": ms}
+               "d2h_bytes_per_step": d2h, "steps": k2, "ms_per_step": ms,
+               "prefill_sources": "left in pinned host memory; the compaction kernel fetches the kept rows over the "
+                                  "bus itself (h2d counts those rows), dropped rows are never transferred"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

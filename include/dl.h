@@ -149,6 +149,17 @@ int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const u
                       int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
                       void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, void* stream);
 
+/* dl_compact_kv with the SOURCE rows in pinned host memory (Eq. 5 / Eq. 11: only the kept rows enter the
+ * reduced set, so only they need to reach the GPU).  The copy kernel reads the kept rows straight from host
+ * memory over the bus; dropped rows never cross it, and no staging copy of the whole source is made.
+ *   k_src_host, v_src_host HOST, pinned and reachable from the device (cudaHostAlloc / cudaHostRegister,
+ *   e.g. torch's pin_memory()), [B][t_src_max][H][D]; every other argument as for dl_compact_kv (device).
+ * The host buffers must stay valid and unchanged until the stream has passed this call.
+ * DL_ERR_INVALID_ARG if a source is not such host memory. */
+int32_t dl_compact_kv_host(dl_ctx* ctx, const void* k_src_host, const void* v_src_host, const uint8_t* keep,
+                           int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
+                           void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, void* stream);
+
 /* ---- attention over the reduced set --------------------------------------------------- */
 
 /* Prefill (Eq. 1 on S^{P*}): causal scaled-dot-product attention of the compact rows against

@@ -27,7 +27,7 @@ EXPORTS = [
     "dl_topk_from_scores", "dl_prefill_select", "dl_compact_kv", "dl_sparse_attn_prefill",
     "dl_sparse_attn_decode", "dl_decode_keep", "dl_commit_len", "dl_decode_step", "dl_decode_step_host",
     "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers", "dl_decode_nocache_select",
-    "dl_decode_steps_host",
+    "dl_decode_steps_host", "dl_compact_kv_host",
 ]
 
 
@@ -67,6 +67,7 @@ def lib() -> C.CDLL:
             "dl_topk_from_scores": (i32, [vp, vp, vp, vp, i32, i32, vp, i32, vp, vp]),
             "dl_prefill_select": (i32, [vp, P, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp]),
             "dl_compact_kv": (i32, [vp, vp, vp, vp, i32, vp, i32, i32, vp, vp, i32, vp, i32, vp]),
+            "dl_compact_kv_host": (i32, [vp, vp, vp, vp, i32, vp, i32, i32, vp, vp, i32, vp, i32, vp]),
             "dl_sparse_attn_prefill": (i32, [vp, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp]),
             "dl_sparse_attn_decode": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp]),
             "dl_sparse_attn_decode_static": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp]),
@@ -200,6 +201,16 @@ class Context:
         self._check(lib().dl_compact_kv(self._h, _ptr(k_src), _ptr(v_src), _ptr(keep), keep_cols, _ptr(t_src), B, T,
                                         _ptr(k_cache), _ptr(v_cache), cap, _ptr(cache_len), int(bool(commit)),
                                         _stream(stream)), "dl_compact_kv")
+
+    def compact_kv_host(self, k_src_host, v_src_host, keep, t_src, k_cache, v_cache, cache_len, commit=True,
+                        stream=None):
+        """dl_compact_kv with the source rows in pinned host tensors: the kernel fetches the kept rows itself."""
+        B, T = k_src_host.shape[0], k_src_host.shape[1]
+        cap = k_cache.shape[2]
+        keep_cols = 0 if keep is None else keep.shape[1]
+        self._check(lib().dl_compact_kv_host(self._h, _ptr(k_src_host), _ptr(v_src_host), _ptr(keep), keep_cols,
+                                             _ptr(t_src), B, T, _ptr(k_cache), _ptr(v_cache), cap, _ptr(cache_len),
+                                             int(bool(commit)), _stream(stream)), "dl_compact_kv_host")
 
     def sparse_attn_prefill(self, q, k_cache, v_cache, cache_len, n_max, scale, out, stream=None):
         B, cap = k_cache.shape[0], k_cache.shape[2]

@@ -240,6 +240,32 @@ int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const u
                                          cache_len, commit, static_cast<cudaStream_t>(stream)));
 }
 
+// The device's address of a pinned, device-reachable host buffer (nullptr if it is anything else).
+static const void* device_view_of_host(const void* host_ptr) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, host_ptr) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  if (at.type != cudaMemoryTypeHost || at.devicePointer == nullptr) return nullptr;
+  return at.devicePointer;
+}
+
+int32_t dl_compact_kv_host(dl_ctx* ctx, const void* k_src_host, const void* v_src_host, const uint8_t* keep,
+                           int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
+                           void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, void* stream) {
+  if (!ctx || B < 0 || t_src_max < 0 || cap <= 0 || keep_cols < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || t_src_max == 0) return DL_OK;
+  if (!k_src_host || !k_cache || !cache_len) return DL_ERR_INVALID_ARG;
+  if ((v_src_host == nullptr) != (v_cache == nullptr)) return DL_ERR_INVALID_ARG;
+  if (!ctx->ws.base || B > ctx->ws.max_batch) return DL_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  const void* k_dev = device_view_of_host(k_src_host);
+  const void* v_dev = v_src_host ? device_view_of_host(v_src_host) : nullptr;
+  if (!k_dev || (v_src_host && !v_dev)) return DL_ERR_INVALID_ARG;      // not pinned host memory
+  if (misaligned(k_dev) || misaligned(v_dev) || misaligned(k_cache) || misaligned(v_cache)) return DL_ERR_ALIGNMENT;
+  // the copy kernel with plain 16-byte loads: they reach pinned host memory like any other address
+  return cuda_status(ctx, launch_compact(ctx, k_dev, v_dev, keep, keep_cols, t_src, B, t_src_max, k_cache, v_cache, cap,
+                                         cache_len, commit, static_cast<cudaStream_t>(stream), 1));
+}
+
 int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max, float scale,
                                void* out, void* stream) {

@@ -117,7 +117,8 @@ cudaError_t launch_topk(const float* score, const int32_t* n_vis, const int32_t*
 
 cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
                            int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
-                           void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, cudaStream_t s);
+                           void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, cudaStream_t s,
+                           int32_t force_impl = 0);
 
 cudaError_t launch_commit_len(const uint8_t* keep, int32_t B, int32_t cap, int32_t* cache_len,
                               cudaStream_t s);

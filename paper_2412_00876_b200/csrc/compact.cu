@@ -434,8 +434,10 @@ compact_copy_rows_kernel(const char* __restrict__ k_src, const char* __restrict_
 
 cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
                            int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
-                           void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, cudaStream_t s) {
+                           void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, cudaStream_t s,
+                           int32_t force_impl) {
   if (B == 0 || t_src_max == 0) return cudaSuccess;
+  const int impl = force_impl ? force_impl : ctx->opt.compact_impl;
   const dl_model_desc& d = ctx->desc;
   const int elt = d.dtype == DL_F32 ? 4 : 2;
   const int piece_units = d.head_dim * elt / 16;
@@ -454,7 +456,7 @@ cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_s
   // bulk-copy kernel where two row buffers per warp fit the shared memory (they do for every shape at hand:
   // a row is H * D * elt bytes, 8 KB for 32 heads of 128 bf16)
   const size_t row_bytes = (size_t)row_units * 16, bulk_smem = 2 * kBulkWarps * row_bytes;
-  if (ctx->opt.compact_impl != 1 && bulk_smem + 1024 <= (size_t)ctx->smem_optin) {
+  if (impl != 1 && bulk_smem + 1024 <= (size_t)ctx->smem_optin) {
     static int attr_set[64];
     int& set_for = attr_set[ctx->device & 63];
     if (set_for < (int)bulk_smem) {
@@ -465,7 +467,7 @@ cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_s
       set_for = (int)bulk_smem;
     }
     cfg.blockDim = dim3(kBulkWarps * 32); cfg.dynamicSmemBytes = bulk_smem;
-    if (ctx->opt.compact_impl != 2 && B <= kRowsMaxBatch) {
+    if (impl != 2 && B <= kRowsMaxBatch) {
       // evenly dealt rows: as many CTAs as fit the GPU at once, fewer when the batch has few rows
       const size_t per_cta = bulk_smem + 10 * 1024;
       const long long resident = (long long)ctx->sm_count * std::max<size_t>(1, (size_t)ctx->smem_optin / per_cta);

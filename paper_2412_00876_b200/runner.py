@@ -184,7 +184,6 @@ class BatchRunner:
         self.s_logit, self.s_keep = two(self.logit), two(self.keep_t)
         self.h_dec_out2 = [torch.empty_like(self.dec_out, device="cpu").pin_memory() for _ in range(2)]
         self.h_keep2 = [torch.empty(self.cfg.B, dtype=torch.uint8).pin_memory() for _ in range(2)]
-        self.s_qsrc, self.s_ksrc, self.s_vsrc = (torch.empty_like(self.q_src[0]) for _ in range(3))
         self.s_xvis = torch.empty_like(self.x_vis)
 
     def run_batch_host_fed(self):
@@ -196,18 +195,20 @@ class BatchRunner:
         self.s_xvis.copy_(self.h_x_vis, non_blocking=True)
         h2d += self.h_x_vis.numel() * self.h_x_vis.element_size()
         ctx.prefill_select(self.p_img, self.s_xvis, self.n_vis, self.k_arr, self.score, self.kept_idx, self.keep_vis)
+        # the per-layer Q/K/V sources stay in pinned host memory: the compaction kernel fetches the kept rows
+        # itself, so the dropped rows never cross the bus (bytes counted: the kept rows)
+        row_bytes = c.n_heads * c.head_dim * c.elt_bytes
+        kept_bytes = c.B * c.n0 * row_bytes
         for l in range(L):
             i = l % self.src_pool
-            self.s_ksrc.copy_(self.h_k_src[i], non_blocking=True)
-            self.s_vsrc.copy_(self.h_v_src[i], non_blocking=True)
-            h2d += 2 * self.s_ksrc.numel() * self.s_ksrc.element_size()
-            ctx.compact_kv(self.s_ksrc, self.s_vsrc, self.keep_vis, self.t_src, self.k_cache[l], self.v_cache[l],
-                           self.cache_len, commit=(l == L - 1))
+            h2d += 2 * kept_bytes
+            ctx.compact_kv_host(self.h_k_src[i], self.h_v_src[i], self.keep_vis, self.t_src, self.k_cache[l],
+                                self.v_cache[l], self.cache_len, commit=(l == L - 1))
         for l in range(L):
             i = l % self.src_pool
-            self.s_qsrc.copy_(self.h_q_src[i], non_blocking=True)
-            h2d += self.s_qsrc.numel() * self.s_qsrc.element_size()
-            ctx.compact_kv(self.s_qsrc, None, self.keep_vis, self.t_src, self.q_cache, None, self.q_len, commit=False)
+            h2d += kept_bytes
+            ctx.compact_kv_host(self.h_q_src[i], None, self.keep_vis, self.t_src, self.q_cache, None, self.q_len,
+                                commit=False)
             ctx.sparse_attn_prefill(self.q_cache, self.k_cache[l], self.v_cache[l], self.cache_len, c.n0, self.scale,
                                     self.prefill_out)
             self.h_prefill_out.copy_(self.prefill_out, non_blocking=True)

@@ -135,6 +135,38 @@ def test_compaction_does_not_read_a_stale_plan(impl):
     ctx.close()
 
 
+def test_compaction_from_pinned_host_sources():
+    """dl_compact_kv_host (the kernel reads the kept rows from pinned host memory) gives the caches and lengths
+    of dl_compact_kv on a device copy of the same sources, bit for bit; pageable memory is refused."""
+    from paper_2412_00876_b200 import binding as dl
+    B, T, H, D, nv, cap = 4, 300, 32, 128, 200, 320
+    ctx = dl.Context(4096, H, D, 1024, torch.bfloat16, 0, max_batch=B, max_rows=B * nv, cap=cap)
+    g = torch.Generator().manual_seed(11)
+    ks_h = torch.randn(B, T, H, D, generator=g).to(torch.bfloat16).pin_memory()
+    vs_h = torch.randn(B, T, H, D, generator=g).to(torch.bfloat16).pin_memory()
+    keep = (torch.rand(B, nv, generator=g) < 0.3).to(torch.uint8).to(DEV)
+    t_src = torch.tensor([T, T - 9, nv, 5], dtype=torch.int32, device=DEV)
+    res = []
+    for host in (False, True):
+        kc = torch.zeros(B, H, cap, D, dtype=torch.bfloat16, device=DEV)
+        vc = torch.zeros_like(kc)
+        ln = torch.tensor([0, 3, 0, 1], dtype=torch.int32, device=DEV)
+        if host:
+            ctx.compact_kv_host(ks_h, vs_h, keep, t_src, kc, vc, ln, commit=True)
+        else:
+            ctx.compact_kv(ks_h.to(DEV), vs_h.to(DEV), keep, t_src, kc, vc, ln, commit=True)
+        torch.cuda.synchronize()
+        res.append((kc, vc, ln))
+    assert torch.equal(res[0][2], res[1][2]) and int(res[0][2].sum()) > 0
+    assert torch.equal(res[0][0].view(torch.int16), res[1][0].view(torch.int16))
+    assert torch.equal(res[0][1].view(torch.int16), res[1][1].view(torch.int16))
+    assert ctx.device_status()[0] == 0
+    with pytest.raises(dl.DlError) as e:                       # pageable host memory: not reachable from the device
+        ctx.compact_kv_host(torch.zeros(B, T, H, D, dtype=torch.bfloat16), None, keep, t_src, res[0][0], None, res[0][2])
+    assert e.value.code == dl.DL_ERR_INVALID_ARG
+    ctx.close()
+
+
 def test_compaction_keep_all_single_tensor_and_capacity():
     from paper_2412_00876_b200 import binding as dl
     B, T, H, D, cap = 2, 40, 4, 128, 48
