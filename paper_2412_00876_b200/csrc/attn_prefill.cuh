@@ -1,0 +1,174 @@
+// Definitions shared by the tensor-core prefill attention kernels: tile constants, small arithmetic
+// wrappers, tensor maps, the work-item walker and the register-budget instructions.
+#pragma once
+
+#include "common.cuh"
+#include "tc05.cuh"
+
+namespace dl {
+
+constexpr int kAtBM = 128, kAtBN = 128, kAtThreads = 384, kAtRing = 3;
+constexpr int kAtTile = 2 * 128 * 128;                // 32 KB: two [128 rows][64 dims] halves
+constexpr int kAtOffRing = 4 * kAtTile;               // Q: [lane][slot] tiles first
+constexpr int kAtOffBar = kAtOffRing + kAtRing * kAtTile;
+constexpr size_t kAtSmem = kAtOffBar + 512;           // 229888 bytes: one CTA per SM
+constexpr uint32_t kAtColO = 0, kAtColS = 128, kAtLaneCols = 256;   // tensor-memory columns of one lane: O | S
+constexpr float kRescaleStep = 8.0f;                  // log2 units by which the maximum may lag
+
+// 2^x on the special-function unit (x <= 0 here; -inf gives 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// max of three in one instruction
+__device__ __forceinline__ float fmax3(float x, float y, float z) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(x), "f"(y), "f"(z));
+  return r;
+}
+
+// two fp32 lanes in one 64-bit register: fused multiply-add and add on both at once
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t x, uint64_t y, uint64_t z) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(x), "l"(y), "l"(z));
+  return r;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t x, uint64_t y) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(x), "l"(y));
+  return r;
+}
+__device__ __forceinline__ uint64_t fmul2(uint64_t x, uint64_t y) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(x), "l"(y));
+  return r;
+}
+
+// Tensor maps: Q, K and V each with boxes of 128, 64, 32 and 16 rows (index 0..3), so that a ragged
+// tile at the end of a sequence is fetched with the smallest box that covers it; O for the stores.
+struct AtMaps {
+  alignas(64) unsigned char q[4][128]; alignas(64) unsigned char k[4][128];
+  alignas(64) unsigned char v[4][128]; alignas(64) unsigned char o[128];
+};
+// index of the smallest box (128 >> index rows) that covers `rows` (a multiple of 16 in 16..128)
+__device__ __forceinline__ int at_box(int rows) { return rows > 64 ? 0 : rows > 32 ? 1 : rows > 16 ? 2 : 3; }
+
+struct AtArgs {
+  const int32_t* cache_len; __nv_bfloat16* out; DeviceStatus* status;
+  int32_t B, H, cap, n_max, q_pairs, item_rows;     // item_rows: query rows per work item (256: a pair of tiles; 128)
+  float scale_log2;
+};
+
+// Work item -> (b, h, pair p of query tiles).  Pair p counts from the sequence's end: it covers rows
+// [q_hi - 256, q_hi) with q_hi = n - 256 p, clipped at row 0; its keys are [0, q_hi) in n_kv tiles.
+struct AtItem { int b, h, q_hi, n, n_kv, row_base, swap; };
+
+// One lane's share of an item: rows [q0, q_hi) are owned (the Q tile is loaded from row q0, 128 rows;
+// a tile clipped at the top of the sequence loads rows [0, 128) and owns the first q_hi of them),
+// keys [0, q_hi) in n_tiles tiles.  The later query tile of a pair has one key tile more than the
+// earlier one, so the lanes swap tiles from one item to the next (I.swap) and do the same work.
+struct AtLane { int q0, q_hi, n_tiles; bool exists; };
+__device__ __forceinline__ AtLane at_lane(const AtItem& I, int lane_id) {
+  AtLane L;
+  L.q_hi = I.q_hi - (lane_id ^ I.swap) * kAtBM;
+  L.exists = L.q_hi > 0;
+  L.q0 = max(L.q_hi - kAtBM, 0);
+  L.n_tiles = (L.q_hi + kAtBN - 1) / kAtBN;
+  return L;
+}
+// keys of tile j that a lane's MMAs cover: all 128, or what is left of [0, q_hi) rounded up to 16
+__device__ __forceinline__ int at_cols(const AtLane& L, int j) {
+  return min(kAtBN, (L.q_hi - j * kAtBN + 15) & ~15);
+}
+
+// A load the compiler may not sink towards its use (the point is to have it in flight early).
+__device__ __forceinline__ int ld_early(const int32_t* p) {
+  int v;
+  asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+
+// Walks the items of this CTA in the order every role uses: item = p * B * H + b * H + h, stepping by the
+// grid size, so all pairs 0 (the longest) come first.  The position is kept as (p, b, h) and advanced by
+// additions (a division per item and role is what an item's set-up cannot afford); the length of the NEXT
+// item's sequence is requested one item early, so its latency never sits in front of a role's first wait.
+// (Walking head by head instead, all pairs of a head side by side, halves the DRAM reads on long contexts
+// - K and V of a head are then fetched once - but measured 20-60 % slower: the kernel is not DRAM-bound.)
+constexpr bool kAtSwapLanes = true;
+constexpr bool kAtSnake = false;
+struct AtWalker {
+  const AtArgs& a;
+  int p, b, h, len, db0, dh0, db1, dh1, odd, sw;   // next item, its length (in flight), the two steps as (db, dh), swap bit
+  __device__ __forceinline__ explicit AtWalker(const AtArgs& a_) : a(a_) {
+    const int bh_count = a.B * a.H;
+    p = (int)blockIdx.x / bh_count;
+    const int bh = (int)blockIdx.x - p * bh_count;
+    b = bh / a.H;
+    h = bh - b * a.H;
+    // The CTAs take the items (longest first) in rounds that run forwards and backwards in turn, so that the CTA
+    // that got the longest item of one round gets the shortest of the next: CTA c takes items c, 2G-1-c, 2G+c, ...
+    const int G = (int)gridDim.x, s0 = kAtSnake ? 2 * G - 1 - 2 * (int)blockIdx.x : G, s1 = kAtSnake ? 1 + 2 * (int)blockIdx.x : G;
+    db0 = s0 / a.H; dh0 = s0 - db0 * a.H;
+    db1 = s1 / a.H; dh1 = s1 - db1 * a.H;
+    odd = 0;
+    sw = 0;
+    len = p < a.q_pairs ? ld_early(a.cache_len + b) : 0;
+  }
+  // Advances to the next item that exists (a sequence of 256 p rows or fewer has no pair p).
+  __device__ __forceinline__ bool next(AtItem& I) {
+    for (;;) {
+      if (p >= a.q_pairs) return false;
+      const int cp = p, cb = b, ch = h, clen = len;
+      h += odd ? dh1 : dh0;
+      b += odd ? db1 : db0;
+      odd ^= 1;
+      if (h >= a.H) { h -= a.H; ++b; }
+      while (b >= a.B) { b -= a.B; ++p; }
+      if (p < a.q_pairs) len = ld_early(a.cache_len + b);
+      I.b = cb;
+      I.h = ch;
+      I.n = min(max(clen, 0), min(a.cap, a.n_max));
+      I.q_hi = I.n - cp * a.item_rows;
+      if (I.q_hi <= 0) continue;
+      I.n_kv = (I.q_hi + kAtBN - 1) / kAtBN;
+      I.row_base = (cb * a.H + ch) * a.cap;                         // first row of this (b, h) in the caches
+      I.swap = (kAtSwapLanes && a.item_rows == 2 * kAtBM) ? sw : 0;
+      sw ^= 1;
+      return true;
+    }
+  }
+};
+
+// Whether the two MMA-issuing threads take turns (a lane issues a whole block, P V then the next
+// Q K^T, before the other lane's block is queued).  Measured both ways: with turns the lanes run half a
+// period apart, one lane's softmax hiding behind the other's MMAs, but a single thread cannot keep the
+// tensor pipe fed (a chain of eight dependent MMAs costs its issuer ~200 cycles of latency on top of
+// 8 x 64, and each completion signal ~90 more) and a softmax warp alone on its scheduler does not
+// overlap its exponentials with its arithmetic.  Without turns the lanes fall into step: both issue
+// at once (the pipe interleaves the two chains at full rate) and both softmax at once (two warps per
+// scheduler interleave).  The second is 3-7 % faster on the shapes at hand, so it is the default.
+constexpr bool kAtTakeTurns = false;
+__device__ __forceinline__ void pipe_lock(int* l, volatile int* abort) {
+  if (!kAtTakeTurns) return;
+  for (int i = 0; atomicCAS(l, 0, 1) != 0; ++i)
+    if (i > kSpinLimitBusy) { *abort = 1; return; }
+}
+__device__ __forceinline__ void pipe_unlock(int* l) { if (kAtTakeTurns) atomicExch(l, 0); }
+
+// Register budget per role (the kernel starts every thread at 168): the producer / MMA warps give
+// registers back, the softmax warps take them to hold a whole score row.
+constexpr int kAtRegsSmall = 72, kAtRegsSoftmax = 216;
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+}  // namespace dl

@@ -40,176 +40,14 @@
 #include "common.cuh"
 #include "tc05.cuh"
 
+#include "attn_prefill.cuh"
+#include "attn_prefill_softmax.cuh"
+
 namespace dl {
 
-constexpr int kAtBM = 128, kAtBN = 128, kAtThreads = 384, kAtRing = 3;
-constexpr int kAtTile = 2 * 128 * 128;                // 32 KB: two [128 rows][64 dims] halves
-constexpr int kAtOffRing = 4 * kAtTile;               // Q: [lane][slot] tiles first
-constexpr int kAtOffBar = kAtOffRing + kAtRing * kAtTile;
-constexpr size_t kAtSmem = kAtOffBar + 512;           // 229888 bytes: one CTA per SM
-constexpr uint32_t kAtColO = 0, kAtColS = 128, kAtLaneCols = 256;   // tensor-memory columns of one lane: O | S
-constexpr float kRescaleStep = 8.0f;                  // log2 units by which the maximum may lag
 
-// 2^x on the special-function unit (x <= 0 here; -inf gives 0)
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-// max of three in one instruction
-__device__ __forceinline__ float fmax3(float x, float y, float z) {
-  float r;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(x), "f"(y), "f"(z));
-  return r;
-}
-
-// two fp32 lanes in one 64-bit register: fused multiply-add and add on both at once
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t ffma2(uint64_t x, uint64_t y, uint64_t z) {
-  uint64_t r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(x), "l"(y), "l"(z));
-  return r;
-}
-__device__ __forceinline__ uint64_t fadd2(uint64_t x, uint64_t y) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(x), "l"(y));
-  return r;
-}
-__device__ __forceinline__ uint64_t fmul2(uint64_t x, uint64_t y) {
-  uint64_t r;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(x), "l"(y));
-  return r;
-}
-
-// Tensor maps: Q, K and V each with boxes of 128, 64, 32 and 16 rows (index 0..3), so that a ragged
-// tile at the end of a sequence is fetched with the smallest box that covers it; O for the stores.
-struct AtMaps {
-  alignas(64) unsigned char q[4][128]; alignas(64) unsigned char k[4][128];
-  alignas(64) unsigned char v[4][128]; alignas(64) unsigned char o[128];
-};
-// index of the smallest box (128 >> index rows) that covers `rows` (a multiple of 16 in 16..128)
-__device__ __forceinline__ int at_box(int rows) { return rows > 64 ? 0 : rows > 32 ? 1 : rows > 16 ? 2 : 3; }
-
-struct AtArgs {
-  const int32_t* cache_len; __nv_bfloat16* out; DeviceStatus* status;
-  int32_t B, H, cap, n_max, q_pairs, item_rows;     // item_rows: query rows per work item (256: a pair of tiles; 128)
-  float scale_log2;
-};
-
-// Work item -> (b, h, pair p of query tiles).  Pair p counts from the sequence's end: it covers rows
-// [q_hi - 256, q_hi) with q_hi = n - 256 p, clipped at row 0; its keys are [0, q_hi) in n_kv tiles.
-struct AtItem { int b, h, q_hi, n, n_kv, row_base, swap; };
-
-// One lane's share of an item: rows [q0, q_hi) are owned (the Q tile is loaded from row q0, 128 rows;
-// a tile clipped at the top of the sequence loads rows [0, 128) and owns the first q_hi of them),
-// keys [0, q_hi) in n_tiles tiles.  The later query tile of a pair has one key tile more than the
-// earlier one, so the lanes swap tiles from one item to the next (I.swap) and do the same work.
-struct AtLane { int q0, q_hi, n_tiles; bool exists; };
-__device__ __forceinline__ AtLane at_lane(const AtItem& I, int lane_id) {
-  AtLane L;
-  L.q_hi = I.q_hi - (lane_id ^ I.swap) * kAtBM;
-  L.exists = L.q_hi > 0;
-  L.q0 = max(L.q_hi - kAtBM, 0);
-  L.n_tiles = (L.q_hi + kAtBN - 1) / kAtBN;
-  return L;
-}
-// keys of tile j that a lane's MMAs cover: all 128, or what is left of [0, q_hi) rounded up to 16
-__device__ __forceinline__ int at_cols(const AtLane& L, int j) {
-  return min(kAtBN, (L.q_hi - j * kAtBN + 15) & ~15);
-}
-
-// A load the compiler may not sink towards its use (the point is to have it in flight early).
-__device__ __forceinline__ int ld_early(const int32_t* p) {
-  int v;
-  asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(p));
-  return v;
-}
-
-// Walks the items of this CTA in the order every role uses: item = p * B * H + b * H + h, stepping by the
-// grid size, so all pairs 0 (the longest) come first.  The position is kept as (p, b, h) and advanced by
-// additions (a division per item and role is what an item's set-up cannot afford); the length of the NEXT
-// item's sequence is requested one item early, so its latency never sits in front of a role's first wait.
-// (Walking head by head instead, all pairs of a head side by side, halves the DRAM reads on long contexts
-// - K and V of a head are then fetched once - but measured 20-60 % slower: the kernel is not DRAM-bound.)
-constexpr bool kAtSwapLanes = true;
-struct AtWalker {
-  const AtArgs& a;
-  int p, b, h, len, db, dh, sw;               // next item, its length (in flight), the step as (db, dh), swap bit
-  __device__ __forceinline__ explicit AtWalker(const AtArgs& a_) : a(a_) {
-    const int bh_count = a.B * a.H;
-    p = (int)blockIdx.x / bh_count;
-    const int bh = (int)blockIdx.x - p * bh_count;
-    b = bh / a.H;
-    h = bh - b * a.H;
-    db = (int)gridDim.x / a.H;
-    dh = (int)gridDim.x - db * a.H;
-    sw = 0;
-    len = p < a.q_pairs ? ld_early(a.cache_len + b) : 0;
-  }
-  // Advances to the next item that exists (a sequence of 256 p rows or fewer has no pair p).
-  __device__ __forceinline__ bool next(AtItem& I) {
-    for (;;) {
-      if (p >= a.q_pairs) return false;
-      const int cp = p, cb = b, ch = h, clen = len;
-      h += dh;
-      b += db;
-      if (h >= a.H) { h -= a.H; ++b; }
-      while (b >= a.B) { b -= a.B; ++p; }
-      if (p < a.q_pairs) len = ld_early(a.cache_len + b);
-      I.b = cb;
-      I.h = ch;
-      I.n = min(max(clen, 0), min(a.cap, a.n_max));
-      I.q_hi = I.n - cp * a.item_rows;
-      if (I.q_hi <= 0) continue;
-      I.n_kv = (I.q_hi + kAtBN - 1) / kAtBN;
-      I.row_base = (cb * a.H + ch) * a.cap;                         // first row of this (b, h) in the caches
-      I.swap = (kAtSwapLanes && a.item_rows == 2 * kAtBM) ? sw : 0;
-      sw ^= 1;
-      return true;
-    }
-  }
-};
-
-// Whether the two MMA-issuing threads take turns (a lane issues a whole block, P V then the next
-// Q K^T, before the other lane's block is queued).  Measured both ways: with turns the lanes run half a
-// period apart, one lane's softmax hiding behind the other's MMAs, but a single thread cannot keep the
-// tensor pipe fed (a chain of eight dependent MMAs costs its issuer ~200 cycles of latency on top of
-// 8 x 64, and each completion signal ~90 more) and a softmax warp alone on its scheduler does not
-// overlap its exponentials with its arithmetic.  Without turns the lanes fall into step: both issue
-// at once (the pipe interleaves the two chains at full rate) and both softmax at once (two warps per
-// scheduler interleave).  The second is 3-7 % faster on the shapes at hand, so it is the default.
-constexpr bool kAtTakeTurns = false;
-__device__ __forceinline__ void pipe_lock(int* l, volatile int* abort) {
-  if (!kAtTakeTurns) return;
-  for (int i = 0; atomicCAS(l, 0, 1) != 0; ++i)
-    if (i > kSpinLimitBusy) { *abort = 1; return; }
-}
-__device__ __forceinline__ void pipe_unlock(int* l) { if (kAtTakeTurns) atomicExch(l, 0); }
-
-// Register budget per role (the kernel starts every thread at 168): the producer / MMA warps give
-// registers back, the softmax warps take them to hold a whole score row.
-constexpr int kAtRegsSmall = 72, kAtRegsSoftmax = 216;
-template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-
-// SUB = 1: a lane works on whole 128-key tiles (one S buffer; softmax and MMAs of a lane alternate).
-// SUB = 2: a lane works on 64-key half tiles with two S buffers of 64 columns, so the Q K^T of the next
-// half tile runs while the softmax works on this one.  An MMA of N = 64 costs the tensor pipe as much as
-// one of N = 128, so this trades pipe time (and twice the hand-overs) for overlap; measured, it loses:
-// 447 against 481 TFLOP/s at 832 rows, 373 against 401 at ~1650.  Kept selectable, not the default.
-template <int SUB>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
-  constexpr int Wd = kAtBN / SUB;                      // keys per sub-tile = columns of one S buffer
-  constexpr int NCH = Wd / 32;                         // 32-column chunks per sub-tile
   extern __shared__ __align__(1024) char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (smem_u32(smem) & 1023u) {                        // the swizzled tiles need 1024-byte alignment
@@ -221,9 +59,9 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
   // Ring tile T of this CTA (running count over its items; K and V of key tile j of an item are tiles
   // base + 2j and base + 2j + 1) lives in slot T % 3 and completes phase (T / 3) & 1 of that slot's
   // `full` barrier; lane X's MMAs that read it complete a phase of the slot's `free_X` barrier.
-  // A lane's own barriers: its g-th sub-tile (running count) uses S buffer g % SUB and completes phase
-  // (g / SUB) & 1 of that buffer's s_full / p_full / pv_done (per buffer, so that a waiter is never two
-  // phases behind: before sub-tile g's S is ready, the P V of g - SUB has completed); its i-th item completes
+  // A lane's own barriers: its g-th key tile (running count) completes phase g & 1 of s_full / p_full /
+  // pv_done (a waiter is never two phases behind: before tile g's S is ready, the P V of g - 1 has
+  // completed); its i-th item completes
   // phase i & 1 of o_free and phase (i >> 1) & 1 of q_full / q_done of Q slot i & 1.
   auto ring_full = [&](int s) { return smem_u32(bars + s); };
   auto ring_free = [&](int x, int s) { return smem_u32(bars + 3 + 3 * x + s); };
@@ -381,25 +219,28 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         }
         const int qs = n_item & 1;
         const uint64_t q_desc = smem_desc_sw128(smem_u32(smem + (2 * x + qs) * kAtTile));
-        // Sub-tile u of the item covers keys [u Wd, u Wd + sub_cols(u)): it is half u % SUB of ring tile
-        // pair u / SUB and uses S buffer (g0 + u) % SUB.
-        const int n_sub = (L.q_hi + Wd - 1) / Wd;
-        auto sub_cols = [&](int u) { return min(Wd, (L.q_hi - u * Wd + 15) & ~15); };
+        const int n_sub = L.n_tiles;
+        auto sub_cols = [&](int u) { return at_cols(L, u); };
         auto issue_qk = [&](int u) {
-          const int s = (T0 + 2 * (u / SUB)) % kAtRing;
-          const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile) + (u % SUB) * (Wd * 128));
+          const int s = (T0 + 2 * u) % kAtRing;
+          const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile));
           const uint32_t idesc_qk = idesc_bf16(kAtBM, (uint32_t)sub_cols(u));
-          const uint32_t d = t_s + ((g0 + u) % SUB) * Wd;
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            mma_ss(d, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
-                   k_desc + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
+          // not unrolled (an MMA holds the thread for 64 cycles anyway; short code is what counts here): 16 dims
+          // further per step, and from the fourth step on in the tile's second 64-dim half
+          uint64_t qd = q_desc, kd = k_desc;
+#pragma unroll 1
+          for (int ks = 0; ks < 8; ++ks) {
+            mma_ss(t_s, qd, kd, idesc_qk, ks != 0);
+            const uint64_t step = (ks == 3) ? (uint64_t)((kAtBM * 128 - 96) >> 4) : 2ull;
+            qd += step;
+            kd += step;
+          }
         };
         // Completion signals: a commit covers every MMA this thread has issued so far.  The K tile is
         // released by the Q K^T of its last sub-tile.
         auto commit_qk = [&](int u) {
-          mma_commit(s_full(x, (g0 + u) % SUB));                       // first: the softmax warps wait on it
-          if (u % SUB == SUB - 1 || u == n_sub - 1) mma_commit(ring_free(x, (T0 + 2 * (u / SUB)) % kAtRing));
+          mma_commit(s_full(x, 0));                       // first: the softmax warps wait on it
+          mma_commit(ring_free(x, (T0 + 2 * u) % kAtRing));
         };
         mbar_wait_spin(q_full(x, qs), (n_item >> 1) & 1, abort_flag);
         wait_ring(T0);
@@ -408,21 +249,17 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         issue_qk(0);
         pipe_unlock(pipe_turn);
         commit_qk(0);
-        if (SUB == 2 && n_sub > 1) {                                   // the second S buffer: same K tile
-          issue_qk(1);
-          commit_qk(1);
-        }
         for (int u = 0; u < n_sub; ++u) {
-          const int g = g0 + u, b = g % SUB;
-          const int T = T0 + 2 * (u / SUB) + 1, s = T % kAtRing;       // the V tile of this sub-tile
-          const int un = u + SUB;                                      // the sub-tile whose Q K^T reuses this S buffer
+          const int g = g0 + u, b = 0;
+          const int T = T0 + 2 * u + 1, s = T % kAtRing;                 // the V tile of this key tile
+          const int un = u + 1;                                          // the tile whose Q K^T reuses the S buffer
           // operands first (they land long before), then the softmax's hand-over
           wait_ring(T);
-          if (un < n_sub) wait_ring(T0 + 2 * (un / SUB));
+          if (un < n_sub) wait_ring(T0 + 2 * un);
           if (u == 0) mbar_wait_spin(o_free(x), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
           // polled without suspending: the wake-up of a suspended wait costs this thread ~600 cycles per tile
           {
-            const uint32_t pb = p_full(x, b), ph = (uint32_t)(g / SUB) & 1u;
+            const uint32_t pb = p_full(x, b), ph = (uint32_t)g & 1u;
             int spins = 0;
             while (!mbar_test(pb, ph)) {
               if ((++spins & 1023) == 0 && (*abort_flag || spins > (kSpinLimitBusy << 4))) { *abort_flag = 1; break; }
@@ -430,16 +267,16 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           }
           tc_fence_after();
           const uint64_t v_desc =
-              smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128) + (uint64_t)(((u % SUB) * Wd * 128) >> 4);
+              smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128);
           const int ksteps = sub_cols(u) >> 4;
           pipe_lock(pipe_turn, abort_flag);
           for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(t_o, t_s + b * Wd + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv, (u | ks) != 0);
+            mma_ts(t_o, t_s + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv, (u | ks) != 0);
           if (un < n_sub) issue_qk(un);                                // overwrites P: in order behind the P V
           pipe_unlock(pipe_turn);
           if (un < n_sub) commit_qk(un);
           mma_commit(pv_done(x, b));
-          if (u % SUB == SUB - 1 || u == n_sub - 1) mma_commit(ring_free(x, s));
+          mma_commit(ring_free(x, s));
         }
         pass_tiles(T0 + 2 * L.n_tiles, T0 + 2 * I.n_kv);
         g0 += n_sub;
@@ -467,108 +304,21 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       const int grow = L.q0 + row;                                     // row within the sequence
       const int r0 = L.q0 + quad * 32;                                 // this warp's first row
       float m_used = -INFINITY, l_run = 0.f;
-      const int n_sub = (L.q_hi + Wd - 1) / Wd;
+      const int n_sub = L.n_tiles;
       for (int u = 0; u < n_sub; ++u) {
-        const int g = g0 + u, sbuf = g % SUB;
-        const int c0 = u * Wd;
-        const uint32_t sa = s_addr + sbuf * Wd;                         // this sub-tile's S buffer
+        const int g = g0 + u, sbuf = 0;
+        const int c0 = u * kAtBN;
+        const uint32_t sa = s_addr;
         // 32-column chunks of this sub-tile that some row of the warp may see
-        const int n_ch = min(NCH, (min(L.q_hi, r0 + 32) - c0 + 31) >> 5);
-        mbar_wait_spin(s_full(x, sbuf), (g / SUB) & 1, abort_flag);
+        const int n_ch = min(4, (min(L.q_hi, r0 + 32) - c0 + 31) >> 5);
+        mbar_wait_spin(s_full(x, sbuf), g & 1, abort_flag);
         tc_fence_after();
-        // ---- one pass over the tile in 32-column chunks, the next chunk's load in flight while this one is
-        // worked on.  Exponentials are taken against the maximum the row already uses (the first chunk's
-        // own maximum on an item's first tile); the tile's true maximum is tracked alongside, and only if
-        // it turns out more than 2^8 above the one used is the tile done again after rescaling O.
-        uint32_t pw[16 * NCH];                                          // P of the row, bf16 pairs
-        const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2);
-        const int vis = grow - c0;                                      // columns 0..vis are visible to this row
-        float mx_tile;
-        bool first_try = true;
-        for (;;) {
-          uint32_t buf[2][32];
-          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}; // four independent chains
-          uint64_t l2[2] = {0ull, 0ull};                                // two chains of packed row sums
-          if (n_ch > 0) tmem_ld32(sa, buf[0]);
-          tmem_ld_wait();
-#pragma unroll
-          for (int cc = 0; cc < NCH; ++cc) {
-            uint32_t* sr = buf[cc & 1];
-            if (n_ch > cc) {
-              if (n_ch > cc + 1) tmem_ld32(sa + 32 * (cc + 1), buf[(cc + 1) & 1]);
-              if (c0 + 32 * cc + 31 > r0) {                             // the chunk reaches past the warp's first row
-#pragma unroll
-                for (int c = 0; c < 32; ++c)
-                  if (32 * cc + c > vis) sr[c] = 0xFF800000u;           // -inf
-              }
-#pragma unroll
-              for (int c = 0; c < 32; c += 8) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                  mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
-              }
-              if (cc == 0 && u == 0 && first_try)                       // column 0 is visible to every row: finite
-                m_used = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-              const uint64_t nm2 = pack2(-m_used, -m_used);
-#pragma unroll
-              for (int c = 0; c < 16; ++c) {
-                float p0, p1;
-                unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
-                p0 = fast_exp2(p0);
-                p1 = fast_exp2(p1);
-                l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
-                __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                pw[16 * cc + c] = *reinterpret_cast<uint32_t*>(&pk);
-              }
-              tmem_ld_wait();
-            } else {
-#pragma unroll
-              for (int c = 0; c < 16; ++c) pw[16 * cc + c] = 0u;
-            }
-          }
-          mx_tile = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-          const bool need = grow < L.q_hi && mx_tile > m_used + kRescaleStep;   // rows the tile does not own hold stale data
-          if (!__any_sync(0xffffffffu, need)) {
-            float la, lb;
-            unpack2(fadd2(l2[0], l2[1]), la, lb);
-            l_run += la + lb;
-            break;
-          }
-          // rare: raise the maximum (rescaling what O and the row sum hold so far), then redo the tile
-          first_try = false;
-          const float corr = need ? fast_exp2(m_used - mx_tile) : 1.0f;
-          if (need) m_used = mx_tile;
-          if (u > 0) {
-            // O must be at rest: the P V of the previous sub-tile
-            mbar_wait_spin(pv_done(x, (g - 1) % SUB), ((g - 1) / SUB) & 1, abort_flag);
-            tc_fence_after();
-            l_run *= corr;
-            const uint64_t corr2 = pack2(corr, corr);
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-              uint32_t o[32];
-              tmem_ld32(o_addr + cc * 32, o);
-              tmem_ld_wait();
-#pragma unroll
-              for (int i = 0; i < 32; i += 2) {
-                float y0, y1;
-                unpack2(fmul2(pack2(__uint_as_float(o[i]), __uint_as_float(o[i + 1])), corr2), y0, y1);
-                o[i] = __float_as_uint(y0);
-                o[i + 1] = __float_as_uint(y1);
-              }
-              tmem_st32(o_addr + cc * 32, o);
-            }
-            tmem_st_wait();
-          }
-        }
-        tmem_st32(sa, pw);                                             // P (bf16) over the first half of its S buffer
-        if (NCH == 4) tmem_st32(sa + 32, pw + 32 * (NCH / 4));
-        tmem_st_wait();
+        at_softmax_halves<1>(sa, o_addr, n_ch, grow - c0, c0 - r0, grow < L.q_hi, u > 0, a.scale_log2, m_used, l_run);
         if (u == n_sub - 1 && L.q_hi == I.n) {
           // last tile of the sequence (only lane A of pair 0 gets here): the P V covers keys up to the next
           // multiple of 16; zero the V rows between the sequence's end and that bound (both 64-dim halves).
           // Other query tiles need nothing: rows past their end are the sequence's own and P is 0 there.
-          const int j = u / SUB;                                       // in rows of the 128-key ring tile
+          const int j = u;
           const int valid = I.n - j * kAtBN, pad = at_cols(L, j) - valid;
           if (pad > 0) {
             const int T = T0 + 2 * j + 1, s = T % kAtRing;
@@ -593,7 +343,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       // ---- epilogue: O / l -> bf16 -> out[b][row][h][:], 32 columns at a time, staged in this warp's 8 KB of
       // the item's Q slot (16-byte units XOR-swizzled by row pair: the 64-byte swizzle of the tensor map)
       const int gl = g0 + n_sub - 1;
-      mbar_wait_spin(pv_done(x, gl % SUB), (gl / SUB) & 1, abort_flag);   // MMAs complete in order: all of O is in
+      mbar_wait_spin(pv_done(x, 0), gl & 1, abort_flag);   // MMAs complete in order: all of O is in
       tc_fence_after();
       const float inv = 1.0f / l_run;
       const int rows_here = L.q_hi - r0;                               // owned rows among this warp's 32
@@ -601,32 +351,25 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       const int qs = n_item & 1;
       char* so = smem + (2 * x + qs) * kAtTile + quad * 8192;
       __nv_bfloat16* otile = a.out + (((size_t)I.b * a.n_max + r0) * a.H + I.h) * 128;
-      {
-        uint32_t ob[2][32];                              // the next 32 columns load while these are converted
-        tmem_ld32(o_addr, ob[0]);
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {                   // not unrolled: once per item, short code counts for more
+        uint32_t o[32];
+        tmem_ld32(o_addr + cc * 32, o);
         tmem_ld_wait();
+        if (cc == 3) {                                   // all of O is in registers: the next item may overwrite it
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(o_free(x));
+        }
+        char* sb = so + cc * 2048;
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          const uint32_t* o = ob[cc & 1];
-          if (cc < 3) tmem_ld32(o_addr + (cc + 1) * 32, ob[(cc + 1) & 1]);
-          char* sb = so + cc * 2048;
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            uint4 w;
-            __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[8 * u]) * inv, __uint_as_float(o[8 * u + 1]) * inv);
-            __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 2]) * inv, __uint_as_float(o[8 * u + 3]) * inv);
-            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 4]) * inv, __uint_as_float(o[8 * u + 5]) * inv);
-            __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
-            w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
-            w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
-            *reinterpret_cast<uint4*>(sb + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
-          }
-          if (cc < 3) tmem_ld_wait();
-          if (cc == 2) {                                 // all of O is in registers: the next item may overwrite it
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(o_free(x));
-          }
+        for (int u = 0; u < 4; ++u) {
+          uint4 w;
+          w.x = cvt_bf16x2(__uint_as_float(o[8 * u]) * inv, __uint_as_float(o[8 * u + 1]) * inv);
+          w.y = cvt_bf16x2(__uint_as_float(o[8 * u + 2]) * inv, __uint_as_float(o[8 * u + 3]) * inv);
+          w.z = cvt_bf16x2(__uint_as_float(o[8 * u + 4]) * inv, __uint_as_float(o[8 * u + 5]) * inv);
+          w.w = cvt_bf16x2(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
+          *reinterpret_cast<uint4*>(sb + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
         }
       }
       if (whole) {
@@ -665,482 +408,12 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
   if (warp == 11) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
-// ---------------------------------------------------------------------------------------------------
-// Variant with P in shared memory and the score buffer released early.
-// Same roles, items, lanes and ring protocol as the kernel above; what differs is the hand-over
-// between a lane's softmax warps and its MMA-issuing thread:
-//   * a softmax warp works on the tile's two 64-column halves in turn, out of registers; the second
-//     half's scores are loaded as soon as the first half's P is final, and the S buffer is released
-//     right then (s_free), so the NEXT tile's Q K^T runs on the tensor pipe while this tile's second
-//     half is worked on: S of the next tile is complete when the softmax asks for it, and a lane's
-//     softmax warps work back to back instead of waiting for P V + Q K^T between tiles;
-//   * P does not alias S any more: it goes, as bf16, into a 16 KB shared-memory buffer of the lane
-//     (K-major, 128-byte swizzle: the A operand of an SS MMA), one 64-key HALF of the tile at a time.
-//     The first half's P V runs while the second half's exponentials are taken; each half checks
-//     its own maximum against the one in use (rescale-and-redo as above, per half);
-//   * shared memory: Q one slot per lane (released by the item's last Q K^T, which is issued a whole
-//     softmax period before the item ends, so the next Q load still hides), P 16 KB per lane, and
-//     a ring of FOUR K/V tiles: K of tile u+1 is wanted while V of tile u-1 may still be in use;
-//   * the output is staged in the warp's own rows of the P buffer, two 32-column blocks at a time.
-// Measured on B200 it does not pay: 461 against 481-508 TFLOP/s at 832 rows, 193 against 201 at 272.
-// An SS MMA of 128 x 128 x 16 reads 8 KB of shared memory in its 64 cycles, which is all the bandwidth
-// shared memory has; P V from shared memory (instead of tensor memory) adds 4 KB per MMA and the P
-// stores 32 KB per tile on top, so the MMAs, the P stores (~50 cycles per 16-byte store) and the
-// completion signals all slow down, and the time won between tiles is lost inside them.  Kept as a
-// tested option; the kernel above stays the default.
-constexpr int kApRing = 4;
-constexpr int kApPBytes = 128 * 128;                  // one [128 rows][64 keys] bf16 block
-constexpr int kApOffP = 2 * kAtTile;                  // Q of lane 0, Q of lane 1, then the two P buffers
-constexpr int kApOffRing = kApOffP + 2 * kApPBytes;
-constexpr int kApOffBar = kApOffRing + kApRing * kAtTile;
-constexpr size_t kApSmem = kApOffBar + 512;
-static_assert(kApSmem <= kAtSmem, "the variant must fit the same shared-memory budget");
-
 // Polls a barrier without suspending the thread (hand-overs that are a few hundred cycles apart).
 __device__ __forceinline__ void mbar_poll(uint32_t bar, uint32_t parity, volatile int* abort) {
   int spins = 0;
   while (!mbar_test(bar, parity)) {
     if ((++spins & 1023) == 0 && (*abort || spins > (kSpinLimitBusy << 4))) { *abort = 1; break; }
   }
-}
-
-__global__ void __launch_bounds__(kAtThreads, 1)
-attn_prefill_tcp_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
-  extern __shared__ __align__(1024) char smem[];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (smem_u32(smem) & 1023u) {
-    if (tid == 0) report_status(a.status, DL_ERR_ALIGNMENT, -1);
-    return;
-  }
-  char* ring_s = smem + kApOffRing;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kApOffBar);
-  // Ring tile T (running count; K and V of key tile j of an item are tiles base + 2j, base + 2j + 1)
-  // lives in slot T % 4 and completes phase (T / 4) & 1 of the slot's barriers.  A lane's g-th tile
-  // (running count) completes phase g & 1 of s_full / s_free; its halves 2g and 2g + 1 complete
-  // phases of p_full / pv_done in turn; its i-th item completes phase i & 1 of q_full / q_free / o_free.
-  auto ring_full = [&](int s) { return smem_u32(bars + s); };
-  auto ring_free = [&](int x, int s) { return smem_u32(bars + 4 + 4 * x + s); };
-  auto q_full = [&](int x) { return smem_u32(bars + 12 + x); };    // Q tile has landed
-  auto q_free = [&](int x) { return smem_u32(bars + 14 + x); };    // the item's last Q K^T has read it
-  auto s_full = [&](int x) { return smem_u32(bars + 16 + x); };    // Q K^T has completed: S ready
-  auto s_free = [&](int x) { return smem_u32(bars + 18 + x); };    // S is in registers (4 warps)
-  auto p_full = [&](int x) { return smem_u32(bars + 20 + x); };    // half a tile of P is in shared memory (4 warps)
-  auto pv_done = [&](int x) { return smem_u32(bars + 22 + x); };   // that half's P V has completed
-  auto o_free = [&](int x) { return smem_u32(bars + 24 + x); };    // the epilogue has read O (4 warps)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
-
-  if (tid == 0) {
-    *abort_flag = 0;
-    for (int s = 0; s < kApRing; ++s) {
-      mbar_init(ring_full(s), 1);
-      mbar_init(ring_free(0, s), 1);
-      mbar_init(ring_free(1, s), 1);
-    }
-    for (int x = 0; x < 2; ++x) {
-      mbar_init(q_full(x), 1); mbar_init(q_free(x), 1);
-      mbar_init(s_full(x), 1); mbar_init(s_free(x), 4);
-      mbar_init(p_full(x), 4); mbar_init(pv_done(x), 1);
-      mbar_init(o_free(x), 4);
-    }
-    fence_mbar_init();
-  }
-  if (warp == 11) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-
-  if (warp == 8) {
-    // ---------------------------------------------------------------- TMA producer
-    reg_dec<kAtRegsSmall>();
-    if (lane == 0) {
-      for (int i = 0; i < 4; ++i) {
-        tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.q[i]));
-        tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.k[i]));
-        tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.v[i]));
-      }
-      AtWalker Wr(a);
-      AtItem Ir;
-      int T = 0, jr = 0;
-      AtWalker Wq0 = Wr, Wq1 = Wr;
-      AtItem Iq[2];
-      bool hq[2];
-      int nq[2] = {0, 0};
-      bool hr = Wr.next(Ir);
-      hq[0] = Wq0.next(Iq[0]);
-      hq[1] = Wq1.next(Iq[1]);
-      while (hq[0] && !at_lane(Iq[0], 0).exists) hq[0] = Wq0.next(Iq[0]);
-      while (hq[1] && !at_lane(Iq[1], 1).exists) hq[1] = Wq1.next(Iq[1]);
-      int idle = 0;
-      while ((hr || hq[0] || hq[1]) && !*abort_flag) {
-        bool prog = false;
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          if (!hq[x]) continue;
-          if (nq[x] >= 1 && !mbar_test(q_free(x), (nq[x] - 1) & 1)) continue;
-          const AtLane L = at_lane(Iq[x], x);
-          char* dst = smem + x * kAtTile;
-          const int bx = at_box(min(kAtBM, (L.q_hi - L.q0 + 15) & ~15));
-          const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(maps.q[bx]);
-          mbar_expect_tx(q_full(x), kAtTile >> bx);
-          tma_load_2d(smem_u32(dst), mq, 0, Iq[x].row_base + L.q0, q_full(x));
-          tma_load_2d(smem_u32(dst + kAtBM * 128), mq, 64, Iq[x].row_base + L.q0, q_full(x));
-          ++nq[x];
-          if (x == 0) {
-            hq[0] = Wq0.next(Iq[0]);
-            while (hq[0] && !at_lane(Iq[0], 0).exists) hq[0] = Wq0.next(Iq[0]);
-          } else {
-            hq[1] = Wq1.next(Iq[1]);
-            while (hq[1] && !at_lane(Iq[1], 1).exists) hq[1] = Wq1.next(Iq[1]);
-          }
-          prog = true;
-        }
-        if (hr) {
-          const int s = T % kApRing;
-          bool slot_free = true;
-          if (T >= kApRing) {
-            const uint32_t par = (uint32_t)(T / kApRing - 1) & 1u;
-            slot_free = mbar_test(ring_free(0, s), par) && mbar_test(ring_free(1, s), par);
-          }
-          if (slot_free) {
-            const int j = jr >> 1;
-            char* dst = ring_s + s * kAtTile;
-            const int bx = at_box(min(kAtBN, (Ir.q_hi - j * kAtBN + 15) & ~15));
-            const CUtensorMap* m = reinterpret_cast<const CUtensorMap*>((jr & 1) ? maps.v[bx] : maps.k[bx]);
-            const int r = Ir.row_base + j * kAtBN;
-            mbar_expect_tx(ring_full(s), kAtTile >> bx);
-            tma_load_2d(smem_u32(dst), m, 0, r, ring_full(s));
-            tma_load_2d(smem_u32(dst + kAtBN * 128), m, 64, r, ring_full(s));
-            ++T;
-            if (++jr == 2 * Ir.n_kv) { jr = 0; hr = Wr.next(Ir); }
-            prog = true;
-          }
-        }
-        if (prog) {
-          idle = 0;
-        } else if (++idle > kSpinLimitBusy) {
-          *abort_flag = 1;
-        }
-      }
-      if (*abort_flag) {
-        // every copy that was issued must land before the CTA's shared memory is released
-        report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
-        for (int t = max(0, T - kApRing); t < T; ++t)
-          for (int i = 0; i < kSpinLimit && !mbar_try_wait(ring_full(t % kApRing), (t / kApRing) & 1); ++i) __nanosleep(40);
-        for (int x = 0; x < 2; ++x)
-          if (nq[x] > 0)
-            for (int i = 0; i < kSpinLimit && !mbar_try_wait(q_full(x), (nq[x] - 1) & 1); ++i) __nanosleep(40);
-      }
-    }
-  } else if (warp == 9 || warp == 10) {
-    // ---------------------------------------------------------------- MMA issuer of one lane
-    reg_dec<kAtRegsSmall>();
-    if (lane == 0) {
-      const int x = warp - 9;
-      const uint32_t t_o = tmem + x * kAtLaneCols + kAtColO, t_s = tmem + x * kAtLaneCols + kAtColS;
-      const uint32_t idesc_pv = idesc_bf16(kAtBM, 128, 0, 1);          // A (= P) K-major, B (= V) MN-major
-      const uint64_t q_desc = smem_desc_sw128(smem_u32(smem + x * kAtTile));
-      const uint64_t p_desc = smem_desc_sw128(smem_u32(smem + kApOffP + x * kApPBytes));
-      AtWalker W(a);
-      AtItem I;
-      int n_item = 0, g0 = 0, T0 = 0;
-      while (W.next(I)) {
-        const AtLane L = at_lane(I, x);
-        auto wait_ring = [&](int T) { mbar_wait_spin(ring_full(T % kApRing), (T / kApRing) & 1, abort_flag); };
-        auto pass_tiles = [&](int from, int to) {
-          for (int T = from; T < to; ++T) {
-            wait_ring(T);
-            mbar_arrive(ring_free(x, T % kApRing));
-          }
-        };
-        if (!L.exists) {
-          pass_tiles(T0, T0 + 2 * I.n_kv);
-          T0 += 2 * I.n_kv;
-          continue;
-        }
-        const int n_t = L.n_tiles;
-        // S = Q K^T of tile u, once its K tile has landed and the softmax warps hold the previous S in registers
-        auto issue_qk = [&](int u) {
-          const int T = T0 + 2 * u, s = T % kApRing, g = g0 + u;
-          wait_ring(T);
-          if (g > 0) mbar_poll(s_free(x), (uint32_t)(g - 1) & 1u, abort_flag);
-          tc_fence_after();
-          const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile));
-          const uint32_t idesc_qk = idesc_bf16(kAtBM, (uint32_t)at_cols(L, u));
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            mma_ss(t_s, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
-                   k_desc + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
-          mma_commit(s_full(x));                                        // first: the softmax warps wait on it
-          mma_commit(ring_free(x, s));
-          if (u == n_t - 1) mma_commit(q_free(x));                      // the Q slot may take the next item's tile
-        };
-        mbar_wait_spin(q_full(x), n_item & 1, abort_flag);
-        issue_qk(0);
-        for (int u = 0; u < n_t; ++u) {
-          const int g = g0 + u;
-          const int T = T0 + 2 * u + 1, s = T % kApRing;                // the V tile
-          wait_ring(T);
-          if (u == 0) mbar_wait_spin(o_free(x), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
-          const uint64_t v_desc = smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128);
-          const int cols = at_cols(L, u);
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            const int ksteps = max(0, min(cols - 64 * hf, 64)) >> 4;
-            mbar_poll(p_full(x), (uint32_t)(2 * g + hf) & 1u, abort_flag);
-            tc_fence_after();
-            for (int ks = 0; ks < ksteps; ++ks)
-              mma_ss(t_o, p_desc + (uint64_t)((ks * 32) >> 4), v_desc + (uint64_t)(((hf * 4 + ks) * 2048) >> 4), idesc_pv,
-                     (u | hf | ks) != 0);
-            mma_commit(pv_done(x));
-            // S was released together with the first half's P: the next tile's Q K^T runs while the softmax
-            // works on this tile's second half
-            if (hf == 0 && u + 1 < n_t) issue_qk(u + 1);
-          }
-          mma_commit(ring_free(x, s));
-        }
-        pass_tiles(T0 + 2 * L.n_tiles, T0 + 2 * I.n_kv);
-        g0 += n_t;
-        ++n_item;
-        T0 += 2 * I.n_kv;
-      }
-    }
-  } else if (warp < 8) {
-    // ---------------------------------------------------------------- softmax / epilogue warps of one lane
-    reg_inc<kAtRegsSoftmax>();
-    const int x = warp >> 2;
-    const int quad = warp & 3;
-    const int row = quad * 32 + lane;
-    const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
-    const uint32_t s_addr = tmem + lane_off + x * kAtLaneCols + kAtColS;
-    const uint32_t o_addr = tmem + lane_off + x * kAtLaneCols + kAtColO;
-    const CUtensorMap* mo = reinterpret_cast<const CUtensorMap*>(maps.o);
-    char* p_s = smem + kApOffP + x * kApPBytes;                        // the lane's P buffer
-    char* p_row = p_s + row * 128;                                     // this thread's row of it
-    char* so = p_s + quad * 4096;                                      // the warp's rows: also its output staging
-    const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2);
-    AtWalker W(a);
-    AtItem I;
-    int n_item = 0, g0 = 0, T0 = 0;
-    bool stores_pending = false;                                       // staged output still being read by TMA stores
-    while (W.next(I)) {
-      const AtLane L = at_lane(I, x);
-      if (!L.exists) { T0 += 2 * I.n_kv; continue; }
-      const int grow = L.q0 + row;
-      const int r0 = L.q0 + quad * 32;
-      float m_used = -INFINITY, l_run = 0.f;
-      const int n_t = L.n_tiles;
-      for (int u = 0; u < n_t; ++u) {
-        const int g = g0 + u, c0 = u * kAtBN;
-        const int cols = at_cols(L, u);
-        const int n_ch = min(4, (min(L.q_hi, r0 + 32) - c0 + 31) >> 5);  // chunks some row of the warp may see
-        const int vis = grow - c0;
-        uint32_t S[64];                                                // the 64 score columns of the half at hand
-        mbar_poll(s_full(x), g & 1, abort_flag);
-        tc_fence_after();
-        tmem_ld32(s_addr, S);                                          // n_ch >= 1
-        if (n_ch > 1) tmem_ld32(s_addr + 32, S + 32);
-        tmem_ld_wait();
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          const int gh = 2 * g + hf;
-          const bool used = 64 * hf < cols;                            // the P V reads this half
-          uint32_t pw[32];
-          if (used) {
-            bool first_try = true;
-            for (;;) {
-              float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-              uint64_t l2[2] = {0ull, 0ull};
-#pragma unroll
-              for (int c2 = 0; c2 < 2; ++c2) {
-                const int cc = 2 * hf + c2;
-                uint32_t* sr = S + 32 * c2;
-                if (cc < n_ch) {
-                  if (c0 + 32 * cc + 31 > r0) {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                      if (32 * cc + c > vis) sr[c] = 0xFF800000u;      // -inf
-                  }
-#pragma unroll
-                  for (int c = 0; c < 32; c += 8) {
-#pragma unroll
-                    for (int w = 0; w < 4; ++w)
-                      mx4[w] = fmax3(mx4[w], __uint_as_float(sr[c + 2 * w]), __uint_as_float(sr[c + 2 * w + 1]));
-                  }
-                  if (cc == 0 && u == 0 && first_try)                  // column 0 is visible to every row: finite
-                    m_used = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-                  const uint64_t nm2 = pack2(-m_used, -m_used);
-#pragma unroll
-                  for (int c = 0; c < 16; ++c) {
-                    float p0, p1;
-                    unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
-                    p0 = fast_exp2(p0);
-                    p1 = fast_exp2(p1);
-                    l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
-                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                    pw[16 * c2 + c] = *reinterpret_cast<uint32_t*>(&pk);
-                  }
-                } else {
-#pragma unroll
-                  for (int c = 0; c < 16; ++c) pw[16 * c2 + c] = 0u;
-                }
-              }
-              const float mx_half = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-              const bool need = grow < L.q_hi && mx_half > m_used + kRescaleStep;
-              if (!__any_sync(0xffffffffu, need)) {
-                float la, lb;
-                unpack2(fadd2(l2[0], l2[1]), la, lb);
-                l_run += la + lb;
-                break;
-              }
-              // rare: raise the maximum (rescaling what O and the row sum hold so far), then redo the half
-              first_try = false;
-              const float corr = need ? fast_exp2(m_used - mx_half) : 1.0f;
-              if (need) m_used = mx_half;
-              if (gh > 2 * g0) {
-                mbar_wait_spin(pv_done(x), (gh - 1) & 1, abort_flag);   // O must be at rest
-                tc_fence_after();
-                l_run *= corr;
-                const uint64_t corr2 = pack2(corr, corr);
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                  uint32_t o[32];
-                  tmem_ld32(o_addr + cc * 32, o);
-                  tmem_ld_wait();
-#pragma unroll
-                  for (int i = 0; i < 32; i += 2) {
-                    float y0, y1;
-                    unpack2(fmul2(pack2(__uint_as_float(o[i]), __uint_as_float(o[i + 1])), corr2), y0, y1);
-                    o[i] = __float_as_uint(y0);
-                    o[i + 1] = __float_as_uint(y1);
-                  }
-                  tmem_st32(o_addr + cc * 32, o);
-                }
-                tmem_st_wait();
-              }
-            }
-          }
-          if (hf == 0) {                                               // the second half's scores, in flight from here
-            if (n_ch > 2) tmem_ld32(s_addr + 64, S);
-            if (n_ch > 3) tmem_ld32(s_addr + 96, S + 32);
-          }
-          // the P buffer is free once the previous half's P V has completed (every half waits, used or
-          // not, so that no phase of the barrier goes unobserved)
-          if (gh > 0) mbar_poll(pv_done(x), (gh - 1) & 1, abort_flag);
-          if (used) {
-            if (stores_pending) {                                      // the previous item's staged output
-              if (lane == 0) bulk_wait_read<0>();
-              __syncwarp();
-              stores_pending = false;
-            }
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-              *reinterpret_cast<uint4*>(p_row + ((c ^ (row & 7)) << 4)) =
-                  make_uint4(pw[4 * c], pw[4 * c + 1], pw[4 * c + 2], pw[4 * c + 3]);
-          }
-          if (hf == 0 && u == n_t - 1 && L.q_hi == I.n) {
-            // last tile of the sequence: the P V covers keys up to the next multiple of 16; zero the V rows
-            // between the sequence's end and that bound (both 64-dim halves)
-            const int valid = I.n - u * kAtBN, pad = cols - valid;
-            if (pad > 0) {
-              const int T = T0 + 2 * u + 1, s = T % kApRing;
-              mbar_wait_spin(ring_full(s), (T / kApRing) & 1, abort_flag);
-              char* v_s = ring_s + s * kAtTile;
-              for (int w = quad * 32 + lane; w < pad * 16; w += 128) {
-                const int r = valid + (w >> 4);
-                *reinterpret_cast<uint4*>(v_s + ((w >> 3) & 1) * (kAtBN * 128) + r * 128 + (w & 7) * 16) = make_uint4(0, 0, 0, 0);
-              }
-            }
-          }
-          fence_proxy_async();
-          if (hf == 0) tmem_ld_wait();                                 // all of S is in registers or consumed
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(p_full(x));
-            if (hf == 0) mbar_arrive(s_free(x));                       // the next tile's Q K^T may overwrite S
-          }
-        }
-      }
-      // ---- epilogue: O / l -> bf16 -> out[b][row][h][:], 32 columns at a time, two blocks staged per round in
-      // the warp's own 4 KB of the P buffer (16-byte units XOR-swizzled by row pair: the 64-byte swizzle of the
-      // tensor map)
-      const int gl = g0 + n_t - 1;
-      mbar_wait_spin(pv_done(x), (2 * gl + 1) & 1, abort_flag);       // MMAs complete in order: all of O is in
-      tc_fence_after();
-      const float inv = 1.0f / l_run;
-      const int rows_here = L.q_hi - r0;
-      const bool whole = rows_here >= 32;                              // warp-uniform
-      __nv_bfloat16* otile = a.out + (((size_t)I.b * a.n_max + r0) * a.H + I.h) * 128;
-      {
-        uint32_t ob[2][32];
-        tmem_ld32(o_addr, ob[0]);
-        tmem_ld_wait();
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          const uint32_t* o = ob[cc & 1];
-          if (cc < 3) tmem_ld32(o_addr + (cc + 1) * 32, ob[(cc + 1) & 1]);
-          if (cc == 2 && whole) {                                      // round two reuses the staging blocks
-            if (lane == 0) bulk_wait_read<0>();
-            __syncwarp();
-          }
-          char* sb = so + (cc & 1) * 2048;
-#pragma unroll
-          for (int w4 = 0; w4 < 4; ++w4) {
-            uint4 w;
-            __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[8 * w4]) * inv, __uint_as_float(o[8 * w4 + 1]) * inv);
-            __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[8 * w4 + 2]) * inv, __uint_as_float(o[8 * w4 + 3]) * inv);
-            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[8 * w4 + 4]) * inv, __uint_as_float(o[8 * w4 + 5]) * inv);
-            __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[8 * w4 + 6]) * inv, __uint_as_float(o[8 * w4 + 7]) * inv);
-            w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
-            w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
-            *reinterpret_cast<uint4*>(sb + lane * 64 + ((w4 ^ ((lane >> 1) & 3)) << 4)) = w;
-          }
-          if (cc < 3) tmem_ld_wait();
-          if (cc == 2) {                                               // all of O is in registers
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(o_free(x));
-          }
-          if (cc & 1) {                                                // a round of two blocks is staged
-            if (whole) {
-              fence_proxy_async();
-              __syncwarp();
-              if (lane == 0) {
-                tma_store_4d(mo, smem_u32(so), (cc - 1) * 32, I.h, r0, I.b);
-                tma_store_4d(mo, smem_u32(so + 2048), cc * 32, I.h, r0, I.b);
-                bulk_commit();
-              }
-            } else {
-              __syncwarp();
-#pragma unroll
-              for (int c2 = 0; c2 < 2; ++c2) {
-#pragma unroll
-                for (int it = 0; it < 4; ++it) {
-                  const int r = it * 8 + (lane >> 2), w4 = lane & 3;
-                  const uint4 w = *reinterpret_cast<const uint4*>(so + c2 * 2048 + r * 64 + ((w4 ^ ((r >> 1) & 3)) << 4));
-                  if (r < rows_here) *reinterpret_cast<uint4*>(otile + (size_t)r * a.H * 128 + (cc - 1 + c2) * 32 + w4 * 8) = w;
-                }
-              }
-              __syncwarp();
-            }
-          }
-        }
-      }
-      stores_pending = whole;
-      g0 += n_t;
-      ++n_item;
-      T0 += 2 * I.n_kv;
-    }
-    if (stores_pending && lane == 0) bulk_wait_read<0>();
-    if (*abort_flag && row == 0) report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
-  } else {
-    reg_dec<kAtRegsSmall>();
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 11) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1576,11 +849,7 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
   a.scale_log2 = scale * 1.4426950408889634f;
   static int attr_set[64];
   if (!attr_set[ctx->device & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attn_prefill_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attn_prefill_tcp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kApSmem);
+    cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(attn_prefill_tc1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kA1Smem);
     if (e != cudaSuccess) return e;
@@ -1589,13 +858,8 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
   const long long items = (long long)B * d.n_heads * a.q_pairs;
   if (items >= (1LL << 31)) return cudaErrorInvalidValue;
   const int grid = (int)std::min<long long>(items, (long long)ctx->sm_count);
-  // half tiles (two S buffers per lane) only on request (option value 3)
-  const bool halves = ctx->opt.prefill_attn_impl == 3;
-  // P through shared memory with the score buffer released early (option value 4)
   if (one_tile) attn_prefill_tc1_kernel<<<grid, kAtThreads, kA1Smem, s>>>(maps, a);
-  else if (ctx->opt.prefill_attn_impl == 4) attn_prefill_tcp_kernel<<<grid, kAtThreads, kApSmem, s>>>(maps, a);
-  else if (halves) attn_prefill_tc_kernel<2><<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
-  else attn_prefill_tc_kernel<1><<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
+  else attn_prefill_tc_kernel<<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
   return cudaGetLastError();
 }
 

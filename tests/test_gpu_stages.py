@@ -288,7 +288,7 @@ def _prefill_case(dtype, H, D, lens, amp=1.0):
         q, k = q * amp, k * amp
     scale = 1 / np.sqrt(D)
     n_max = max(lens)
-    for impl in (1, 2, 3, 4, 5):                 # CUDA cores; tensor cores: whole tiles / half tiles / P in shared memory / one tile per item
+    for impl in (1, 2, 5):                       # CUDA cores; tensor cores: pairs of query tiles / one tile per item
         ctx = _ctx(dtype, H, D, B=B, cap=cap)
         ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, impl)
         out = torch.full((B, n_max, H, D), 7.0, dtype=wl.torch_dtype(dtype), device=DEV)
