@@ -52,9 +52,7 @@ enum {
 /* Implementation selectors for dl_set_option. */
 enum {
   DL_OPT_PREDICTOR_IMPL = 1,    /* 0 auto, 1 CUDA-core kernel, 2 tcgen05 tensor-core kernel (bf16) */
-  DL_OPT_PREFILL_ATTN_IMPL = 2, /* 0 auto, 1 CUDA-core kernel, 2 / 5 tcgen05 tensor-core kernel (bf16, D=128): pairs of
-                                 * query tiles sharing their K/V tiles / one query tile per work item with two score
-                                 * buffers and the softmax split by columns (auto: 5 for n_max <= 512, else 2) */
+  DL_OPT_PREFILL_ATTN_IMPL = 2, /* 0 auto, 1 CUDA-core kernel, 2 tcgen05 tensor-core kernel (bf16, D=128) */
   DL_OPT_DECODE_CHUNK = 3,      /* cache rows per decode work item (0 = chosen by the library) */
   DL_OPT_DECODE_IMPL = 4,       /* 0 auto, 1 CUDA-core kernel, 2 tensor-core (mma.sync) kernel (bf16, D=128) */
   DL_OPT_COMPACT_IMPL = 5       /* 0 auto, 1 register-staged copy kernel, 2 bulk-copy (TMA) kernel by tiles of 32

@@ -151,7 +151,7 @@ int32_t dl_set_option(dl_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx || value < 0) return DL_ERR_INVALID_ARG;
   switch (option) {
     case DL_OPT_PREDICTOR_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.predictor_impl = value; break;
-    case DL_OPT_PREFILL_ATTN_IMPL: if (value > 5 || value == 3 || value == 4) return DL_ERR_INVALID_ARG; ctx->opt.prefill_attn_impl = value; break;
+    case DL_OPT_PREFILL_ATTN_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.prefill_attn_impl = value; break;
     case DL_OPT_DECODE_CHUNK: ctx->opt.decode_chunk = value; break;
     case DL_OPT_DECODE_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.decode_impl = value; break;
     case DL_OPT_COMPACT_IMPL: if (value > 3) return DL_ERR_INVALID_ARG; ctx->opt.compact_impl = value; break;

@@ -103,24 +103,20 @@ __device__ __forceinline__ int ld_early(const int32_t* p) {
 // additions (a division per item and role is what an item's set-up cannot afford); the length of the NEXT
 // item's sequence is requested one item early, so its latency never sits in front of a role's first wait.
 // (Walking head by head instead, all pairs of a head side by side, halves the DRAM reads on long contexts
-// - K and V of a head are then fetched once - but measured 20-60 % slower: the kernel is not DRAM-bound.)
+// - K and V of a head are then fetched once - but measured 20-60 % slower: the kernel is not DRAM-bound.
+// Rounds that run forwards and backwards in turn, to even out the CTAs' totals, measured 7-12 % slower too.)
 constexpr bool kAtSwapLanes = true;
-constexpr bool kAtSnake = false;
 struct AtWalker {
   const AtArgs& a;
-  int p, b, h, len, db0, dh0, db1, dh1, odd, sw;   // next item, its length (in flight), the two steps as (db, dh), swap bit
+  int p, b, h, len, db, dh, sw;               // next item, its length (in flight), the step as (db, dh), swap bit
   __device__ __forceinline__ explicit AtWalker(const AtArgs& a_) : a(a_) {
     const int bh_count = a.B * a.H;
     p = (int)blockIdx.x / bh_count;
     const int bh = (int)blockIdx.x - p * bh_count;
     b = bh / a.H;
     h = bh - b * a.H;
-    // The CTAs take the items (longest first) in rounds that run forwards and backwards in turn, so that the CTA
-    // that got the longest item of one round gets the shortest of the next: CTA c takes items c, 2G-1-c, 2G+c, ...
-    const int G = (int)gridDim.x, s0 = kAtSnake ? 2 * G - 1 - 2 * (int)blockIdx.x : G, s1 = kAtSnake ? 1 + 2 * (int)blockIdx.x : G;
-    db0 = s0 / a.H; dh0 = s0 - db0 * a.H;
-    db1 = s1 / a.H; dh1 = s1 - db1 * a.H;
-    odd = 0;
+    db = (int)gridDim.x / a.H;
+    dh = (int)gridDim.x - db * a.H;
     sw = 0;
     len = p < a.q_pairs ? ld_early(a.cache_len + b) : 0;
   }
@@ -129,9 +125,8 @@ struct AtWalker {
     for (;;) {
       if (p >= a.q_pairs) return false;
       const int cp = p, cb = b, ch = h, clen = len;
-      h += odd ? dh1 : dh0;
-      b += odd ? db1 : db0;
-      odd ^= 1;
+      h += dh;
+      b += db;
       if (h >= a.H) { h -= a.H; ++b; }
       while (b >= a.B) { b -= a.B; ++p; }
       if (p < a.q_pairs) len = ld_early(a.cache_len + b);
@@ -148,22 +143,6 @@ struct AtWalker {
     }
   }
 };
-
-// Whether the two MMA-issuing threads take turns (a lane issues a whole block, P V then the next
-// Q K^T, before the other lane's block is queued).  Measured both ways: with turns the lanes run half a
-// period apart, one lane's softmax hiding behind the other's MMAs, but a single thread cannot keep the
-// tensor pipe fed (a chain of eight dependent MMAs costs its issuer ~200 cycles of latency on top of
-// 8 x 64, and each completion signal ~90 more) and a softmax warp alone on its scheduler does not
-// overlap its exponentials with its arithmetic.  Without turns the lanes fall into step: both issue
-// at once (the pipe interleaves the two chains at full rate) and both softmax at once (two warps per
-// scheduler interleave).  The second is 3-7 % faster on the shapes at hand, so it is the default.
-constexpr bool kAtTakeTurns = false;
-__device__ __forceinline__ void pipe_lock(int* l, volatile int* abort) {
-  if (!kAtTakeTurns) return;
-  for (int i = 0; atomicCAS(l, 0, 1) != 0; ++i)
-    if (i > kSpinLimitBusy) { *abort = 1; return; }
-}
-__device__ __forceinline__ void pipe_unlock(int* l) { if (kAtTakeTurns) atomicExch(l, 0); }
 
 // Register budget per role (the kernel starts every thread at 168): the producer / MMA warps give
 // registers back, the softmax warps take them to hold a whole score row.

@@ -73,11 +73,9 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
   auto o_free = [&](int x) { return smem_u32(bars + 29 + x); };   // the epilogue has read O (4 warps)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
-  int* pipe_turn = reinterpret_cast<int*>(bars + 34);
 
   if (tid == 0) {
     *abort_flag = 0;
-    *pipe_turn = 0;
     for (int s = 0; s < kAtRing; ++s) {
       mbar_init(ring_full(s), 1);
       mbar_init(ring_free(0, s), 1);
@@ -109,48 +107,51 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.k[i]));
         tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.v[i]));
       }
-      // cursor of the ring
-      AtWalker Wr(a);
-      AtItem Ir;
+      // Two cursors over the CTA's items: the ring's (K and V tiles, in order) and the Q loads' (per item, either
+      // lane's tile as soon as its slot is free; the item is left when both are on their way).  Each cursor
+      // advances in ONE place: the walker's step is inlined wherever it is called, and this role's code is
+      // fetched cold at every item.
+      AtWalker Wr(a), Wq(a);
+      AtItem Ir, Iq;
       int T = 0, jr = 0;                       // ring tiles issued so far / tile index within Ir (K, V alternating)
-      // cursors of the Q loads
-      AtWalker Wq0 = Wr, Wq1 = Wr;
-      AtItem Iq[2];
-      bool hq[2];
       int nq[2] = {0, 0};                      // Q loads issued so far per lane
-      bool hr = Wr.next(Ir);
-      hq[0] = Wq0.next(Iq[0]);
-      hq[1] = Wq1.next(Iq[1]);
-      while (hq[0] && !at_lane(Iq[0], 0).exists) hq[0] = Wq0.next(Iq[0]);
-      while (hq[1] && !at_lane(Iq[1], 1).exists) hq[1] = Wq1.next(Iq[1]);
+      bool hr = true, hq = true, need_r = true, need_q = true;
+      int q_todo = 0;                          // lanes of Iq whose Q tile is still to be requested (bit x)
       int idle = 0;
-      while ((hr || hq[0] || hq[1]) && !*abort_flag) {
+      while ((hr || hq) && !*abort_flag) {
         bool prog = false;
-#pragma unroll
+        if (hq && need_q) {
+          hq = Wq.next(Iq);
+          need_q = false;
+          q_todo = hq ? ((at_lane(Iq, 0).exists ? 1 : 0) | (at_lane(Iq, 1).exists ? 2 : 0)) : 0;
+          prog = true;
+        }
+#pragma unroll 1
         for (int x = 0; x < 2; ++x) {
-          if (!hq[x]) continue;
+          if (!((q_todo >> x) & 1)) continue;
           const int s = nq[x] & 1;
           // the slot's previous item (two items back) must have finished its epilogue
           if (nq[x] >= 2 && !mbar_test(q_done(x, s), ((nq[x] - 2) >> 1) & 1)) continue;
-          const AtLane L = at_lane(Iq[x], x);
+          const AtLane L = at_lane(Iq, x);
           char* dst = smem + (2 * x + s) * kAtTile;
           // the rows the lane owns, in 16s (a tile clipped at the top of the sequence owns fewer than 128)
           const int bx = at_box(min(kAtBM, (L.q_hi - L.q0 + 15) & ~15));
           const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(maps.q[bx]);
           mbar_expect_tx(q_full(x, s), kAtTile >> bx);
-          tma_load_2d(smem_u32(dst), mq, 0, Iq[x].row_base + L.q0, q_full(x, s));
-          tma_load_2d(smem_u32(dst + kAtBM * 128), mq, 64, Iq[x].row_base + L.q0, q_full(x, s));
+          tma_load_2d(smem_u32(dst), mq, 0, Iq.row_base + L.q0, q_full(x, s));
+          tma_load_2d(smem_u32(dst + kAtBM * 128), mq, 64, Iq.row_base + L.q0, q_full(x, s));
           ++nq[x];
-          if (x == 0) {
-            hq[0] = Wq0.next(Iq[0]);
-            while (hq[0] && !at_lane(Iq[0], 0).exists) hq[0] = Wq0.next(Iq[0]);
-          } else {
-            hq[1] = Wq1.next(Iq[1]);
-            while (hq[1] && !at_lane(Iq[1], 1).exists) hq[1] = Wq1.next(Iq[1]);
-          }
+          q_todo &= ~(1 << x);
           prog = true;
         }
-        if (hr) {
+        if (hq && !need_q && q_todo == 0) need_q = true;
+        if (hr && need_r) {
+          hr = Wr.next(Ir);
+          need_r = false;
+          jr = 0;
+          prog = true;
+        }
+        if (hr && !need_r) {
           const int s = T % kAtRing;
           bool slot_free = true;
           if (T >= kAtRing) {
@@ -169,7 +170,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
             tma_load_2d(smem_u32(dst), m, 0, r, ring_full(s));
             tma_load_2d(smem_u32(dst + kAtBN * 128), m, 64, r, ring_full(s));
             ++T;
-            if (++jr == 2 * Ir.n_kv) { jr = 0; hr = Wr.next(Ir); }
+            if (++jr == 2 * Ir.n_kv) need_r = true;
             prog = true;
           }
         }
@@ -202,85 +203,71 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       while (W.next(I)) {
         const AtLane L = at_lane(I, x);
         auto wait_ring = [&](int T) { mbar_wait_spin(ring_full(T % kAtRing), (T / kAtRing) & 1, abort_flag); };
-        // A lane does not read every ring tile (not the pair's last key tile when it has the earlier query
-        // tile, nothing of a pair that has no earlier tile).  It still observes every tile's landing and
-        // releases it, in ring order, so that the slot barriers advance one phase per tile for every
-        // waiter: a waiter that had skipped phases could not tell them apart by parity.
-        auto pass_tiles = [&](int from, int to) {
-          for (int T = from; T < to; ++T) {
-            wait_ring(T);
-            mbar_arrive(ring_free(x, T % kAtRing));
-          }
-        };
-        if (!L.exists) {
-          pass_tiles(T0, T0 + 2 * I.n_kv);
-          T0 += 2 * I.n_kv;
-          continue;
-        }
+        const int n_sub = L.exists ? L.n_tiles : 0;
         const int qs = n_item & 1;
         const uint64_t q_desc = smem_desc_sw128(smem_u32(smem + (2 * x + qs) * kAtTile));
-        const int n_sub = L.n_tiles;
-        auto sub_cols = [&](int u) { return at_cols(L, u); };
-        auto issue_qk = [&](int u) {
-          const int s = (T0 + 2 * u) % kAtRing;
-          const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile));
-          const uint32_t idesc_qk = idesc_bf16(kAtBM, (uint32_t)sub_cols(u));
-          // not unrolled (an MMA holds the thread for 64 cycles anyway; short code is what counts here): 16 dims
-          // further per step, and from the fourth step on in the tile's second 64-dim half
-          uint64_t qd = q_desc, kd = k_desc;
-#pragma unroll 1
-          for (int ks = 0; ks < 8; ++ks) {
-            mma_ss(t_s, qd, kd, idesc_qk, ks != 0);
-            const uint64_t step = (ks == 3) ? (uint64_t)((kAtBM * 128 - 96) >> 4) : 2ull;
-            qd += step;
-            kd += step;
-          }
-        };
-        // Completion signals: a commit covers every MMA this thread has issued so far.  The K tile is
-        // released by the Q K^T of its last sub-tile.
-        auto commit_qk = [&](int u) {
-          mma_commit(s_full(x, 0));                       // first: the softmax warps wait on it
-          mma_commit(ring_free(x, (T0 + 2 * u) % kAtRing));
-        };
-        mbar_wait_spin(q_full(x, qs), (n_item >> 1) & 1, abort_flag);
-        wait_ring(T0);
-        tc_fence_after();
-        pipe_lock(pipe_turn, abort_flag);
-        issue_qk(0);
-        pipe_unlock(pipe_turn);
-        commit_qk(0);
-        for (int u = 0; u < n_sub; ++u) {
-          const int g = g0 + u, b = 0;
-          const int T = T0 + 2 * u + 1, s = T % kAtRing;                 // the V tile of this key tile
-          const int un = u + 1;                                          // the tile whose Q K^T reuses the S buffer
+        // Block u of the item: O += P_u V_u, then S = Q K_{u+1}^T (which overwrites P: in order behind the P V).
+        // Block -1 is the first Q K^T alone, the last block the last P V alone.  One copy of the code for all
+        // of them, loops not unrolled: an MMA holds the thread for 64 cycles anyway, and this role's code is
+        // fetched cold at every item.
+        for (int u = L.exists ? -1 : 0; u < n_sub; ++u) {
+          const int g = g0 + u;
+          const int Tv = T0 + 2 * u + 1, sv = Tv % kAtRing;              // the V tile of this key tile
+          const int sk = (Tv + 1) % kAtRing;                             // the K tile of the next one
+          const bool has_pv = u >= 0, has_qk = u + 1 < n_sub;
           // operands first (they land long before), then the softmax's hand-over
-          wait_ring(T);
-          if (un < n_sub) wait_ring(T0 + 2 * un);
+          if (has_pv) wait_ring(Tv);
+          else mbar_wait_spin(q_full(x, qs), (n_item >> 1) & 1, abort_flag);
+          if (has_qk) wait_ring(Tv + 1);
           if (u == 0) mbar_wait_spin(o_free(x), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
-          // polled without suspending: the wake-up of a suspended wait costs this thread ~600 cycles per tile
-          {
-            const uint32_t pb = p_full(x, b), ph = (uint32_t)g & 1u;
+          if (has_pv) {
+            // polled without suspending: the wake-up of a suspended wait costs this thread ~600 cycles per tile
+            const uint32_t pb = p_full(x, 0), ph = (uint32_t)g & 1u;
             int spins = 0;
             while (!mbar_test(pb, ph)) {
               if ((++spins & 1023) == 0 && (*abort_flag || spins > (kSpinLimitBusy << 4))) { *abort_flag = 1; break; }
             }
           }
           tc_fence_after();
-          const uint64_t v_desc =
-              smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128);
-          const int ksteps = sub_cols(u) >> 4;
-          pipe_lock(pipe_turn, abort_flag);
-          for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(t_o, t_s + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv, (u | ks) != 0);
-          if (un < n_sub) issue_qk(un);                                // overwrites P: in order behind the P V
-          pipe_unlock(pipe_turn);
-          if (un < n_sub) commit_qk(un);
-          mma_commit(pv_done(x, b));
-          mma_commit(ring_free(x, s));
+          if (has_pv) {
+            uint64_t v_desc = smem_desc_sw128_mn(smem_u32(ring_s + sv * kAtTile), kAtBN * 128);
+            const int ksteps = at_cols(L, u) >> 4;
+#pragma unroll 1
+            for (int ks = 0; ks < ksteps; ++ks, v_desc += 2048 >> 4)
+              mma_ts(t_o, t_s + ks * 8, v_desc, idesc_pv, (u | ks) != 0);
+          }
+          if (has_qk) {
+            // 16 dims further per step, and from the fourth step on in the tile's second 64-dim half
+            uint64_t qd = q_desc, kd = smem_desc_sw128(smem_u32(ring_s + sk * kAtTile));
+            const uint32_t idesc_qk = idesc_bf16(kAtBM, (uint32_t)at_cols(L, u + 1));
+#pragma unroll 1
+            for (int ks = 0; ks < 8; ++ks) {
+              mma_ss(t_s, qd, kd, idesc_qk, ks != 0);
+              const uint64_t step = (ks == 3) ? (uint64_t)((kAtBM * 128 - 96) >> 4) : 2ull;
+              qd += step;
+              kd += step;
+            }
+            // Completion signals: a commit covers every MMA this thread has issued so far.
+            mma_commit(s_full(x, 0));                                    // first: the softmax warps wait on it
+            mma_commit(ring_free(x, sk));
+          }
+          if (has_pv) {
+            mma_commit(pv_done(x, 0));
+            mma_commit(ring_free(x, sv));
+          }
         }
-        pass_tiles(T0 + 2 * L.n_tiles, T0 + 2 * I.n_kv);
-        g0 += n_sub;
-        ++n_item;
+        // A lane does not read every ring tile (not the pair's last key tile when it has the earlier query
+        // tile, nothing of a pair that has no earlier tile).  It still observes every tile's landing and
+        // releases it, in ring order, so that the slot barriers advance one phase per tile for every
+        // waiter: a waiter that had skipped phases could not tell them apart by parity.
+        for (int T = T0 + 2 * n_sub; T < T0 + 2 * I.n_kv; ++T) {
+          wait_ring(T);
+          mbar_arrive(ring_free(x, T % kAtRing));
+        }
+        if (L.exists) {
+          g0 += n_sub;
+          ++n_item;
+        }
         T0 += 2 * I.n_kv;
       }
     }
@@ -408,408 +395,6 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
   if (warp == 11) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
-// Polls a barrier without suspending the thread (hand-overs that are a few hundred cycles apart).
-__device__ __forceinline__ void mbar_poll(uint32_t bar, uint32_t parity, volatile int* abort) {
-  int spins = 0;
-  while (!mbar_test(bar, parity)) {
-    if ((++spins & 1023) == 0 && (*abort || spins > (kSpinLimitBusy << 4))) { *abort = 1; break; }
-  }
-}
-
-// ---------------------------------------------------------------------------------------------------
-// Variant with ONE query tile per CTA, two score buffers and the softmax of a tile split by columns.
-// Work item = (sequence, head, one 128-row query tile, end-aligned).  Tensor memory: O | S0 | S1, so the
-// Q K^T of key tile j+1 runs into the other score buffer while the softmax works on tile j, and a tile's
-// softmax never waits for MMAs.  The softmax of a tile is taken by EIGHT warps: warps 0-3 own the tile's
-// first 64 key columns, warps 4-7 the last 64 (the same 128 rows, one row per thread each), two warps per
-// scheduler, which is what keeps the special-function unit busy.  The two halves agree on the row
-// maximum in use through shared memory once per tile (raised only when the tile's maximum exceeds it by
-// 2^8; then each half rescales its 64 columns of O), add up their own row sums and combine them at the
-// end.  P (bf16) overwrites the first half of its own score buffer and feeds the P V MMA from tensor
-// memory, so shared-memory traffic stays with the operands; K and V are fetched per query tile (not
-// shared by a pair), which costs L2 reads, not DRAM reads.  Shared memory: two Q slots, a four-slot
-// K/V ring, 32 KB of output staging.
-constexpr int kA1Ring = 4;
-constexpr int kA1OffRing = 2 * kAtTile;               // Q slot 0, Q slot 1, then the ring
-constexpr int kA1OffStage = kA1OffRing + kA1Ring * kAtTile;
-constexpr int kA1OffBar = kA1OffStage + kAtTile;
-constexpr int kA1OffX = kA1OffBar + 256;              // [2 halves][128 rows] floats exchanged between the halves
-constexpr size_t kA1Smem = kA1OffX + 2 * 1024;       // one set per tile parity
-static_assert(kA1Smem <= 232448, "one CTA per SM");
-constexpr uint32_t kA1ColO = 0, kA1ColS = 128;        // tensor-memory columns: O, then S0 and S1 (128 each)
-
-// barrier of the eight softmax warps only (the other roles never join it)
-__device__ __forceinline__ void softmax_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-
-__global__ void __launch_bounds__(kAtThreads, 1)
-attn_prefill_tc1_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
-  extern __shared__ __align__(1024) char smem[];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (smem_u32(smem) & 1023u) {
-    if (tid == 0) report_status(a.status, DL_ERR_ALIGNMENT, -1);
-    return;
-  }
-  char* ring_s = smem + kA1OffRing;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kA1OffBar);
-  float* xch = reinterpret_cast<float*>(smem + kA1OffX);
-  // Ring tile T (running count; K and V of key tile j of an item are tiles base + 2j, base + 2j + 1) lives in
-  // slot T % 4, phase (T / 4) & 1.  The CTA's g-th key tile (running count) uses score buffer g & 1 and
-  // completes phase (g >> 1) & 1 of that buffer's s_full / p_full / pv_done; its i-th item completes phase
-  // i & 1 of o_free and phase (i >> 1) & 1 of q_full / q_free of Q slot i & 1.
-  auto ring_full = [&](int s) { return smem_u32(bars + s); };
-  auto ring_free = [&](int s) { return smem_u32(bars + 4 + s); };
-  auto q_full = [&](int s) { return smem_u32(bars + 8 + s); };
-  auto q_free = [&](int s) { return smem_u32(bars + 10 + s); };     // the item's last Q K^T has read the slot
-  auto s_full = [&](int b) { return smem_u32(bars + 12 + b); };     // Q K^T has completed: S ready
-  auto p_full = [&](int b) { return smem_u32(bars + 14 + b); };     // P is in tensor memory (8 warps)
-  auto pv_done = [&](int b) { return smem_u32(bars + 16 + b); };    // P V has completed: O at rest
-  auto o_free = [&]() { return smem_u32(bars + 18); };              // the epilogue has read O (8 warps)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 21);
-
-  if (tid == 0) {
-    *abort_flag = 0;
-    for (int s = 0; s < kA1Ring; ++s) { mbar_init(ring_full(s), 1); mbar_init(ring_free(s), 1); }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(q_full(s), 1); mbar_init(q_free(s), 1);
-      mbar_init(s_full(s), 1); mbar_init(p_full(s), 8); mbar_init(pv_done(s), 1);
-    }
-    mbar_init(o_free(), 8);
-    fence_mbar_init();
-  }
-  if (warp == 11) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-
-  if (warp == 8) {
-    // ---------------------------------------------------------------- TMA producer
-    reg_dec<kAtRegsSmall>();
-    if (lane == 0) {
-      for (int i = 0; i < 4; ++i) {
-        tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.q[i]));
-        tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.k[i]));
-        tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(maps.v[i]));
-      }
-      AtWalker Wr(a), Wq(a);
-      AtItem Ir, Iq;
-      int T = 0, jr = 0, nq = 0;
-      bool hr = Wr.next(Ir), hq = Wq.next(Iq);
-      int idle = 0;
-      while ((hr || hq) && !*abort_flag) {
-        bool prog = false;
-        if (hq && (nq < 2 || mbar_test(q_free(nq & 1), ((nq - 2) >> 1) & 1))) {
-          const AtLane L = at_lane(Iq, 0);
-          char* dst = smem + (nq & 1) * kAtTile;
-          const int bx = at_box(min(kAtBM, (L.q_hi - L.q0 + 15) & ~15));
-          const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(maps.q[bx]);
-          mbar_expect_tx(q_full(nq & 1), kAtTile >> bx);
-          tma_load_2d(smem_u32(dst), mq, 0, Iq.row_base + L.q0, q_full(nq & 1));
-          tma_load_2d(smem_u32(dst + kAtBM * 128), mq, 64, Iq.row_base + L.q0, q_full(nq & 1));
-          ++nq;
-          hq = Wq.next(Iq);
-          prog = true;
-        }
-        if (hr) {
-          const int s = T % kA1Ring;
-          if (T < kA1Ring || mbar_test(ring_free(s), (uint32_t)(T / kA1Ring - 1) & 1u)) {
-            const int j = jr >> 1;
-            char* dst = ring_s + s * kAtTile;
-            const int bx = at_box(min(kAtBN, (Ir.q_hi - j * kAtBN + 15) & ~15));
-            const CUtensorMap* m = reinterpret_cast<const CUtensorMap*>((jr & 1) ? maps.v[bx] : maps.k[bx]);
-            const int r = Ir.row_base + j * kAtBN;
-            mbar_expect_tx(ring_full(s), kAtTile >> bx);
-            tma_load_2d(smem_u32(dst), m, 0, r, ring_full(s));
-            tma_load_2d(smem_u32(dst + kAtBN * 128), m, 64, r, ring_full(s));
-            ++T;
-            if (++jr == 2 * Ir.n_kv) { jr = 0; hr = Wr.next(Ir); }
-            prog = true;
-          }
-        }
-        if (prog) {
-          idle = 0;
-        } else if (++idle > kSpinLimitBusy) {
-          *abort_flag = 1;
-        }
-      }
-      if (*abort_flag) {
-        // every copy that was issued must land before the CTA's shared memory is released
-        report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
-        for (int t = max(0, T - kA1Ring); t < T; ++t)
-          for (int i = 0; i < kSpinLimit && !mbar_try_wait(ring_full(t % kA1Ring), (t / kA1Ring) & 1); ++i) __nanosleep(40);
-        for (int t = max(0, nq - 2); t < nq; ++t)
-          for (int i = 0; i < kSpinLimit && !mbar_try_wait(q_full(t & 1), (t >> 1) & 1); ++i) __nanosleep(40);
-      }
-    }
-  } else if (warp == 9) {
-    // ---------------------------------------------------------------- MMA issuer
-    reg_dec<kAtRegsSmall>();
-    if (lane == 0) {
-      const uint32_t t_o = tmem + kA1ColO;
-      const uint32_t idesc_pv = idesc_bf16(kAtBM, 128, 0, 1);          // B (= V) is MN-major
-      AtWalker W(a);
-      AtItem I;
-      int n_item = 0, g0 = 0, T0 = 0;
-      while (W.next(I)) {
-        const AtLane L = at_lane(I, 0);
-        const int n_t = L.n_tiles, qs = n_item & 1;
-        const uint64_t q_desc = smem_desc_sw128(smem_u32(smem + qs * kAtTile));
-        auto wait_ring = [&](int T) { mbar_wait_spin(ring_full(T % kA1Ring), (T / kA1Ring) & 1, abort_flag); };
-        // S[g & 1] = Q K^T of tile u.  The buffer's previous user is tile g - 2: its P V is in front of this
-        // MMA in the pipe (same issuing thread), and its softmax has long handed over.
-        auto issue_qk = [&](int u) {
-          const int T = T0 + 2 * u, s = T % kA1Ring, g = g0 + u;
-          wait_ring(T);
-          tc_fence_after();
-          const uint64_t k_desc = smem_desc_sw128(smem_u32(ring_s + s * kAtTile));
-          const uint32_t idesc_qk = idesc_bf16(kAtBM, (uint32_t)at_cols(L, u));
-          const uint32_t d = tmem + kA1ColS + (g & 1) * 128;
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            mma_ss(d, q_desc + (uint64_t)(((ks >> 2) * (kAtBM * 128) + (ks & 3) * 32) >> 4),
-                   k_desc + (uint64_t)(((ks >> 2) * (kAtBN * 128) + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
-          mma_commit(s_full(g & 1));
-          mma_commit(ring_free(s));
-          if (u == n_t - 1) mma_commit(q_free(qs));
-        };
-        mbar_wait_spin(q_full(qs), (n_item >> 1) & 1, abort_flag);
-        issue_qk(0);
-        for (int u = 0; u < n_t; ++u) {
-          const int g = g0 + u;
-          if (u + 1 < n_t) issue_qk(u + 1);                             // runs while the softmax works on tile u
-          const int T = T0 + 2 * u + 1, s = T % kA1Ring;                // the V tile
-          wait_ring(T);
-          if (u == 0) mbar_wait_spin(o_free(), (n_item & 1) ^ 1, abort_flag);   // previous item's O has been read
-          mbar_poll(p_full(g & 1), (uint32_t)(g >> 1) & 1u, abort_flag);
-          tc_fence_after();
-          const uint64_t v_desc = smem_desc_sw128_mn(smem_u32(ring_s + s * kAtTile), kAtBN * 128);
-          const uint32_t t_p = tmem + kA1ColS + (g & 1) * 128;
-          const int ksteps = at_cols(L, u) >> 4;
-          for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(t_o, t_p + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv, (u | ks) != 0);
-          mma_commit(pv_done(g & 1));
-          mma_commit(ring_free(s));
-        }
-        g0 += n_t;
-        ++n_item;
-        T0 += 2 * I.n_kv;
-      }
-    }
-  } else if (warp < 8) {
-    // ---------------------------------------------------------------- softmax / epilogue: two halves of four warps
-    reg_inc<kAtRegsSoftmax>();
-    const int half = warp >> 2;                                        // key columns [64 half, 64 half + 64) of a tile
-    const int quad = warp & 3;
-    const int row = quad * 32 + lane;
-    const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
-    const uint32_t o_addr = tmem + lane_off + kA1ColO + half * 64;     // this half's 64 columns of O
-    const CUtensorMap* mo = reinterpret_cast<const CUtensorMap*>(maps.o);
-    char* so = smem + kA1OffStage + quad * 8192 + half * 4096;         // this warp's two 32 x 32 output blocks
-    const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2);
-    AtWalker W(a);
-    AtItem I;
-    int n_item = 0, g0 = 0, T0 = 0;
-    bool stores_pending = false;
-    while (W.next(I)) {
-      const AtLane L = at_lane(I, 0);
-      const int grow = L.q0 + row;
-      const int r0 = L.q0 + quad * 32;
-      float m_used = -INFINITY, l_run = 0.f;
-      const int n_t = L.n_tiles;
-      for (int u = 0; u < n_t; ++u) {
-        const int g = g0 + u, sb = g & 1;
-        const int c0 = u * kAtBN + half * 64;                           // first key of this half
-        const uint32_t sa = tmem + lane_off + kA1ColS + sb * 128 + half * 64;
-        // 32-column chunks of this half that some row of the warp may see (0, 1 or 2)
-        const int n_ch = max(0, min(2, (min(L.q_hi, r0 + 32) - c0 + 31) >> 5));
-        const int vis = grow - c0;
-        uint32_t S[64];
-        mbar_poll(s_full(sb), (g >> 1) & 1, abort_flag);
-        tc_fence_after();
-        if (n_ch > 0) tmem_ld32(sa, S);
-        if (n_ch > 1) tmem_ld32(sa + 32, S + 32);
-        tmem_ld_wait();
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          if (cc < n_ch) {
-            uint32_t* sr = S + 32 * cc;
-            if (c0 + 32 * cc + 31 > r0) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (32 * cc + c > vis) sr[c] = 0xFF800000u;            // -inf
-            }
-#pragma unroll
-            for (int c = 0; c < 32; c += 8) {
-#pragma unroll
-              for (int w = 0; w < 4; ++w)
-                mx4[w] = fmax3(mx4[w], __uint_as_float(sr[c + 2 * w]), __uint_as_float(sr[c + 2 * w + 1]));
-            }
-          }
-        }
-        // the row's maximum over both halves
-        const float mx_own = fmax3(mx4[0], mx4[1], fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-        float* xg = xch + (g & 1) * 256;                               // by tile parity: a warp is never two tiles ahead
-        xg[half * 128 + row] = mx_own;
-        softmax_sync();
-        const float mx_tile = fmaxf(mx_own, xg[(half ^ 1) * 128 + row]);
-        // raise the maximum in use (first tile: set it; column 0 is visible to every row, so it is finite)
-        const bool need = grow < L.q_hi && (u == 0 || mx_tile > m_used + kRescaleStep);
-        if (__any_sync(0xffffffffu, need)) {
-          const float corr = (need && u > 0) ? fast_exp2(m_used - mx_tile) : 1.0f;
-          if (need) m_used = mx_tile;
-          if (u > 0) {
-            // O must be at rest: the P V of the previous tile (the other half decides the same, row by row)
-            mbar_wait_spin(pv_done((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag);
-            tc_fence_after();
-            l_run *= corr;
-            const uint64_t corr2 = pack2(corr, corr);
-#pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-              uint32_t o[32];
-              tmem_ld32(o_addr + cc * 32, o);
-              tmem_ld_wait();
-#pragma unroll
-              for (int i = 0; i < 32; i += 2) {
-                float y0, y1;
-                unpack2(fmul2(pack2(__uint_as_float(o[i]), __uint_as_float(o[i + 1])), corr2), y0, y1);
-                o[i] = __float_as_uint(y0);
-                o[i + 1] = __float_as_uint(y1);
-              }
-              tmem_st32(o_addr + cc * 32, o);
-            }
-            tmem_st_wait();
-          }
-        }
-        // exponentials against the maximum in use, row sum, P as bf16 pairs
-        uint32_t pw[32];
-        const uint64_t nm2 = pack2(-m_used, -m_used);
-        uint64_t l2[2] = {0ull, 0ull};
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          if (cc < n_ch) {
-            const uint32_t* sr = S + 32 * cc;
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-              float p0, p1;
-              unpack2(ffma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), p0, p1);
-              p0 = fast_exp2(p0);
-              p1 = fast_exp2(p1);
-              l2[c & 1] = fadd2(l2[c & 1], pack2(p0, p1));
-              __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-              pw[16 * cc + c] = *reinterpret_cast<uint32_t*>(&pk);
-            }
-          } else {
-#pragma unroll
-            for (int c = 0; c < 16; ++c) pw[16 * cc + c] = 0u;
-          }
-        }
-        {
-          float la, lb;
-          unpack2(fadd2(l2[0], l2[1]), la, lb);
-          l_run += la + lb;
-        }
-        // P over the first half of the tile's own score buffer: this half's 64 keys are 32 columns of bf16 pairs.
-        // Every thread has read the buffer (the exchange above came after the loads).
-        tmem_st32(tmem + lane_off + kA1ColS + sb * 128 + half * 32, pw);
-        tmem_st_wait();
-        if (u == n_t - 1 && L.q_hi == I.n) {
-          // last tile of the sequence: zero the V rows between the sequence's end and the 16-key bound of the P V
-          const int valid = I.n - u * kAtBN, pad = at_cols(L, u) - valid;
-          if (pad > 0) {
-            const int T = T0 + 2 * u + 1, s = T % kA1Ring;
-            mbar_wait_spin(ring_full(s), (T / kA1Ring) & 1, abort_flag);
-            char* v_s = ring_s + s * kAtTile;
-            for (int w = warp * 32 + lane; w < pad * 16; w += 256) {
-              const int r = valid + (w >> 4);
-              *reinterpret_cast<uint4*>(v_s + ((w >> 3) & 1) * (kAtBN * 128) + r * 128 + (w & 7) * 16) = make_uint4(0, 0, 0, 0);
-            }
-            fence_proxy_async();
-          }
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(p_full(sb));
-      }
-      // ---- epilogue: the halves add up their row sums, then each writes its 64 columns of O / l
-      const int gl = g0 + n_t - 1;
-      float* xl = xch + ((gl + 1) & 1) * 256;                         // the set the last tile did not use
-      xl[half * 128 + row] = l_run;
-      softmax_sync();
-      const float inv = 1.0f / (l_run + xl[(half ^ 1) * 128 + row]);
-      softmax_sync();                                                  // the words may be rewritten by the next item
-      mbar_wait_spin(pv_done(gl & 1), (gl >> 1) & 1, abort_flag);      // MMAs complete in order: all of O is in
-      tc_fence_after();
-      const int rows_here = L.q_hi - r0;
-      const bool whole = rows_here >= 32;                              // warp-uniform
-      __nv_bfloat16* otile = a.out + (((size_t)I.b * a.n_max + r0) * a.H + I.h) * 128 + half * 64;
-      if (stores_pending) {                                            // the previous item's staged output
-        if (lane == 0) bulk_wait_read<0>();
-        __syncwarp();
-        stores_pending = false;
-      }
-      {
-        uint32_t ob[2][32];
-        tmem_ld32(o_addr, ob[0]);
-        tmem_ld32(o_addr + 32, ob[1]);
-        tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(o_free());                          // all of this warp's O is in registers
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          const uint32_t* o = ob[cc];
-          char* sb2 = so + cc * 2048;
-#pragma unroll
-          for (int w4 = 0; w4 < 4; ++w4) {
-            uint4 w;
-            __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[8 * w4]) * inv, __uint_as_float(o[8 * w4 + 1]) * inv);
-            __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[8 * w4 + 2]) * inv, __uint_as_float(o[8 * w4 + 3]) * inv);
-            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[8 * w4 + 4]) * inv, __uint_as_float(o[8 * w4 + 5]) * inv);
-            __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[8 * w4 + 6]) * inv, __uint_as_float(o[8 * w4 + 7]) * inv);
-            w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
-            w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
-            *reinterpret_cast<uint4*>(sb2 + lane * 64 + ((w4 ^ ((lane >> 1) & 3)) << 4)) = w;
-          }
-        }
-      }
-      if (whole) {
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) {
-          tma_store_4d(mo, smem_u32(so), half * 64, I.h, r0, I.b);
-          tma_store_4d(mo, smem_u32(so + 2048), half * 64 + 32, I.h, r0, I.b);
-          bulk_commit();
-        }
-        stores_pending = true;
-      } else {
-        __syncwarp();
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-#pragma unroll
-          for (int it = 0; it < 4; ++it) {
-            const int r = it * 8 + (lane >> 2), w4 = lane & 3;
-            const uint4 w = *reinterpret_cast<const uint4*>(so + cc * 2048 + r * 64 + ((w4 ^ ((r >> 1) & 3)) << 4));
-            if (r < rows_here) *reinterpret_cast<uint4*>(otile + (size_t)r * a.H * 128 + cc * 32 + w4 * 8) = w;
-          }
-        }
-        __syncwarp();
-      }
-      g0 += n_t;
-      ++n_item;
-      T0 += 2 * I.n_kv;
-    }
-    if (stores_pending && lane == 0) bulk_wait_read<0>();
-    if (*abort_flag && tid == 0) report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
-  } else {
-    reg_dec<kAtRegsSmall>();                             // warps 10, 11: same budget as the rest of their warpgroup
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 11) { tc_fence_after(); tmem_dealloc(tmem, 512); }
-}
-
 bool attn_prefill_tc_supported(const dl_ctx* ctx) {
   const dl_model_desc& d = ctx->desc;
   return d.dtype == DL_BF16 && d.head_dim == 128 && ctx->tmap_encode != nullptr && (size_t)ctx->smem_optin >= kAtSmem;
@@ -841,25 +426,19 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
     return cudaErrorInvalidValue;
   AtArgs a;
   a.cache_len = cache_len; a.out = static_cast<__nv_bfloat16*>(out); a.status = ctx->ws.base ? ctx->ws.status : nullptr;
-  // one query tile per item (two score buffers, softmax split by columns): on request, and the library's
-  // choice up to 512 rows, where it measured 14 % faster (272 rows) to equal (240, 832 rows)
-  const bool one_tile = ctx->opt.prefill_attn_impl == 5 || (ctx->opt.prefill_attn_impl == 0 && n_max <= 512);
-  a.item_rows = one_tile ? kAtBM : 2 * kAtBM;
+  a.item_rows = 2 * kAtBM;
   a.B = B; a.H = d.n_heads; a.cap = cap; a.n_max = n_max; a.q_pairs = (n_max + a.item_rows - 1) / a.item_rows;
   a.scale_log2 = scale * 1.4426950408889634f;
   static int attr_set[64];
   if (!attr_set[ctx->device & 63]) {
     cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attn_prefill_tc1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kA1Smem);
     if (e != cudaSuccess) return e;
     attr_set[ctx->device & 63] = 1;
   }
   const long long items = (long long)B * d.n_heads * a.q_pairs;
   if (items >= (1LL << 31)) return cudaErrorInvalidValue;
   const int grid = (int)std::min<long long>(items, (long long)ctx->sm_count);
-  if (one_tile) attn_prefill_tc1_kernel<<<grid, kAtThreads, kA1Smem, s>>>(maps, a);
-  else attn_prefill_tc_kernel<<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
+  attn_prefill_tc_kernel<<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
   return cudaGetLastError();
 }
 

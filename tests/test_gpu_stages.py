@@ -288,7 +288,7 @@ def _prefill_case(dtype, H, D, lens, amp=1.0):
         q, k = q * amp, k * amp
     scale = 1 / np.sqrt(D)
     n_max = max(lens)
-    for impl in (1, 2, 5):                       # CUDA cores; tensor cores: pairs of query tiles / one tile per item
+    for impl in (1, 2):                          # CUDA cores; tensor cores
         ctx = _ctx(dtype, H, D, B=B, cap=cap)
         ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, impl)
         out = torch.full((B, n_max, H, D), 7.0, dtype=wl.torch_dtype(dtype), device=DEV)
@@ -333,7 +333,7 @@ def test_prefill_attention_large_scores():
 
 
 def test_prefill_attention_large_grid_is_reproducible():
-    """Several waves of work items per CTA: the tensor-core kernels (query-tile pairs; one tile per item) must
+    """Several waves of work items per CTA: the tensor-core kernel must
     give the same bits every time and agree with the CUDA-core kernel (which the oracle checks above)."""
     from paper_2412_00876_b200 import binding as dl
     B, H, D, cap, n = 8, 32, 128, 1024, 832
@@ -343,7 +343,7 @@ def test_prefill_attention_large_grid_is_reproducible():
     ln = torch.full((B,), n, dtype=torch.int32, device=DEV)
     scale = 1 / np.sqrt(D)
     outs = {}
-    for impl in (2, 5, 1):
+    for impl in (2, 1):
         ctx = _ctx("bf16", H, D, B=B, cap=cap)
         ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, impl)
         first = None
@@ -357,6 +357,6 @@ def test_prefill_attention_large_grid_is_reproducible():
                 assert torch.equal(first.view(torch.int16), out.view(torch.int16)), f"run {rep} differs"
         outs[impl] = wl.from_torch(first)
         assert ctx.device_status()[0] == 0
-    for impl in (2, 5):
+    for impl in (2,):
         mx, rl = pc.att_errors(outs[impl], outs[1])
         assert mx <= pc.ATT_MAXABS and rl <= pc.ATT_RELL2, (impl, mx, rl)
