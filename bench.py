@@ -39,7 +39,7 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-every", type=int, default=64, help="decode steps between timed attention launches")
-    ap.add_argument("--micro", default="", choices=["", "decode", "predictor", "select", "compact", "prefill", "nocache"],
+    ap.add_argument("--micro", default="", choices=["", "decode", "predictor", "select", "compact", "compact_layers", "prefill", "nocache"],
                     help="time one stage alone on the config's shapes (small memory; used for ncu captures)")
     ap.add_argument("--micro-layers", type=int, default=2, help="layers of cache / source held in --micro mode")
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
@@ -112,6 +112,21 @@ def micro(args):
         keepm = torch.empty(B, cfg.n_vis, dtype=torch.uint8, device=dev)
         work, unit = 2.0 * rows * cfg.hidden * cfg.pred_hidden, "TFLOP/s"
         calls = [lambda l=l: ctx.prefill_select(pd, xs[l], n_vis, k_arr, score, kept, keepm) for l in range(NL)]
+    elif args.micro == "compact_layers":
+        # K and V of `micro_layers` layers under one decision in ONE call (one plan, a run of overlapped copies)
+        T = cfg.n_vis + cfg.n_text
+        pool = min(NL, 4)
+        src = [wl.device_normal(cfg, wl.S_K, (B, T, H, D), dev, sub=i) for i in range(2 * pool)]
+        caches = [torch.empty(B, H, cfg.cap, D, dtype=tdt, device=dev) for _ in range(2 * NL)]
+        keep = torch.zeros(B, cfg.n_vis, dtype=torch.uint8, device=dev)
+        idx = torch.stack([torch.randperm(cfg.n_vis, device=dev)[: cfg.k_vis] for _ in range(B)])
+        keep.scatter_(1, idx, 1)
+        t_src = torch.full((B,), T, **i32)
+        ln, zero = torch.zeros(B, **i32), torch.zeros(B, **i32)
+        srcs = [src[j % (2 * pool)] for j in range(2 * NL)]
+        work = 2 * 2 * B * cfg.n0 * H * D * cfg.elt_bytes * NL
+        calls = [lambda: (ln.copy_(zero), ctx.compact_kv_layers(srcs, caches, keep, t_src, ln, commit=True))]
+        NL = 1
     elif args.micro in ("compact", "prefill"):
         T = cfg.n_vis + cfg.n_text
         src = [wl.device_normal(cfg, wl.S_K, (B, T, H, D), dev, sub=i) for i in range(2 * NL)]

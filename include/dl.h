@@ -55,9 +55,8 @@ enum {
   DL_OPT_PREFILL_ATTN_IMPL = 2, /* 0 auto, 1 CUDA-core kernel, 2 tcgen05 tensor-core kernel (bf16, D=128) */
   DL_OPT_DECODE_CHUNK = 3,      /* cache rows per decode work item (0 = chosen by the library) */
   DL_OPT_DECODE_IMPL = 4,       /* 0 auto, 1 CUDA-core kernel, 2 tensor-core (mma.sync) kernel (bf16, D=128) */
-  DL_OPT_COMPACT_IMPL = 5       /* 0 auto, 1 register-staged copy kernel, 2 bulk-copy (TMA) kernel by tiles of 32
-                                 * source tokens, 3 bulk-copy kernel over even ranges of kept rows with one tensor
-                                 * store per row (auto: 3 for up to 2048 sequences, else 2) */
+  DL_OPT_COMPACT_IMPL = 5       /* 0 auto, 1 register-staged copy kernel, 2 bulk-copy (TMA) kernel over even ranges of kept
+                                 * rows with one tensor store per row (auto: 2 for up to 2048 sequences, else 1) */
 };
 
 typedef struct {
@@ -117,7 +116,9 @@ int32_t dl_predictor_scores(dl_ctx* ctx, const dl_predictor* p, const void* x, i
  * as -inf (and sets DL_WARN_NAN).
  *   score dev [B][n_vis_max]; n_vis dev [B] or NULL (= n_vis_max); k dev [B], 0 <= k[b] <= n_vis[b]
  *   (a larger k[b] is clamped to n_vis[b]); kept_idx_out dev [B][k_max] ascending, unused slots -1
- *   (may be NULL); keep_out dev [B][n_vis_max] 0/1 (padding slots 0).  n_vis_max <= 16384. */
+ *   (may be NULL); keep_out dev [B][n_vis_max] 0/1 (padding slots 0).  n_vis_max <= 16384.
+ *   k_max must cover every k[b]: where it does not, the index list holds the first k_max kept indices only
+ *   (the mask is complete) and DL_ERR_INVALID_ARG is recorded in the status word with the sequence index. */
 int32_t dl_topk_from_scores(dl_ctx* ctx, const float* score, const int32_t* n_vis, const int32_t* k,
                             int32_t B, int32_t n_vis_max, int32_t* kept_idx_out, int32_t k_max,
                             uint8_t* keep_out, void* stream);
@@ -146,6 +147,17 @@ int32_t dl_prefill_select(dl_ctx* ctx, const dl_predictor* p_img, const void* x_
 int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
                       int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
                       void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, void* stream);
+
+/* The same for n_tensors tensors that share ONE decision (Sec. 3.3.1: the mask is made once and used by every
+ * later layer): K, V (and Q or hidden rows) of all layers in one call.  One plan (count, capacity check, length
+ * commit) and a run of copy launches that overlap one another's start-up and tail; everything queued after the
+ * call still finds all copies complete.  Same result, bit for bit, as n_tensors single-tensor calls of
+ * dl_compact_kv with commit = 0 followed by the length commit.
+ *   srcs, caches HOST arrays of n_tensors device pointers: srcs[i] [B][t_src_max][H][D] -> caches[i] [B][H][cap][D],
+ *   every tensor appended at row cache_len[b]; the other arguments as for dl_compact_kv.  Needs the workspace. */
+int32_t dl_compact_kv_layers(dl_ctx* ctx, int32_t n_tensors, const void* const* srcs, void* const* caches,
+                             const uint8_t* keep, int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max,
+                             int32_t cap, int32_t* cache_len, int32_t commit, void* stream);
 
 /* dl_compact_kv with the SOURCE rows in pinned host memory (Eq. 5 / Eq. 11: only the kept rows enter the
  * reduced set, so only they need to reach the GPU).  The copy kernel reads the kept rows straight from host
@@ -257,6 +269,15 @@ int32_t dl_decode_steps_host(dl_ctx* ctx, const dl_predictor* p_txt, int32_t n_s
                              void* stage_v, void* stage_out, float* logit_dev, uint8_t* keep_dev,
                              void* const* k_caches, void* const* v_caches, int32_t cap,
                              int32_t* cache_len, float scale, void* stream);
+
+/* ---- diagnostics ----------------------------------------------------------------------- */
+
+/* Self-test of the bounded waits (no counterpart in the paper): launches one small kernel that waits, with
+ * the library's own wait routine and a bound of `polls` polls (1 .. 65536), on a barrier that can never
+ * complete.  The wait gives up, the kernel records DL_ERR_TIMEOUT (detail 0x5e1f) in the status word and
+ * returns; nothing traps and the context stays usable.  Asynchronous on `stream`; needs the workspace.
+ * dl_device_status then reports the code. */
+int32_t dl_selftest_wait_timeout(dl_ctx* ctx, int32_t polls, void* stream);
 
 /* ---- decode attention without any allocation ------------------------------------------- */
 

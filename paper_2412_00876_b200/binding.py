@@ -27,7 +27,7 @@ EXPORTS = [
     "dl_topk_from_scores", "dl_prefill_select", "dl_compact_kv", "dl_sparse_attn_prefill",
     "dl_sparse_attn_decode", "dl_decode_keep", "dl_commit_len", "dl_decode_step", "dl_decode_step_host",
     "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers", "dl_decode_nocache_select",
-    "dl_decode_steps_host", "dl_compact_kv_host",
+    "dl_decode_steps_host", "dl_compact_kv_host", "dl_selftest_wait_timeout", "dl_compact_kv_layers",
 ]
 
 
@@ -68,12 +68,14 @@ def lib() -> C.CDLL:
             "dl_prefill_select": (i32, [vp, P, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp]),
             "dl_compact_kv": (i32, [vp, vp, vp, vp, i32, vp, i32, i32, vp, vp, i32, vp, i32, vp]),
             "dl_compact_kv_host": (i32, [vp, vp, vp, vp, i32, vp, i32, i32, vp, vp, i32, vp, i32, vp]),
+            "dl_compact_kv_layers": (i32, [vp, i32, C.POINTER(vp), C.POINTER(vp), vp, i32, vp, i32, i32, i32, vp, i32, vp]),
             "dl_sparse_attn_prefill": (i32, [vp, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp]),
             "dl_sparse_attn_decode": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp]),
             "dl_sparse_attn_decode_static": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp]),
             "dl_sparse_attn_decode_layers": (i32, [vp, i32, vp, vp, vp, C.POINTER(vp), C.POINTER(vp), vp, vp, i32, i32,
                                                   f32, vp, vp]),
             "dl_decode_keep": (i32, [vp, P, vp, i32, f32, vp, vp, vp]),
+            "dl_selftest_wait_timeout": (i32, [vp, i32, vp]),
             "dl_decode_nocache_select": (i32, [vp, P, vp, vp, i32, i32, f32, vp, vp, vp]),
             "dl_commit_len": (i32, [vp, vp, i32, i32, vp, vp]),
             "dl_decode_step": (i32, [vp, P, vp, i32, f32, vp, vp, i32, vp, vp, vp, C.POINTER(vp),
@@ -202,6 +204,17 @@ class Context:
                                         _ptr(k_cache), _ptr(v_cache), cap, _ptr(cache_len), int(bool(commit)),
                                         _stream(stream)), "dl_compact_kv")
 
+    def compact_kv_layers(self, srcs, caches, keep, t_src, cache_len, commit=True, stream=None):
+        """dl_compact_kv_layers: len(srcs) tensors (K, V, Q ... of any number of layers) under one decision."""
+        n = len(srcs)
+        B, T = srcs[0].shape[0], srcs[0].shape[1]
+        cap = caches[0].shape[2]
+        keep_cols = 0 if keep is None else keep.shape[1]
+        sp, cp = self.pointer_array(srcs), self.pointer_array(caches)
+        self._check(lib().dl_compact_kv_layers(self._h, n, sp, cp, _ptr(keep), keep_cols, _ptr(t_src), B, T, cap,
+                                               _ptr(cache_len), int(bool(commit)), _stream(stream)),
+                    "dl_compact_kv_layers")
+
     def compact_kv_host(self, k_src_host, v_src_host, keep, t_src, k_cache, v_cache, cache_len, commit=True,
                         stream=None):
         """dl_compact_kv with the source rows in pinned host tensors: the kernel fetches the kept rows itself."""
@@ -257,6 +270,9 @@ class Context:
     def commit_len(self, keep, cache_len, cap, stream=None):
         self._check(lib().dl_commit_len(self._h, _ptr(keep), keep.shape[0], cap, _ptr(cache_len),
                                         _stream(stream)), "dl_commit_len")
+
+    def selftest_wait_timeout(self, polls: int = 64, stream=None):
+        self._check(lib().dl_selftest_wait_timeout(self._h, int(polls), _stream(stream)), "dl_selftest_wait_timeout")
 
     @staticmethod
     def pointer_array(tensors):

@@ -154,7 +154,7 @@ int32_t dl_set_option(dl_ctx* ctx, int32_t option, int32_t value) {
     case DL_OPT_PREFILL_ATTN_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.prefill_attn_impl = value; break;
     case DL_OPT_DECODE_CHUNK: ctx->opt.decode_chunk = value; break;
     case DL_OPT_DECODE_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.decode_impl = value; break;
-    case DL_OPT_COMPACT_IMPL: if (value > 3) return DL_ERR_INVALID_ARG; ctx->opt.compact_impl = value; break;
+    case DL_OPT_COMPACT_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.compact_impl = value; break;
     default: return DL_ERR_INVALID_ARG;
   }
   return DL_OK;
@@ -238,6 +238,33 @@ int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const u
   DeviceGuard g(ctx->device);
   return cuda_status(ctx, launch_compact(ctx, k_src, v_src, keep, keep_cols, t_src, B, t_src_max, k_cache, v_cache, cap,
                                          cache_len, commit, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t dl_compact_kv_layers(dl_ctx* ctx, int32_t n_tensors, const void* const* srcs, void* const* caches,
+                             const uint8_t* keep, int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max,
+                             int32_t cap, int32_t* cache_len, int32_t commit, void* stream) {
+  if (!ctx || n_tensors < 0 || B < 0 || t_src_max < 0 || cap <= 0 || keep_cols < 0) return DL_ERR_INVALID_ARG;
+  if (n_tensors == 0 || B == 0 || t_src_max == 0) return DL_OK;
+  if (!srcs || !caches || !cache_len) return DL_ERR_INVALID_ARG;
+  for (int32_t i = 0; i < n_tensors; ++i) {
+    if (!srcs[i] || !caches[i]) return DL_ERR_INVALID_ARG;
+    if (misaligned(srcs[i]) || misaligned(caches[i])) return DL_ERR_ALIGNMENT;
+  }
+  if (!ctx->ws.base || B > ctx->ws.max_batch) return DL_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // one plan, then the tensors two by two: every copy launch lets the next one start while it drains and
+  // waits for its predecessor before it ends
+  const int32_t launches = (n_tensors + 1) / 2;
+  for (int32_t l = 0; l < launches; ++l) {
+    const void* v_src = 2 * l + 1 < n_tensors ? srcs[2 * l + 1] : nullptr;
+    void* v_cache = 2 * l + 1 < n_tensors ? caches[2 * l + 1] : nullptr;
+    const int32_t chained = launches > 1 ? (1 | (l > 0 ? 2 : 0)) : 0;
+    cudaError_t e = launch_compact(ctx, srcs[2 * l], v_src, keep, keep_cols, t_src, B, t_src_max, caches[2 * l], v_cache,
+                                   cap, cache_len, commit, s, 0, l > 0, chained);
+    if (e != cudaSuccess) return cuda_status(ctx, e);
+  }
+  return DL_OK;
 }
 
 // The device's address of a pinned, device-reachable host buffer (nullptr if it is anything else).

@@ -63,7 +63,7 @@ struct Options {
   int32_t prefill_attn_impl = 0;
   int32_t decode_chunk = 0;
   int32_t decode_impl = 0;
-  int32_t compact_impl = 0;            // 0 auto, 1 register-staged copy kernel, 2 bulk-copy kernel
+  int32_t compact_impl = 0;            // 0 auto, 1 register-staged copy kernel, 2 bulk-copy (TMA) kernel
   int32_t in_layer_stack = 0;          // set by the layer-stack call around its launches (not a user option)
 };
 
@@ -84,7 +84,7 @@ struct dl_ctx {
   cudaEvent_t ev_fork = nullptr;
   // tensor maps of cache tensors seen before (decode attention); see attn_decode.cu
   static constexpr int kMapCache = 256;
-  struct MapEntry { const void* base = nullptr; long long rows = 0; unsigned char map[128]; };
+  struct MapEntry { const void* base = nullptr; long long rows = 0, aux = 0; unsigned char map[128]; };
   mutable MapEntry map_cache[kMapCache];
   mutable int map_next = 0;
 };
@@ -118,7 +118,7 @@ cudaError_t launch_topk(const float* score, const int32_t* n_vis, const int32_t*
 cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
                            int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
                            void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, cudaStream_t s,
-                           int32_t force_impl = 0);
+                           int32_t force_impl = 0, int32_t reuse_plan = 0, int32_t chained = 0);
 
 cudaError_t launch_commit_len(const uint8_t* keep, int32_t B, int32_t cap, int32_t* cache_len,
                               cudaStream_t s);

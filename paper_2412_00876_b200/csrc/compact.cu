@@ -8,9 +8,11 @@
 //   copy : per tile of 32 source tokens, rank the kept ones by a ballot scan on top of the
 //          count of kept tokens before the tile, then move each kept row with 16-byte loads
 //          and stores (a warp moves 512 contiguous source bytes per instruction).
-// Dropped rows are never read.  The copy exists in three forms (DL_OPT_COMPACT_IMPL): register-staged by
-// token tiles, bulk (TMA) copies by token tiles, and bulk copies over even row ranges with one tensor
-// store per row, which is the one the library picks where it applies.
+// Dropped rows are never read.  The copy exists in two forms (DL_OPT_COMPACT_IMPL): register-staged by token
+// tiles (also the one that reads sources in pinned host memory), and bulk (TMA) copies over even row ranges
+// with one tensor store per row, which is the one the library picks where it applies.  Several tensors that
+// share one decision (K, V and Q of every layer) are compacted by one plan and a run of copy launches that
+// overlap each other's start-up and tail (dl_compact_kv_layers).
 #include <algorithm>
 #include <cstring>
 
@@ -86,7 +88,7 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
                     const uint8_t* __restrict__ keep, int32_t keep_cols, const int32_t* __restrict__ t_src,
                     int32_t t_max, uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, int32_t cap, int32_t H,
                     int32_t row_units, int32_t piece_units, const int32_t* plan_base,
-                    const int32_t* plan_count) {
+                    const int32_t* plan_count, int32_t chained) {
   __shared__ int sh[8];
   __shared__ int tile_tok[kTileTokens];
   __shared__ int tile_kept;
@@ -95,7 +97,13 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
   int tb = t_src ? t_src[b] : t_max;
   tb = max(0, min(tb, t_max));
   const int t0 = blockIdx.x * kTileTokens;
-  if (t0 >= tb) return;
+  // A CTA without tokens still waits for the plan kernel before it leaves: a grid whose CTAs all left early
+  // would retire before its predecessor, and the next kernel of the stream would no longer be ordered behind
+  // the plan's writes.
+  if (t0 >= tb) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    return;
+  }
   const uint8_t* kp = keep ? keep + (size_t)b * keep_cols : nullptr;
 
   // kept tokens before this tile
@@ -115,9 +123,14 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
     if (threadIdx.x == 0) tile_kept = __popc(m);
   }
   __syncthreads();
-  // launched with programmatic stream serialisation: the plan of this call is complete from here on
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (ld_plan(plan_count + b) <= 0) return;
+  // launched with programmatic stream serialisation: the plan of this call is complete from here on (a copy
+  // that follows another copy of the same plan need not wait here: its predecessor did; it waits before it ends)
+  if (!(chained & 2)) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (chained & 1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (ld_plan(plan_count + b) <= 0) {
+    if (chained & 2) asm volatile("griddepcontrol.wait;" ::: "memory");
+    return;
+  }
   const int nk = tile_kept;
   const int dst0 = ld_plan(plan_base + b) + before;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -149,123 +162,20 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
       }
     }
   }
+  // completion order inside a run of copies: this one may not end before its predecessor has
+  if (chained & 2) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-// The same copy with bulk (TMA, 1-D) transfers: a kept token row travels global -> shared memory as ONE
-// bulk load and leaves as H bulk stores of one head piece each, so no register holds data and a warp keeps
-// two rows in flight (the next row loads while this one's pieces are stored).  Four warps per CTA, two row
-// buffers per warp in dynamic shared memory.
 constexpr int kBulkWarps = 4;
 
-__global__ void __launch_bounds__(kBulkWarps * 32)
-compact_copy_bulk_kernel(const char* __restrict__ k_src, const char* __restrict__ v_src,
-                         const uint8_t* __restrict__ keep, int32_t keep_cols, const int32_t* __restrict__ t_src,
-                         int32_t t_max, char* __restrict__ k_cache, char* __restrict__ v_cache, int32_t cap, int32_t H,
-                         int32_t row_bytes, int32_t piece_bytes, const int32_t* plan_base,
-                         const int32_t* plan_count, DeviceStatus* st) {
-  extern __shared__ __align__(128) char rows_s[];
-  __shared__ uint64_t bars[kBulkWarps][2];
-  __shared__ int sh[kBulkWarps];
-  __shared__ int tile_tok[kTileTokens];
-  __shared__ int tile_kept;
-  __shared__ int sh_abort;
-  volatile int* abort_flag = &sh_abort;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int b = blockIdx.y;
-  int tb = t_src ? t_src[b] : t_max;
-  tb = max(0, min(tb, t_max));
-  const int t0 = blockIdx.x * kTileTokens;
-  if (t0 >= tb) return;
-  const uint8_t* kp = keep ? keep + (size_t)b * keep_cols : nullptr;
-  if (threadIdx.x == 0) sh_abort = 0;
-  if (lane == 0) {
-    mbar_init(smem_u32(&bars[warp][0]), 1);
-    mbar_init(smem_u32(&bars[warp][1]), 1);
-    fence_mbar_init();
-  }
-  // kept tokens before this tile
-  int before = 0;
-  if (kp) {
-    for (int i = threadIdx.x; i < t0; i += kBulkWarps * 32) before += (i >= keep_cols || kp[i] != 0);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
-    if (lane == 0) sh[warp] = before;
-  }
-  // rank the tile's kept tokens
-  if (threadIdx.x < 32) {
-    int t = t0 + threadIdx.x;
-    bool f = (t < tb) && (kp == nullptr || t >= keep_cols || kp[t] != 0);
-    unsigned m = __ballot_sync(0xffffffffu, f);
-    if (f) tile_tok[__popc(m & ((1u << threadIdx.x) - 1u))] = t;
-    if (threadIdx.x == 0) tile_kept = __popc(m);
-  }
-  __syncthreads();
-  if (kp) {
-    before = 0;
-#pragma unroll
-    for (int w = 0; w < kBulkWarps; ++w) before += sh[w];
-  } else {
-    before = t0;
-  }
-  // launched with programmatic stream serialisation: the plan of this call is complete from here on
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (ld_plan(plan_count + b) <= 0) return;
-  const int nk = tile_kept;
-  const int dst0 = ld_plan(plan_base + b) + before;
-  const int n_tensors = v_src ? 2 : 1;
-  const int total = nk * n_tensors;
-  const int my_jobs = total > warp ? (total - warp + kBulkWarps - 1) / kBulkWarps : 0;
-  char* buf = rows_s + (size_t)warp * 2 * row_bytes;
-  const size_t head_stride = (size_t)cap * piece_bytes;
-  auto load = [&](int idx) {                      // job idx of this warp: (token, tensor) pair warp + idx * warps
-    const int job = warp + idx * kBulkWarps;
-    const int j = job / n_tensors, which = job - j * n_tensors;
-    const char* src = (which ? v_src : k_src) + ((size_t)b * t_max + tile_tok[j]) * row_bytes;
-    const uint32_t bar = smem_u32(&bars[warp][idx & 1]);
-    mbar_expect_tx(bar, (uint32_t)row_bytes);
-    bulk_g2s(smem_u32(buf + (size_t)(idx & 1) * row_bytes), src, (uint32_t)row_bytes, bar);
-  };
-  int issued = 0;                                 // loads issued so far (the same count in every lane)
-  if (my_jobs > 0) {
-    if (lane == 0) load(0);
-    issued = 1;
-  }
-  for (int idx = 0; idx < my_jobs; ++idx) {
-    if (idx + 1 < my_jobs) {
-      // the other buffer held job idx - 1: every lane's stores of it must have read it before it is refilled
-      bulk_group_wait_read_all();
-      __syncwarp();
-      if (lane == 0) load(idx + 1);
-      issued = idx + 2;
-    }
-    const bool ok = mbar_wait(smem_u32(&bars[warp][idx & 1]), (idx >> 1) & 1, abort_flag);
-    if (!ok) break;
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    const int job = warp + idx * kBulkWarps;
-    const int j = job / n_tensors, which = job - j * n_tensors;
-    char* dst = (which ? v_cache : k_cache) + (size_t)b * H * head_stride + (size_t)(dst0 + j) * piece_bytes;
-    const uint32_t src = smem_u32(buf + (size_t)(idx & 1) * row_bytes);
-    for (int h = lane; h < H; h += 32) bulk_s2g(dst + (size_t)h * head_stride, src + (uint32_t)(h * piece_bytes), (uint32_t)piece_bytes);
-    bulk_group_commit();
-  }
-  bulk_group_wait_read_all();                     // shared memory is read before the CTA ends
-  if (*abort_flag) {
-    // a load that was issued must land before the CTA's shared memory is released
-    if (lane == 0) {
-      report_status(st, DL_ERR_TIMEOUT, blockIdx.y);
-      for (int j = max(0, issued - 2); j < issued; ++j)
-        for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&bars[warp][j & 1]), (j >> 1) & 1); ++i) __nanosleep(40);
-    }
-  }
-}
-
-// The bulk copy again, with the work dealt evenly: the kept rows of the whole batch, in (sequence, rank)
-// order, are cut into one contiguous range per CTA (the tile kernel above gives a CTA 32 source tokens,
-// so a tile of text tokens, all kept, carries four times the rows of a tile of vision tokens at a 25 % keep
-// rate, and the CTAs that start last finish long after the rest).  A CTA reads the per-sequence row counts
-// of the plan, finds its range, and for each sequence the range touches ranks the sequence's mask once
-// (a block scan over 128 token segments) to list the tokens whose rank falls inside; its warps then move
-// those rows exactly as above, their two-buffer pipelines running on across lists.  Up to 2048 sequences.
+// The copy with bulk (TMA) transfers and the work dealt evenly: a kept token row travels global -> shared
+// memory as ONE 1-D bulk load and leaves as one tensor store (or H bulk stores of one head piece each), so no
+// register holds data and a warp keeps two rows in flight.  The kept rows of the whole batch, in (sequence,
+// rank) order, are cut into one contiguous range per CTA (dealing source tokens instead would give a CTA of
+// text tokens, all kept, four times the rows of a CTA of vision tokens at a 25 % keep rate).  A CTA reads the
+// per-sequence row counts of the plan, finds its range, and for each sequence the range touches ranks the
+// sequence's mask once (a block scan over 128 token segments) to list the tokens whose rank falls inside; its
+// warps then move those rows, their two-buffer pipelines running on across lists.  Up to 2048 sequences.
 constexpr int kRowsList = 64;
 constexpr int kRowsMaxBatch = 2048;
 
@@ -291,13 +201,31 @@ static bool encode_row_map(void* fn, void* out, const void* base, int piece_byte
                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Encoding a tensor map costs a few microseconds on the host; the caches of a model come back at every batch,
+// so the context remembers the row maps it has built (keyed by base, shape and row pitch).
+static bool cached_row_map(const dl_ctx* ctx, void* out, const void* base, int piece_bytes, int cap, long long bh, int H) {
+  const long long key_rows = -((long long)cap * 1024 + piece_bytes / 4);    // negative: never equal to a decode map's row count
+  for (int i = 0; i < dl_ctx::kMapCache; ++i) {
+    const dl_ctx::MapEntry& e = ctx->map_cache[i];
+    if (e.base == base && e.rows == key_rows && e.aux == bh) { memcpy(out, e.map, 128); return true; }
+  }
+  alignas(64) unsigned char tmp[128];
+  if (!encode_row_map(ctx->tmap_encode, tmp, base, piece_bytes, cap, bh, H)) return false;
+  dl_ctx::MapEntry& e = ctx->map_cache[ctx->map_next];
+  memcpy(e.map, tmp, 128);
+  e.base = base; e.rows = key_rows; e.aux = bh;
+  ctx->map_next = (ctx->map_next + 1) % dl_ctx::kMapCache;
+  memcpy(out, tmp, 128);
+  return true;
+}
+
 __global__ void __launch_bounds__(kBulkWarps * 32)
 compact_copy_rows_kernel(const char* __restrict__ k_src, const char* __restrict__ v_src,
                          const uint8_t* __restrict__ keep, int32_t keep_cols, const int32_t* __restrict__ t_src,
                          int32_t t_max, char* __restrict__ k_cache, char* __restrict__ v_cache, int32_t cap, int32_t H,
                          int32_t row_bytes, int32_t piece_bytes, int32_t B, const int32_t* plan_base,
                          const int32_t* plan_count, DeviceStatus* st, const __grid_constant__ RowMaps maps,
-                         int32_t use_maps) {
+                         int32_t use_maps, int32_t chained) {
   extern __shared__ __align__(128) char rows_s[];
   __shared__ uint64_t bars[kBulkWarps][2];
   __shared__ int sh[kBulkWarps];
@@ -313,8 +241,13 @@ compact_copy_rows_kernel(const char* __restrict__ k_src, const char* __restrict_
     mbar_init(smem_u32(&bars[warp][1]), 1);
     fence_mbar_init();
   }
-  // launched with programmatic stream serialisation: the plan of this call is complete from here on
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Launched with programmatic stream serialisation: the plan of this call is complete from here on.  In a run of
+  // copies that share one plan (chained: bit 0 = let the next kernel of the stream start while this one drains,
+  // bit 1 = this copy follows another copy of the same plan) only the first waits here; the others started after
+  // it had, so the plan is complete for them too, and they wait for their predecessor before they END, which keeps
+  // the order of completion that the stream promises to whatever follows the run.
+  if (!(chained & 2)) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (chained & 1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   int part = 0;
   for (int b = tid; b < B; b += kThreads) {
     const int c = max(ld_plan(plan_count + b), 0);                    // -1: the sequence does not fit, skip it
@@ -329,7 +262,10 @@ compact_copy_rows_kernel(const char* __restrict__ k_src, const char* __restrict_
 #pragma unroll
   for (int w = 0; w < kBulkWarps; ++w) n_rows += sh[w];
   const long long lo = n_rows * blockIdx.x / gridDim.x, hi = n_rows * (blockIdx.x + 1) / gridDim.x;
-  if (hi <= lo) return;
+  if (hi <= lo) {
+    if (chained & 2) asm volatile("griddepcontrol.wait;" ::: "memory");
+    return;
+  }
 
   const int n_tensors = v_src ? 2 : 1;
   char* buf = rows_s + (size_t)warp * 2 * row_bytes;
@@ -422,6 +358,7 @@ compact_copy_rows_kernel(const char* __restrict__ k_src, const char* __restrict_
     }
   }
   bulk_group_wait_read_all();                     // shared memory is read before the CTA ends
+  if (chained & 2) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (*abort_flag) {
     // a load that was issued must land before the CTA's shared memory is released
     if (lane == 0) {
@@ -432,20 +369,27 @@ compact_copy_rows_kernel(const char* __restrict__ k_src, const char* __restrict_
   }
 }
 
+// One compaction call: the plan kernel (unless `reuse_plan`: the caller's previous launch in this stream made it
+// for the same mask), then the copy.  With `chained` the copy kernel is one of a run of copies that share a
+// plan (several layers, one decision): it lets the next one start while it drains and, before it ends, waits for
+// its predecessor, so that whatever follows the run finds all of it complete.
 cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
                            int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache,
                            void* v_cache, int32_t cap, int32_t* cache_len, int32_t commit, cudaStream_t s,
-                           int32_t force_impl) {
+                           int32_t force_impl, int32_t reuse_plan, int32_t chained) {
   if (B == 0 || t_src_max == 0) return cudaSuccess;
   const int impl = force_impl ? force_impl : ctx->opt.compact_impl;
   const dl_model_desc& d = ctx->desc;
   const int elt = d.dtype == DL_F32 ? 4 : 2;
   const int piece_units = d.head_dim * elt / 16;
   const int row_units = piece_units * d.n_heads;
-  compact_plan_kernel<<<B, kPlanThreads, 0, s>>>(keep, keep_cols, t_src, t_src_max, cap, cache_len, commit,
-                                                 ctx->ws.plan_base, ctx->ws.plan_count, ctx->ws.status);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  cudaError_t e = cudaSuccess;
+  if (!reuse_plan) {
+    compact_plan_kernel<<<B, kPlanThreads, 0, s>>>(keep, keep_cols, t_src, t_src_max, cap, cache_len, commit,
+                                                   ctx->ws.plan_base, ctx->ws.plan_count, ctx->ws.status);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
   dim3 grid((t_src_max + kTileTokens - 1) / kTileTokens, B);
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
@@ -454,48 +398,40 @@ cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_s
   cfg.attrs = attr; cfg.numAttrs = 1;
   cfg.gridDim = grid; cfg.stream = s;
   // bulk-copy kernel where two row buffers per warp fit the shared memory (they do for every shape at hand:
-  // a row is H * D * elt bytes, 8 KB for 32 heads of 128 bf16)
+  // a row is H * D * elt bytes, 8 KB for 32 heads of 128 bf16) and the batch fits its table of row counts
   const size_t row_bytes = (size_t)row_units * 16, bulk_smem = 2 * kBulkWarps * row_bytes;
-  if (impl != 1 && bulk_smem + 1024 <= (size_t)ctx->smem_optin) {
+  if (impl != 1 && B <= kRowsMaxBatch && bulk_smem + 1024 <= (size_t)ctx->smem_optin) {
     static int attr_set[64];
     int& set_for = attr_set[ctx->device & 63];
     if (set_for < (int)bulk_smem) {
-      e = cudaFuncSetAttribute(compact_copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk_smem);
-      if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(compact_copy_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk_smem);
+      e = cudaFuncSetAttribute(compact_copy_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk_smem);
       if (e != cudaSuccess) return e;
       set_for = (int)bulk_smem;
     }
     cfg.blockDim = dim3(kBulkWarps * 32); cfg.dynamicSmemBytes = bulk_smem;
-    if (impl != 2 && B <= kRowsMaxBatch) {
-      // evenly dealt rows: as many CTAs as fit the GPU at once, fewer when the batch has few rows
-      const size_t per_cta = bulk_smem + 10 * 1024;
-      const long long resident = (long long)ctx->sm_count * std::max<size_t>(1, (size_t)ctx->smem_optin / per_cta);
-      const long long by_rows = ((long long)B * t_src_max + 7) / 8;
-      cfg.gridDim = dim3((unsigned)std::max(1LL, std::min(resident, by_rows)));
-      // one tensor store per row where the row buffers are 128-byte aligned and the maps can be made
-      RowMaps maps;
-      memset(&maps, 0, sizeof(maps));
-      const int piece_bytes = piece_units * 16;
-      int32_t use_maps = (row_bytes % 128 == 0) &&
-                         encode_row_map(ctx->tmap_encode, maps.k, k_cache, piece_bytes, cap, (long long)B * d.n_heads, d.n_heads) &&
-                         (!v_src || encode_row_map(ctx->tmap_encode, maps.v, v_cache, piece_bytes, cap, (long long)B * d.n_heads, d.n_heads));
-      return cudaLaunchKernelEx(&cfg, compact_copy_rows_kernel, (const char*)k_src, (const char*)v_src, keep,
-                                (int32_t)keep_cols, t_src, (int32_t)t_src_max, (char*)k_cache, (char*)v_cache,
-                                (int32_t)cap, (int32_t)d.n_heads, (int32_t)row_bytes, (int32_t)piece_bytes,
-                                (int32_t)B, (const int32_t*)ctx->ws.plan_base, (const int32_t*)ctx->ws.plan_count,
-                                ctx->ws.status, maps, use_maps);
-    }
-    return cudaLaunchKernelEx(&cfg, compact_copy_bulk_kernel, (const char*)k_src, (const char*)v_src, keep,
-                              (int32_t)keep_cols, t_src, (int32_t)t_src_max, (char*)k_cache, (char*)v_cache, (int32_t)cap,
-                              (int32_t)d.n_heads, (int32_t)row_bytes, (int32_t)(piece_units * 16),
-                              (const int32_t*)ctx->ws.plan_base, (const int32_t*)ctx->ws.plan_count, ctx->ws.status);
+    // evenly dealt rows: as many CTAs as fit the GPU at once, fewer when the batch has few rows
+    const size_t per_cta = bulk_smem + 10 * 1024;
+    const long long resident = (long long)ctx->sm_count * std::max<size_t>(1, (size_t)ctx->smem_optin / per_cta);
+    const long long by_rows = ((long long)B * t_src_max + 7) / 8;
+    cfg.gridDim = dim3((unsigned)std::max(1LL, std::min(resident, by_rows)));
+    // one tensor store per row where the row buffers are 128-byte aligned and the maps can be made
+    RowMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    const int piece_bytes = piece_units * 16;
+    int32_t use_maps = (row_bytes % 128 == 0) &&
+                       cached_row_map(ctx, maps.k, k_cache, piece_bytes, cap, (long long)B * d.n_heads, d.n_heads) &&
+                       (!v_src || cached_row_map(ctx, maps.v, v_cache, piece_bytes, cap, (long long)B * d.n_heads, d.n_heads));
+    return cudaLaunchKernelEx(&cfg, compact_copy_rows_kernel, (const char*)k_src, (const char*)v_src, keep,
+                              (int32_t)keep_cols, t_src, (int32_t)t_src_max, (char*)k_cache, (char*)v_cache,
+                              (int32_t)cap, (int32_t)d.n_heads, (int32_t)row_bytes, (int32_t)piece_bytes,
+                              (int32_t)B, (const int32_t*)ctx->ws.plan_base, (const int32_t*)ctx->ws.plan_count,
+                              ctx->ws.status, maps, use_maps, (int32_t)chained);
   }
   cfg.blockDim = dim3(kCopyThreads); cfg.dynamicSmemBytes = 0;
   return cudaLaunchKernelEx(&cfg, compact_copy_kernel, (const uint4*)k_src, (const uint4*)v_src, keep, (int32_t)keep_cols,
                             t_src, (int32_t)t_src_max, (uint4*)k_cache, (uint4*)v_cache, (int32_t)cap, (int32_t)d.n_heads,
                             (int32_t)row_units, (int32_t)piece_units, (const int32_t*)ctx->ws.plan_base,
-                            (const int32_t*)ctx->ws.plan_count);
+                            (const int32_t*)ctx->ws.plan_count, (int32_t)chained);
 }
 
 __global__ void commit_len_kernel(const uint8_t* __restrict__ keep, int32_t B, int32_t cap,

@@ -44,9 +44,9 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false (and raises *abort) when the bound is hit or another warp aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, int limit = kSpinLimit) {
   if (mbar_try_wait(bar, parity)) return !*abort;            // fast path: the phase is already complete
-  for (int i = 0; i < kSpinLimit; ++i) {
+  for (int i = 0; i < limit; ++i) {
     if (*abort) return false;
     if (mbar_try_wait(bar, parity)) return true;
     if (i > 32) __nanosleep(40);

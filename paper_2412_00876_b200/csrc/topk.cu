@@ -68,6 +68,7 @@ topk_kernel(const float* __restrict__ score, const int32_t* __restrict__ n_vis,
   bool saw_nan = false;
   for (int i = tid; i < n; i += kTopkThreads) keys[i] = score_key(s[i], &saw_nan);
   if (saw_nan) report_status(st, DL_WARN_NAN, b);
+  if (tid == 0 && kept_idx != nullptr && kk > k_max) report_status(st, DL_ERR_INVALID_ARG, b);   // the index list is cut
   if (tid == 0) { sh_prefix = 0u; sh_remaining = kk; }
   __syncthreads();
 

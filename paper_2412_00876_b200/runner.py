@@ -85,11 +85,14 @@ class BatchRunner:
         self.cache_len.zero_()
         ctx.prefill_select(self.p_img, self.x_vis, self.n_vis, self.k_arr, self.score, self.kept_idx, self.keep_vis)
         self.launches += 2
+        # K and V of every layer under the one decision: one plan, one run of overlapped copy launches
+        srcs, caches = [], []
         for l in range(L):
             i = l % self.src_pool
-            ctx.compact_kv(self.k_src[i], self.v_src[i], self.keep_vis, self.t_src, self.k_cache[l], self.v_cache[l],
-                           self.cache_len, commit=(l == L - 1))
-        self.launches += 2 * L
+            srcs += [self.k_src[i], self.v_src[i]]
+            caches += [self.k_cache[l], self.v_cache[l]]
+        ctx.compact_kv_layers(srcs, caches, self.keep_vis, self.t_src, self.cache_len, commit=True)
+        self.launches += 1 + L
         for l in range(L):
             i = l % self.src_pool
             ctx.compact_kv(self.q_src[i], None, self.keep_vis, self.t_src, self.q_cache, None, self.q_len, commit=False)

@@ -126,3 +126,23 @@ def test_pipelined_host_fed_steps_equal_single_host_steps():
         assert torch.equal(a[3][l].view(torch.int16), b[3][l].view(torch.int16))
     assert torch.equal(a[4], b[4])
 
+
+
+def test_a_bounded_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """The library's wait routine on a barrier that never completes (a dedicated self-test kernel: no copy in
+    flight, nothing to drain): it gives up after its bound, DL_ERR_TIMEOUT reaches the status word, the call
+    returns well within a second and the next kernels of the same context work."""
+    import time
+    from paper_2412_00876_b200 import binding as dl
+    ctx = dl.Context(256, 4, 128, 64, torch.bfloat16, 0, max_batch=4, max_rows=4, cap=128)
+    t0 = time.perf_counter()
+    ctx.selftest_wait_timeout(polls=200)
+    code, detail = ctx.device_status()                    # synchronises
+    assert time.perf_counter() - t0 < 1.0
+    assert code == dl.DL_ERR_TIMEOUT and detail == 0x5E1F
+    assert ctx.device_status()[0] == 0                    # reading clears it
+    logit = torch.tensor([1.0, -1.0, 0.0, 2.0], device="cuda:0")
+    keep = torch.empty(4, dtype=torch.uint8, device="cuda:0")
+    ctx.decode_keep(None, None, logit, keep)
+    assert keep.cpu().tolist() == [1, 0, 0, 1] and ctx.device_status()[0] == 0
+    ctx.close()

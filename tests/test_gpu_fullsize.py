@@ -20,7 +20,7 @@ def _f64(t):
     return wl.from_torch(t)
 
 
-@pytest.mark.parametrize("cid,n_steps", [(3, 24), (5, 8)])
+@pytest.mark.parametrize("cid,n_steps", [(3, 24), (4, 8), (5, 8)])
 def test_full_size_sampled(cid, n_steps):
     from paper_2412_00876_b200.runner import BatchRunner
     free, _ = torch.cuda.mem_get_info()

@@ -106,3 +106,36 @@ def test_nocache_mask_keeps_the_last_generated_token():
             assert m[b, i] == int(want)
     # without the forced token it is Eq. 6's per-token decision
     assert np.array_equal(orc.nocache_keep(z, None)[:, :-1], orc.decode_keep(z)[:, :-1])
+
+
+def test_prefill_keep_mask_ragged_batch_by_brute_force():
+    """M = M^I u {1}^{N_T} (Sec. 3.3.3) for a batch whose sequences have different numbers of vision AND text
+    tokens: written out slot by slot (no slicing), and applied through append_rows it must leave exactly
+    k_b + N_T(b) rows, the kept vision rows first and in order, then the text rows."""
+    rng = np.random.default_rng(5)
+    B, nv_max = 4, 9
+    n_vis = np.array([9, 4, 0, 7])
+    n_text = np.array([3, 5, 2, 0])
+    k = np.array([2, 4, 0, 3])
+    score = rng.normal(size=(B, nv_max))
+    _, keep_vis = orc.prefill_select(score, n_vis, k)
+    m = orc.prefill_keep_mask(keep_vis, n_vis, n_text)
+    assert m.shape == (B, nv_max + 5)
+    for b in range(B):
+        for t in range(m.shape[1]):
+            if t < nv_max:
+                want = 1 if (t < n_vis[b] and keep_vis[b, t]) else 0
+            else:
+                want = 1 if t - nv_max < n_text[b] else 0
+            assert m[b, t] == want, (b, t)
+        assert m[b].sum() == k[b] + n_text[b]
+    # through the compaction: source rows are numbered, so the cache shows which rows arrived and in what order
+    T = m.shape[1]
+    src = np.arange(B * T, dtype=np.float32).reshape(B, T, 1, 1)
+    cache = np.full((B, 1, T, 1), -1.0, np.float32)
+    ln = np.zeros(B, np.int32)
+    st, cnt = orc.append_rows(src, src, m, None, cache, cache.copy(), ln)
+    assert st == orc.OK and list(ln) == list(k + n_text)
+    for b in range(B):
+        rows = [t for t in range(nv_max) if t < n_vis[b] and keep_vis[b, t]] + [nv_max + j for j in range(n_text[b])]
+        assert list(cache[b, 0, : ln[b], 0]) == [float(b * T + t) for t in rows]
