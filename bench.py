@@ -38,8 +38,9 @@ def parse():
                     help="replay decode steps from CUDA graphs: 1 yes, 0 no, -1 only for launch-bound workloads (B*L < 64)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill-record", action="store_true")
     ap.add_argument("--sample-every", type=int, default=64, help="decode steps between timed attention launches")
-    ap.add_argument("--micro", default="", choices=["", "decode", "predictor", "select", "compact", "compact_layers", "prefill", "nocache"],
+    ap.add_argument("--micro", default="", choices=["", "decode", "keep", "predictor", "select", "compact", "compact_layers", "prefill", "nocache"],
                     help="time one stage alone on the config's shapes (small memory; used for ncu captures)")
     ap.add_argument("--micro-layers", type=int, default=2, help="layers of cache / source held in --micro mode")
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
@@ -53,7 +54,7 @@ def parse():
 
 
 # ------------------------------------------------------------------------------ single-stage timing
-def micro(args):
+def micro(args, emit=True):
     """Times one kernel family alone, launches rotating over `micro_layers` independent buffers so
     that consecutive launches never find their inputs in L2.  Prints one JSON line."""
     import numpy as np
@@ -91,6 +92,16 @@ def micro(args):
         work = (2 * (int(lens.sum()) + B) + 2 * B) * H * D * cfg.elt_bytes
         calls = [lambda l=l: ctx.sparse_attn_decode(q[l], kt[l], vt[l], kc[l], vc[l], ln, keep, scale, out[l])
                  for l in range(NL)]
+    elif args.micro == "keep":
+        # the decode decision of one step: predictor on B rows + keep test (one launch for bf16 models)
+        p = wl.make_predictor(cfg, "txt")
+        pd = dl.Predictor(wl.to_torch(p.w1, cfg.dtype, dev), torch.from_numpy(p.b1).to(dev),
+                          torch.from_numpy(p.w2).to(dev), p.b2)
+        xs = [wl.device_normal(cfg, wl.S_X_TXT, (B, cfg.hidden), dev, sub=i) for i in range(NL)]
+        logit = torch.empty(B, dtype=torch.float32, device=dev)
+        keepf = torch.empty(B, dtype=torch.uint8, device=dev)
+        work, unit = (cfg.hidden * cfg.pred_hidden + B * cfg.hidden) * cfg.elt_bytes, "GB/s"     # weights + rows read
+        calls = [lambda l=l: ctx.decode_keep(pd, xs[l], logit, keepf) for l in range(NL)]
     elif args.micro == "predictor":
         p = wl.make_predictor(cfg, "img")
         pd = dl.Predictor(wl.to_torch(p.w1, cfg.dtype, dev), torch.from_numpy(p.b1).to(dev),
@@ -204,12 +215,48 @@ def micro(args):
     queued = a.elapsed_time(b) / args.steps
     code, detail = ctx.device_status()
     rate = work / (med * 1e-3) / (1e9 if unit == "GB/s" else 1e12)
-    print(json.dumps({"micro": args.micro, "workload": cfg.name, "median_us": med * 1e3, "min_us": ts[0] * 1e3,
-                      "algorithmic_work": work, "rate": rate, "unit": unit, "launches": args.steps,
-                      "queued_us": queued * 1e3,
-                      "queued_rate": work / (queued * 1e-3) / (1e9 if unit == "GB/s" else 1e12),
-                      "device_status": code}), flush=True)
+    rec = {"micro": args.micro, "workload": cfg.name, "median_us": med * 1e3, "min_us": ts[0] * 1e3,
+           "algorithmic_work": work, "rate": rate, "unit": unit, "launches": args.steps,
+           "queued_us": queued * 1e3,
+           "queued_rate": work / (queued * 1e-3) / (1e9 if unit == "GB/s" else 1e12),
+           "device_status": code}
+    if emit:
+        print(json.dumps(rec), flush=True)
     ctx.close()
+    del gate, calls
+    torch.cuda.empty_cache()
+    return rec
+
+
+def measured_peaks():
+    """(HBM GB/s, bf16 TFLOP/s burst, source): the machine's measured peaks, else the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        pj = json.load(open(path))
+        return float(pj["hbm_gbs"]), float(pj["bf16_tflops"]), "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def prefill_record(cids, reps=24):
+    """The prefill half of the metric, stage by stage (CUDA events, launches rotating over buffers larger than L2):
+    select = predictor scores + top-k of a whole batch; compaction = K and V of 8 layers under one decision in one
+    call; attention = one layer.  One entry per workload."""
+    import types
+    hbm, tfl, src = measured_peaks()
+    out = []
+    for cid in cids:
+        def run(stage, layers):
+            return micro(types.SimpleNamespace(config=cid, micro=stage, steps=reps, warmup=4, micro_layers=layers,
+                                               micro_len=0, decode_chunk=0, prefill_impl=0, compact_impl=0), emit=False)
+        sel, cmp_, att = run("select", 4), run("compact_layers", 8), run("prefill", 4)
+        out.append({"workload": sel["workload"], "select_us": sel["median_us"], "select_tflops": sel["rate"],
+                    "select_frac_of_bf16_peak": sel["rate"] / tfl,
+                    "compact_8_layers_us": cmp_["median_us"], "compact_gbs": cmp_["rate"],
+                    "compact_frac_of_hbm_peak": cmp_["rate"] / hbm,
+                    "attn_us_per_layer": att["median_us"], "attn_tflops_causal": att["rate"],
+                    "attn_frac_of_bf16_peak": att["rate"] / tfl,
+                    "select_plus_attn_us": sel["median_us"] + att["median_us"], "peaks": src, "launches_timed": reps})
+    return out
 
 
 # ------------------------------------------------------------------------------ clocks
@@ -257,7 +304,7 @@ def oracle_sample(cfg, budget_s: float = 20.0):
     import numpy as np
     from oracle import dl_oracle as orc
     from paper_2412_00876_b200 import workloads as wl
-    t_all = time.perf_counter()
+    t_all, cpu_all = time.perf_counter(), time.process_time()
     Bs, H, D = min(2, cfg.B), cfg.n_heads, cfg.head_dim
     sc = cfg.scaled(B=Bs)
     scale = 1 / np.sqrt(D)
@@ -311,15 +358,24 @@ def oracle_sample(cfg, budget_s: float = 20.0):
         td = np.interp(n, lens, t_dec)
         t_decode += B * (t_keep + L * td)
     total = t_prefill + t_decode
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
-    except Exception:
-        cores = 1
+    # threads the oracle actually kept busy: its CPU time over its wall time (numpy's matmul runs on the BLAS
+    # threads, the loops over rows and heads on one)
+    wall = time.perf_counter() - t_all
+    cores = max(1, int(round((time.process_time() - cpu_all) / max(wall, 1e-9))))
     sample = (f"{Bs} sequences: prefill select; 1 layer compaction; prefill attention {hs}/{H} heads; decode "
               f"attention+append 1 layer, all heads at cache lengths {lens}; extrapolated linearly to "
-              f"B={B}, L={L}, {cfg.n_gen} decode steps (sample took {time.perf_counter() - t_all:.1f} s)")
+              f"B={B}, L={L}, {cfg.n_gen} decode steps (sample took {wall:.1f} s on "
+              f"{len(os.sched_getaffinity(0))} available host cores)")
     return B * cfg.n_gen / total, cores, sample
+
+
+def config_of(cfg, world: int) -> dict:
+    """The workload description both arms print (same keys, same values)."""
+    return {"workload": cfg.name, "B_per_gpu": cfg.B, "layers": cfg.n_layers, "n_vis": cfg.n_vis,
+            "k_vis": cfg.k_vis, "n_text": cfg.n_text, "n_gen": cfg.n_gen, "keep_rate": cfg.keep_rate,
+            "parallelism": f"batch-shards x{world}",
+            "layer_stack": "q/k/v of all layers of a step are inputs; launches of consecutive layers overlap",
+            "l2": "inputs larger than L2 (caches tens of GB; input pools > 126 MB)"}
 
 
 def reference_arm(args):
@@ -342,8 +398,7 @@ def reference_arm(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": len(vals), "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "B": cfg.B, "layers": cfg.n_layers, "n_vis": cfg.n_vis,
-                       "k_vis": cfg.k_vis, "n_text": cfg.n_text, "n_gen": cfg.n_gen},
+            "config": config_of(cfg, args.gpus),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -452,6 +507,18 @@ def main():
                "prefill_sources": "left in pinned host memory; the compaction kernel fetches the kept rows over the "
                                   "bus itself (h2d counts those rows), dropped rows are never transferred"}
 
+    # ---- the prefill half of the metric and the dominant kernel as a single launch (rank 0; small buffers of
+    # their own beside the runner's caches)
+    prefill = None
+    if rank == 0 and not args.no_prefill_record:
+        import types
+        cids = [args.config] + ([5] if args.config != 5 else [])
+        prefill = prefill_record(cids)
+        one = micro(types.SimpleNamespace(config=args.config, micro="decode", steps=24, warmup=4, micro_layers=2,
+                                          micro_len=0, decode_chunk=0, prefill_impl=0, compact_impl=0), emit=False)
+        roofline["single_launch_gbs"] = one["rate"]
+        roofline["frac_single_launch"] = one["rate"] / peak
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, cores, sample = oracle_sample(cfg)
@@ -461,12 +528,8 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-                "config": {"workload": cfg.name, "B_per_gpu": cfg.B, "layers": cfg.n_layers, "n_vis": cfg.n_vis,
-                           "k_vis": cfg.k_vis, "n_text": cfg.n_text, "n_gen": cfg.n_gen, "keep_rate": cfg.keep_rate,
-                           "parallelism": f"batch-shards x{world}", "decode_steps_from_cuda_graphs": use_graphs,
-                           "layer_stack": "q/k/v of all layers of a step are inputs; launches of consecutive layers overlap",
-                           "l2": "inputs larger than L2 (caches tens of GB; input pools > 126 MB)"},
-                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+                "config": config_of(cfg, world), "decode_steps_from_cuda_graphs": use_graphs,
+                "roofline": roofline, "prefill": prefill, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
                 "clocks": clocks}
         print(json.dumps(line), flush=True)
     runner.close()

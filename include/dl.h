@@ -229,7 +229,9 @@ int32_t dl_commit_len(dl_ctx* ctx, const uint8_t* keep, int32_t B, int32_t cap, 
                       void* stream);
 
 /* One whole decode step over a stack of L layers that share the decision: dl_decode_keep, then
- * per layer dl_sparse_attn_decode with the fused append, then dl_commit_len.
+ * per layer dl_sparse_attn_decode with the fused append, then dl_commit_len.  Same results as those calls; the
+ * library folds the decision into the predictor's launch and the length commit into the last layer's (1 + L
+ * launches per step for bf16 models).
  *   q_t, k_t, v_t, out: dev [L][B][H][D]; k_caches, v_caches: HOST arrays of L device pointers,
  *   each [B][H][cap][D].  Other arguments as in the single calls. */
 int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B,

@@ -14,23 +14,31 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdl_sparse.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-         "-Xcompiler", "-fPIC", "--use_fast_math=false"]
-FLAGS = [f for f in FLAGS if f != "--use_fast_math=false"]
+FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
+STAMP = LIB + ".src_hash"
 
 
 def _sources():
     return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cu"))
 
 
-def _newest_input():
-    paths = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
+def source_hash() -> str:
+    """SHA-256 over every file the library is built from (sources, headers, the C header) and the flags."""
+    import hashlib
+    h = hashlib.sha256(" ".join(FLAGS).encode())
+    paths = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC))
     paths.append(os.path.join(os.path.dirname(HERE), "include", "dl.h"))
-    return max(os.path.getmtime(p) for p in paths)
+    for p in paths:
+        h.update(os.path.basename(p).encode())
+        h.update(open(p, "rb").read())
+    return h.hexdigest()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_input():
+    """Builds the library unless the one in place was built from exactly these sources: the decision is taken on
+    a hash of the sources stored beside the library, not on file times (a snapshot copied elsewhere keeps neither)."""
+    want = source_hash()
+    if not force and os.path.exists(LIB) and os.path.exists(STAMP) and open(STAMP).read().strip() == want:
         return LIB
     os.makedirs(OBJ, exist_ok=True)
     extra = ["-Xptxas", "-v"] if verbose else []
@@ -51,6 +59,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
+    with open(STAMP, "w") as f:
+        f.write(want + "\n")
     return LIB
 
 

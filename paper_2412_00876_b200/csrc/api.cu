@@ -22,6 +22,7 @@ int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_
   const int32_t rows_pad = (max_rows + kPredRowTile - 1) / kPredRowTile * kPredRowTile;
   const int64_t o_ppart = take((int64_t)kPredMaxSplit * rows_pad * 4);
   const int64_t o_ptick = take((int64_t)(rows_pad / kPredRowTile + 1) * 4);
+  const int64_t o_commit = take(4);
   if (ws) {
     char* b = ws->base;
     ws->status = reinterpret_cast<DeviceStatus*>(b + o_status);
@@ -32,6 +33,7 @@ int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_
     ws->dec_slots = slots;
     ws->pred_partial = reinterpret_cast<float*>(b + o_ppart);
     ws->pred_ticket = reinterpret_cast<int32_t*>(b + o_ptick);
+    ws->dec_commit = reinterpret_cast<int32_t*>(b + o_commit);
     ws->pred_rows_padded = rows_pad;
     ws->max_batch = max_batch; ws->max_rows = max_rows; ws->cap = cap;
   }
@@ -57,8 +59,10 @@ static inline int32_t cuda_status(dl_ctx* ctx, cudaError_t e) {
 
 static inline int elt_bytes(const dl_ctx* ctx) { return ctx->desc.dtype == DL_F32 ? 4 : 2; }
 
+// *keep_done (if given) tells whether the launch also wrote keep = score > threshold
 static int32_t run_predictor(dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows, float* score,
-                             cudaStream_t s) {
+                             cudaStream_t s, uint8_t* keep = nullptr, float threshold = 0.f, bool* keep_done = nullptr) {
+  if (keep_done) *keep_done = false;
   if (!p || !p->w1 || !p->b1 || !p->w2 || !x || !score) return DL_ERR_INVALID_ARG;
   if (misaligned(p->w1) || misaligned(x)) return DL_ERR_ALIGNMENT;
   int impl = ctx->opt.predictor_impl;
@@ -66,7 +70,8 @@ static int32_t run_predictor(dl_ctx* ctx, const dl_predictor* p, const void* x, 
   if (impl == 2) {
     if (!predictor_tc_supported(ctx)) return DL_ERR_UNSUPPORTED;
     if (!ctx->ws.base || rows > ctx->ws.max_rows) return DL_ERR_WORKSPACE;
-    return cuda_status(ctx, launch_predictor_tc(ctx, p, x, rows, score, s));
+    if (keep_done) *keep_done = keep != nullptr;
+    return cuda_status(ctx, launch_predictor_tc(ctx, p, x, rows, score, s, keep, threshold));
   }
   return cuda_status(ctx, launch_predictor_simt(ctx, p, x, rows, score, s));
 }
@@ -144,6 +149,7 @@ int32_t dl_set_workspace(dl_ctx* ctx, void* dev_ptr, int64_t bytes, int32_t max_
     e = cudaMemsetAsync(ctx->ws.dec_ticket, 0, (size_t)kDecodeScratchSets * max_batch * ctx->desc.n_heads * 4, s);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ctx->ws.pred_ticket, 0, (size_t)(ctx->ws.pred_rows_padded / kPredRowTile + 1) * 4, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.dec_commit, 0, 4, s);
   return cuda_status(ctx, e);
 }
 
@@ -316,7 +322,8 @@ int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, 
 // caches and outputs are distinct tensors).
 static int32_t decode_layer(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
                             void* v_cache, const int32_t* cache_len, const uint8_t* keep, int32_t B,
-                            int32_t cap, float scale, void* out, bool overlap_prev, int scratch_set, void* stream) {
+                            int32_t cap, float scale, void* out, bool overlap_prev, int scratch_set, void* stream,
+                            int32_t* commit_len = nullptr) {
   if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
   if (B == 0) return DL_OK;
   if (!q_t || !k_t || !v_t || !k_cache || !v_cache || !cache_len || !out) return DL_ERR_INVALID_ARG;
@@ -327,7 +334,8 @@ static int32_t decode_layer(dl_ctx* ctx, const void* q_t, const void* k_t, const
   if (B > 2048) return DL_ERR_UNSUPPORTED;
   DeviceGuard g(ctx->device);
   return cuda_status(ctx, launch_attn_decode(ctx, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, B, cap,
-                                             scale, out, overlap_prev, scratch_set, static_cast<cudaStream_t>(stream)));
+                                             scale, out, overlap_prev, scratch_set, static_cast<cudaStream_t>(stream),
+                                             commit_len));
 }
 
 int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
@@ -344,8 +352,10 @@ int32_t dl_decode_keep(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, 
   DeviceGuard g(ctx->device);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (x_t) {
-    int32_t st = run_predictor(ctx, p_txt, x_t, B, logit_inout, s);
-    if (st != DL_OK) return st;
+    // the tensor-core predictor takes the decision where it completes the logit: no second launch
+    bool keep_done = false;
+    int32_t st = run_predictor(ctx, p_txt, x_t, B, logit_inout, s, keep_out, threshold, &keep_done);
+    if (st != DL_OK || keep_done) return st;
   }
   return cuda_status(ctx, launch_decode_keep(logit_inout, B, threshold, keep_out, ctx->ws.status, s));
 }
@@ -376,10 +386,12 @@ int32_t dl_commit_len(dl_ctx* ctx, const uint8_t* keep, int32_t B, int32_t cap, 
   return cuda_status(ctx, launch_commit_len(keep, B, cap, cache_len, static_cast<cudaStream_t>(stream)));
 }
 
-int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
-                                     void* const* k_caches, void* const* v_caches, const int32_t* cache_len,
-                                     const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                                     void* stream) {
+// The layer stack of a decode step.  commit_len (null or the lengths, writable): the last layer's launch also closes
+// the step, cache_len[b] += keep[b], once every launch of the stack has read the lengths for the last time.
+static int32_t decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
+                             void* const* k_caches, void* const* v_caches, const int32_t* cache_len,
+                             const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out, void* stream,
+                             int32_t* commit_len) {
   if (!ctx || L < 0 || B < 0) return DL_ERR_INVALID_ARG;
   if (B == 0 || L == 0) return DL_OK;
   if (!k_caches || !v_caches || !q_t || !k_t || !v_t || !out) return DL_ERR_INVALID_ARG;
@@ -393,11 +405,18 @@ int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, co
     // consecutive layers touch different caches and outputs, so layer l may start while layer l-1 drains
     const bool overlap = l > 0 && k_caches[l] != k_caches[l - 1] && v_caches[l] != v_caches[l - 1];
     int32_t st = decode_layer(ctx, ql, kl, vl, k_caches[l], v_caches[l], cache_len, keep, B, cap, scale, ol, overlap,
-                              l % kDecodeScratchSets, stream);
+                              l % kDecodeScratchSets, stream, l == L - 1 ? commit_len : nullptr);
     if (st != DL_OK) { ctx->opt.in_layer_stack = 0; return st; }
   }
   ctx->opt.in_layer_stack = 0;
   return DL_OK;
+}
+
+int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
+                                     void* const* k_caches, void* const* v_caches, const int32_t* cache_len,
+                                     const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
+                                     void* stream) {
+  return decode_layers(ctx, L, q_t, k_t, v_t, k_caches, v_caches, cache_len, keep, B, cap, scale, out, stream, nullptr);
 }
 
 int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
@@ -409,10 +428,11 @@ int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, 
   if (L > 0 && (!k_caches || !v_caches || !q_t || !k_t || !v_t || !out)) return DL_ERR_INVALID_ARG;
   int32_t st = dl_decode_keep(ctx, p_txt, x_t, B, threshold, logit_inout, keep_out, stream);
   if (st != DL_OK) return st;
-  st = dl_sparse_attn_decode_layers(ctx, L, q_t, k_t, v_t, k_caches, v_caches, cache_len, keep_out, B, cap, scale, out,
-                                    stream);
-  if (st != DL_OK) return st;
-  return dl_commit_len(ctx, keep_out, B, cap, cache_len, stream);
+  // the step is closed by its last attention launch; without layers the commit is a launch of its own
+  if (L == 0) return dl_commit_len(ctx, keep_out, B, cap, cache_len, stream);
+  if (!cache_len) return DL_ERR_INVALID_ARG;
+  return decode_layers(ctx, L, q_t, k_t, v_t, k_caches, v_caches, cache_len, keep_out, B, cap, scale, out, stream,
+                       cache_len);
 }
 
 int32_t dl_decode_step_host(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_host, int32_t B,

@@ -85,6 +85,8 @@ struct DecodeArgs {
   void* out;
   float* partial; int32_t* ticket; DeviceStatus* status;
   int32_t B, H, cap, chunk, per_bh, slots, n_stages;
+  int32_t* commit_len;    // not null: this launch is the last of a step; it closes the step with cache_len[b] += keep[b]
+  int32_t* commit_count;  // CTAs of this launch that have finished (zero between launches)
   int32_t overlap;        // launched with programmatic stream serialisation (see launch_mma)
   int32_t one_slot;       // host only: one CTA per SM (see launch_attn_decode)
   float scale_log2;
@@ -103,6 +105,26 @@ static inline int max_chunks(const DecodeArgs& a) {
 }
 
 struct DecodeItem { int b, h, c, nch, n_b, r0, rows, nst; };
+
+// Closes a decode step inside its last attention launch (Eq. 6: the length grows by the decision, once, after
+// every layer has appended): the CTA that finishes last - every other CTA of this launch has read the lengths
+// for the last time, and every earlier layer's launch is complete - advances them.  Called by all threads.
+__device__ __forceinline__ void decode_commit(const DecodeArgs& a) {
+  if (a.commit_len == nullptr) return;
+  __shared__ int sh_last;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    sh_last = atomicAdd(a.commit_count, 1) == (int)gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!sh_last) return;
+  for (int b = threadIdx.x; b < a.B; b += blockDim.x) {
+    const int n = a.commit_len[b];
+    if (a.keep[b] != 0 && n < a.cap) a.commit_len[b] = n + 1;
+  }
+  if (threadIdx.x == 0) *a.commit_count = 0;
+}
 
 template <typename T, int D, int RS, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32, 1)
@@ -377,6 +399,7 @@ attn_decode_kernel(const DecodeArgs a) {
         for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&bars[j % NS]), (j / NS) & 1); ++i) __nanosleep(40);
     }
   }
+  decode_commit(a);
 }
 
 template <typename T, int D, int RS, int WARPS>
@@ -735,6 +758,7 @@ attn_decode_mma_kernel(const __grid_constant__ TmapPair maps, const DecodeArgs a
         for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&bars[j % NS]), (j / NS) & 1); ++i) __nanosleep(40);
     }
   }
+  decode_commit(a);
 }
 
 // Tensor maps over a cache viewed as [B*H*cap rows][128 dims]: box 64 dims x 16 rows, 128-byte swizzle.
@@ -838,11 +862,13 @@ static int scratch_slots(const DecodeArgs& a) { return max_chunks(a) + 1; }
 cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t,
                                void* k_cache, void* v_cache, const int32_t* cache_len,
                                const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                               bool overlap_prev, int scratch_set, cudaStream_t s) {
+                               bool overlap_prev, int scratch_set, cudaStream_t s, int32_t* commit_len) {
   if (B == 0) return cudaSuccess;
   if (B > kMaxDecodeBatch) return cudaErrorInvalidValue;
   const dl_model_desc& d = ctx->desc;
   DecodeArgs a;
+  a.commit_len = keep ? commit_len : nullptr;
+  a.commit_count = ctx->ws.dec_commit;
   a.q = q; a.k_t = k_t; a.v_t = v_t; a.k_cache = k_cache; a.v_cache = v_cache;
   a.cache_len = cache_len; a.keep = keep; a.out = out;
   a.status = ctx->ws.status;
@@ -929,6 +955,7 @@ extern "C" int32_t dl_sparse_attn_decode_static(dl_ctx* ctx, const void* q_t, co
   const dl_model_desc& d = ctx->desc;
   DecodeArgs a;
   a.B = B; a.H = d.n_heads; a.cap = cap;
+  a.commit_len = nullptr; a.commit_count = nullptr;
   pick_split(ctx, a);
   a.overlap = 0;
   a.one_slot = 0;

@@ -8,42 +8,62 @@
 // that run side by side share one X tile through L2; a row tile's partial sums (one per unit
 // tile) are added in tile order by the CTA that finishes last (a ticket, not a wait), so the
 // logits are reproducible bit for bit.
-//   warp 0 : TMA producer (X and W1 tiles, 128-byte swizzle, 4-stage ring)
+//   warp 0 : TMA producer (X and W1 tiles, 128-byte swizzle; a ring of 4 stages for prefill shapes, up to 32
+//            short stages for the few rows of a decode step)
 //   warp 1 : tensor-memory allocation and the single MMA-issuing thread
 //   warps 2-5 : epilogue, one TMEM lane quadrant each; two accumulators ping-pong so the epilogue
 //               of one item overlaps the main loop of the next
 // Every wait is bounded (pipeline.cuh); an abort leaves DL_ERR_TIMEOUT in the status word.
+#include <algorithm>
+
 #include "common.cuh"
 #include "tc05.cuh"
 
 namespace dl {
 
-constexpr int kPtStages = 4;
+constexpr int kPtMaxStages = 32;
 constexpr int kPtBM = 128;
 constexpr int kPtBK = 64;
 constexpr int kPtMaxBN = 256;
 constexpr int kPtThreads = 192;
 constexpr int kPtATile = kPtBM * kPtBK * 2;          // 16 KB
 constexpr int kPtBTile = kPtMaxBN * kPtBK * 2;       // 32 KB
-constexpr int kPtStageBytes = kPtATile + kPtBTile;
-constexpr size_t kPtSmem = (size_t)kPtStages * kPtStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int kPtStageBytes = kPtATile + kPtBTile;   // a stage of the widest form (128 rows, 256 units)
+constexpr int kPtBarBytes = (2 * kPtMaxStages + 4) * 8;
+// the ring, then room for the MMA's 128-row read past a short last stage, the barriers, the alignment slack
+constexpr size_t kPtSmem = (size_t)4 * kPtStageBytes + kPtATile + kPtBarBytes + 1024;
 
 struct PredTcArgs {
   const float* b1; const float* w2; float b2;
   float* score; float* partial; int32_t* ticket; DeviceStatus* status;
   int32_t rows, rows_padded, k_blocks, bn, n_tiles, m_tiles, tmem_cols;
+  int32_t stages, stage_bytes, a_bytes;   // ring depth; bytes per stage; bytes of its X part
+  int32_t kbs, a_tile, b_tile;            // 64-column blocks of the hidden dimension per stage; bytes of one X / one W1 block
+  uint8_t* keep; float threshold;         // decode decision fused into the final sum (keep may be null)
 };
+
+// score and, if asked for, the decision keep = score > threshold (strictly; a NaN score drops and is reported)
+__device__ __forceinline__ void pt_emit(const PredTcArgs& a, int row, float score) {
+  a.score[row] = score;
+  if (a.keep != nullptr) {
+    if (score != score) report_status(a.status, DL_WARN_NAN, row);
+    a.keep[row] = score > a.threshold ? 1 : 0;
+  }
+}
 
 __global__ void __launch_bounds__(kPtThreads, 1)
 predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                     const PredTcArgs a) {
   extern __shared__ char smem_raw[];
   char* smem = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kPtStages * kPtStageBytes);
+  const int NS = a.stages;
+  // The MMA always reads 128 rows of X from a stage; with a short row box (few rows: the decode shape) the rows
+  // past the box are whatever follows in shared memory, and their results are never stored.
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)NS * a.stage_bytes + kPtATile);
   // bars: full[S] | empty[S] | acc_full[2] | acc_empty[2]
   uint64_t* full = bars;
-  uint64_t* empty = bars + kPtStages;
-  uint64_t* acc_full = bars + 2 * kPtStages;
+  uint64_t* empty = bars + NS;
+  uint64_t* acc_full = bars + 2 * NS;
   uint64_t* acc_empty = acc_full + 2;
   __shared__ uint32_t sh_tmem;
   __shared__ int sh_abort;
@@ -55,7 +75,7 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 
   if (tid == 0) {
     sh_abort = 0;
-    for (int s = 0; s < kPtStages; ++s) { mbar_init(smem_u32(&full[s]), 1); mbar_init(smem_u32(&empty[s]), 1); }
+    for (int s = 0; s < NS; ++s) { mbar_init(smem_u32(&full[s]), 1); mbar_init(smem_u32(&empty[s]), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), 4); }
     fence_mbar_init();
   }
@@ -67,30 +87,32 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sh_tmem;
-  const uint32_t b_bytes = (uint32_t)a.bn * kPtBK * 2;
+  const uint32_t b_bytes = (uint32_t)(a.kbs * a.b_tile);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&map_x);
       tma_prefetch_desc(&map_w);
-      int it = 0;
+      int it = 0, s = 0, ph = 0;                 // stage and phase of fill `it`, kept by counting (NS is a run-time value)
       for (int item = blockIdx.x; item < items && !*abort_flag; item += gridDim.x) {
         const int mt = item / a.n_tiles, nt = item - mt * a.n_tiles;
-        for (int kb = 0; kb < a.k_blocks; ++kb, ++it) {
-          const int s = it % kPtStages;
-          if (!mbar_wait(smem_u32(&empty[s]), ((it / kPtStages) & 1) ^ 1, abort_flag)) break;
+        for (int kb = 0; kb < a.k_blocks; kb += a.kbs, ++it) {
+          if (!mbar_wait(smem_u32(&empty[s]), ph ^ 1, abort_flag)) break;
           const uint32_t fb = smem_u32(&full[s]);
-          mbar_expect_tx(fb, kPtATile + b_bytes);
-          char* st = smem + (size_t)s * kPtStageBytes;
-          tma_load_2d(smem_u32(st), &map_x, kb * kPtBK, mt * kPtBM, fb);
-          tma_load_2d(smem_u32(st + kPtATile), &map_w, kb * kPtBK, nt * a.bn, fb);
+          mbar_expect_tx(fb, (uint32_t)a.a_bytes + b_bytes);
+          char* st = smem + (size_t)s * a.stage_bytes;
+          // one copy each for the stage's kbs blocks of X and of W1: the maps see the hidden dimension as
+          // (64 columns, row, block), so the blocks land one after the other as K-major tiles
+          tma_load_3d(smem_u32(st), &map_x, 0, mt * kPtBM, kb, fb);
+          tma_load_3d(smem_u32(st + a.a_bytes), &map_w, 0, nt * a.bn, kb, fb);
+          if (++s == NS) { s = 0; ph ^= 1; }
         }
       }
       if (*abort_flag) {
         report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
-        for (int j = max(0, it - kPtStages); j < it; ++j)
-          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&full[j % kPtStages]), (j / kPtStages) & 1); ++i)
+        for (int j = max(0, it - NS); j < it; ++j)
+          for (int i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&full[j % NS]), (j / NS) & 1); ++i)
             __nanosleep(40);
       }
     }
@@ -99,24 +121,26 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16(kPtBM, (uint32_t)a.bn);
       const uint64_t desc_a0 = smem_desc_sw128(smem_u32(smem));
-      const uint64_t desc_b0 = smem_desc_sw128(smem_u32(smem) + kPtATile);
-      int it = 0, j = 0;
+      const uint64_t desc_b0 = smem_desc_sw128(smem_u32(smem) + (uint32_t)a.a_bytes);
+      int s = 0, ph = 0, j = 0;
       for (int item = blockIdx.x; item < items; item += gridDim.x, ++j) {
         const int buf = j & 1;
         mbar_wait(smem_u32(&acc_empty[buf]), ((j >> 1) & 1) ^ 1, abort_flag);
         tc_fence_after();
         const uint32_t d_tmem = tmem + (uint32_t)(buf * a.bn);
-        for (int kb = 0; kb < a.k_blocks; ++kb, ++it) {
-          const int s = it % kPtStages;
-          mbar_wait(smem_u32(&full[s]), (it / kPtStages) & 1, abort_flag);
+        for (int kb = 0; kb < a.k_blocks; kb += a.kbs) {
+          mbar_wait(smem_u32(&full[s]), ph, abort_flag);
           tc_fence_after();
-          // descriptors differ from the stage-0, k-0 ones only in the start-address field (16-byte units)
-          const uint64_t da = desc_a0 + (uint64_t)((s * kPtStageBytes) >> 4);
-          const uint64_t db = desc_b0 + (uint64_t)((s * kPtStageBytes) >> 4);
+          // descriptors differ from the stage-0, block-0, k-0 ones only in the start-address field (16-byte units)
+          uint64_t da = desc_a0 + (uint64_t)((s * a.stage_bytes) >> 4);
+          uint64_t db = desc_b0 + (uint64_t)((s * a.stage_bytes) >> 4);
+          for (int kk = 0; kk < a.kbs; ++kk, da += a.a_tile >> 4, db += a.b_tile >> 4) {
 #pragma unroll
-          for (int k = 0; k < kPtBK / 16; ++k)
-            mma_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+            for (int k = 0; k < kPtBK / 16; ++k)
+              mma_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | kk | k) != 0);
+          }
           mma_commit(smem_u32(&empty[s]));             // frees the stage when these MMAs have read it
+          if (++s == NS) { s = 0; ph ^= 1; }
         }
         mma_commit(smem_u32(&acc_full[buf]));          // accumulator complete
       }
@@ -148,7 +172,7 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
       if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
       const int row = mt * kPtBM + quad * 32 + lane;
       if (a.n_tiles == 1) {
-        if (row < a.rows) a.score[row] = sum + a.b2;
+        if (row < a.rows) pt_emit(a, row, sum + a.b2);
         continue;
       }
       a.partial[(size_t)nt * a.rows_padded + row] = sum;
@@ -161,7 +185,7 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         const int r2 = mt * kPtBM + et;
         float tot = 0.f;
         for (int t = 0; t < a.n_tiles; ++t) tot += __ldcg(a.partial + (size_t)t * a.rows_padded + r2);
-        if (r2 < a.rows) a.score[r2] = tot + a.b2;
+        if (r2 < a.rows) pt_emit(a, r2, tot + a.b2);
         if (et == 0) a.ticket[mt] = 0;
       }
     }
@@ -185,7 +209,7 @@ bool predictor_tc_supported(const dl_ctx* ctx) {
 }
 
 cudaError_t launch_predictor_tc(dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows, float* score,
-                                cudaStream_t s) {
+                                cudaStream_t s, uint8_t* keep, float threshold) {
   if (rows == 0) return cudaSuccess;
   const dl_model_desc& d = ctx->desc;
   const int m_tiles = (rows + kPtBM - 1) / kPtBM;
@@ -204,22 +228,42 @@ cudaError_t launch_predictor_tc(dl_ctx* ctx, const dl_predictor* p, const void* 
   a.partial = ctx->ws.pred_partial; a.ticket = ctx->ws.pred_ticket; a.status = ctx->ws.status;
   a.rows = rows; a.rows_padded = ctx->ws.pred_rows_padded; a.k_blocks = d.hidden / kPtBK; a.bn = bn;
   a.n_tiles = d.pred_hidden / bn; a.m_tiles = m_tiles;
+  a.keep = keep; a.threshold = threshold;
+  // Few rows (the decode shape, one row per sequence) make this a latency problem: a CTA walks all of the hidden
+  // dimension for its 32 units, one dependent DRAM round trip per ring refill.  A row box of 32 or 64 rows
+  // instead of 128 shrinks a stage from 20 KB to 8 KB, and the ring takes as many stages as fit (up to 32), so
+  // that a third of the walk is in flight at once.
+  const int row_box = m_tiles > 1 ? kPtBM : (rows <= 32 ? 32 : (rows <= 64 ? 64 : kPtBM));
+  // ... and a copy of a 32 x 64 box costs the producer as much as one of 128 x 64, so a stage of the short form takes
+  // four 64-column blocks of the hidden dimension per copy.
+  a.kbs = (row_box < kPtBM && a.k_blocks % 4 == 0) ? 4 : 1;
+  a.a_tile = row_box * kPtBK * 2;
+  a.b_tile = bn * kPtBK * 2;
+  a.a_bytes = a.kbs * a.a_tile;
+  a.stage_bytes = a.a_bytes + a.kbs * a.b_tile;
+  a.stages = std::max(2, std::min({kPtMaxStages, (4 * kPtStageBytes) / a.stage_bytes, a.k_blocks / a.kbs}));
   int cols = 32;
   while (cols < 2 * bn) cols <<= 1;
   a.tmem_cols = cols;
   if (m_tiles * kPtBM > a.rows_padded) return cudaErrorInvalidValue;
 
   CUtensorMap mx, mw;
-  const uint64_t dx[2] = {(uint64_t)d.hidden, (uint64_t)rows};
-  const uint64_t dw[2] = {(uint64_t)d.hidden, (uint64_t)d.pred_hidden};
-  const uint64_t st[1] = {(uint64_t)d.hidden * 2};
-  const uint32_t bx[2] = {kPtBK, kPtBM};
-  const uint32_t bw[2] = {kPtBK, (uint32_t)bn};
-  if (!encode_bf16_map(ctx->tmap_encode, &mx, x, 2, dx, st, bx) ||
-      !encode_bf16_map(ctx->tmap_encode, &mw, p->w1, 2, dw, st, bw))
+  // X [rows][hidden] and W1 [units][hidden] seen as (64 columns, row, 64-column block): a box of kbs blocks lands
+  // as kbs K-major tiles one after the other
+  const uint64_t dx[3] = {(uint64_t)kPtBK, (uint64_t)rows, (uint64_t)a.k_blocks};
+  const uint64_t dw[3] = {(uint64_t)kPtBK, (uint64_t)d.pred_hidden, (uint64_t)a.k_blocks};
+  const uint64_t st[2] = {(uint64_t)d.hidden * 2, (uint64_t)kPtBK * 2};
+  const uint32_t bx[3] = {kPtBK, (uint32_t)row_box, (uint32_t)a.kbs};
+  const uint32_t bw[3] = {kPtBK, (uint32_t)bn, (uint32_t)a.kbs};
+  if (!encode_bf16_map(ctx->tmap_encode, &mx, x, 3, dx, st, bx) ||
+      !encode_bf16_map(ctx->tmap_encode, &mw, p->w1, 3, dw, st, bw))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(predictor_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPtSmem);
-  if (e != cudaSuccess) return e;
+  static int attr_set[64];
+  if (!attr_set[ctx->device & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(predictor_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPtSmem);
+    if (e != cudaSuccess) return e;
+    attr_set[ctx->device & 63] = 1;
+  }
   const int grid = min(ctx->sm_count, m_tiles * a.n_tiles);
   predictor_tc_kernel<<<grid, kPtThreads, kPtSmem, s>>>(mx, mw, a);
   return cudaGetLastError();

@@ -73,6 +73,8 @@ class BatchRunner:
         self.keep_t = torch.empty(B, dtype=torch.uint8, device=dev)
         self.dec_out = torch.empty(L, B, H, D, dtype=tdt, device=dev)
         self.launches = 0
+        # launches of dl_decode_step: predictor (+ keep test unless fused: bf16) + L attention (+ nothing: commit folded)
+        self.step_launches = (1 if cfg.dtype == "bf16" else 2) + cfg.n_layers
         self.use_graphs = use_graphs
         self._graphs: dict = {}            # decode step captured once per input-pool slot
         self.host_fed = host_fed
@@ -116,10 +118,10 @@ class BatchRunner:
                 self.cache_len.copy_(saved)                    # undo the warm run's commit (its appended row
                 self._graphs[i] = g                            # lies past the restored length)
             g.replay()
-            self.launches += 3 + c.n_layers
+            self.launches += self.step_launches
             return
         self._decode_step_eager(i)
-        self.launches += 3 + c.n_layers
+        self.launches += self.step_launches
 
     def _decode_step_eager(self, i: int):
         c = self.cfg
@@ -140,7 +142,7 @@ class BatchRunner:
         e1.record()
         events.append((e0, e1, lens, c.n_layers))
         ctx.commit_len(self.keep_t, self.cache_len, self.cap)
-        self.launches += 3 + c.n_layers
+        self.launches += self.step_launches + 1
 
     def run_batch(self, sample_every: int = 0, events: list | None = None):
         """One whole batch.  With `sample_every`, every sample_every-th decode step is issued call by
