@@ -22,6 +22,7 @@ What each function follows
                         the same quantity evaluated on the compacted cache (Eq. 1 on the
                         reduced set; Eq. 6: Attention(Q, S^K u K, S^V u V))
   prefill_flops         Eq. 13
+  (predictor_paper.py holds the paper's own predictor architectures: App. "Details of Predictor Architecture")
 
 Pins (tests/test_oracle_*.py): closed forms of GELU and of softmax attention,
 brute-force sorting, the dense-causal textbook form, masked-vs-compact equality and

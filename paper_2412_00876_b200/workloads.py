@@ -162,6 +162,39 @@ def make_predictor(cfg: Config, which: str, b2: float | None = None) -> Predicto
     return Predictor(w1, b1, w2, float(np.float32(b2)))
 
 
+S_PAPER_PRED = 40       # streams 40.. : weights of the paper's own predictors
+
+
+def make_predictor_paper(cfg: Config, which: str, width: int = 512, n_blocks: int = 2, mlp_hidden: int = 2048,
+                         out_bias: float = 0.0) -> dict:
+    """Seeded weights of the paper's predictor architecture (linear d -> 512; two transformer blocks for the
+    image predictor; head 512 -> 256 -> 128 -> 2).  Matrices ~ N(0, 1/fan_in), rounded to the storage type;
+    biases and LayerNorm parameters in float32 (scales near 1).  `which` in {"img", "txt"}; the text predictor
+    has no blocks.  out_bias is added to the second output's bias (moves the keep rate)."""
+    base = S_PAPER_PRED + (0 if which == "img" else 20)
+    n = [0]
+
+    def mat(o, i):
+        n[0] += 1
+        return host_normal(cfg, base, (o, i), std=1.0 / np.sqrt(i), sub=n[0])
+
+    def vec(o, std=0.1, mean=0.0):
+        n[0] += 1
+        return (host_normal(cfg, base, (o,), std=std, dtype="f32", sub=n[0]) + np.float32(mean)).astype(np.float32)
+
+    p = {"w_in": mat(width, cfg.hidden), "b_in": vec(width), "blocks": []}
+    for _ in range(n_blocks if which == "img" else 0):
+        p["blocks"].append({"ln1_g": vec(width, 0.1, 1.0), "ln1_b": vec(width), "w_qkv": mat(3 * width, width),
+                            "b_qkv": vec(3 * width), "w_o": mat(width, width), "b_o": vec(width),
+                            "ln2_g": vec(width, 0.1, 1.0), "ln2_b": vec(width), "w_fc1": mat(mlp_hidden, width),
+                            "b_fc1": vec(mlp_hidden), "w_fc2": mat(width, mlp_hidden), "b_fc2": vec(width)})
+    b3 = vec(2)
+    b3[1] += np.float32(out_bias)
+    p["head"] = {"w1": mat(256, width), "b1": vec(256), "w2": mat(128, 256), "b2": vec(128),
+                 "w3": host_normal(cfg, base, (2, 128), std=1.0 / np.sqrt(128), dtype="f32", sub=99), "b3": b3}
+    return p
+
+
 def ragged_text_lengths(cfg: Config) -> np.ndarray:
     """Per-sequence prompt lengths, uniform in [N_T/2, N_T] (correctness variant)."""
     lo = max(1, cfg.n_text // 2)
