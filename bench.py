@@ -40,7 +40,7 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-record", action="store_true")
     ap.add_argument("--sample-every", type=int, default=64, help="decode steps between timed attention launches")
-    ap.add_argument("--micro", default="", choices=["", "decode", "keep", "predictor", "select", "compact", "compact_layers", "prefill", "nocache"],
+    ap.add_argument("--micro", default="", choices=["", "decode", "keep", "select2", "keep2", "predictor", "select", "compact", "compact_layers", "prefill", "nocache"],
                     help="time one stage alone on the config's shapes (small memory; used for ncu captures)")
     ap.add_argument("--micro-layers", type=int, default=2, help="layers of cache / source held in --micro mode")
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
@@ -102,6 +102,40 @@ def micro(args, emit=True):
         keepf = torch.empty(B, dtype=torch.uint8, device=dev)
         work, unit = (cfg.hidden * cfg.pred_hidden + B * cfg.hidden) * cfg.elt_bytes, "GB/s"     # weights + rows read
         calls = [lambda l=l: ctx.decode_keep(pd, xs[l], logit, keepf) for l in range(NL)]
+    elif args.micro in ("select2", "keep2"):
+        # the paper's own predictor architecture: image predictor + top-k by D[:,2] (select2), text predictor + argmax (keep2)
+        def dev_params(pr):
+            def conv(k, v):
+                if isinstance(v, dict):
+                    return {kk: conv(kk, vv) for kk, vv in v.items()}
+                if isinstance(v, list):
+                    return [conv(k, x) for x in v]
+                if v.ndim == 2 and k != "w3":
+                    return wl.to_torch(v, "bf16", dev)
+                return torch.from_numpy(np.ascontiguousarray(v, dtype=np.float32)).to(dev)
+            return conv("", pr)
+        which = "img" if args.micro == "select2" else "txt"
+        p2 = dl.Predictor2(dev_params(wl.make_predictor_paper(cfg, which)))
+        if which == "img":
+            scratch = ctx.predictor2_scratch(rows)
+            xs = [wl.device_normal(cfg, wl.S_X_VIS, (B, cfg.n_vis, cfg.hidden), dev, sub=i) for i in range(NL)]
+            n_vis = torch.full((B,), cfg.n_vis, **i32)
+            k_arr = torch.full((B,), cfg.k_vis, **i32)
+            d_out = torch.empty(rows, 2, dtype=torch.float32, device=dev)
+            score = torch.empty(B, cfg.n_vis, dtype=torch.float32, device=dev)
+            kept = torch.empty(B, cfg.k_vis, dtype=torch.int32, device=dev)
+            keepm = torch.empty(B, cfg.n_vis, dtype=torch.uint8, device=dev)
+            per_tok = 2.0 * (cfg.hidden * 512 + 2 * (512 * 1536 + 512 * 512 + 2 * 512 * 2048) + 512 * 256 + 256 * 128 + 256)
+            work, unit = rows * per_tok + 2 * 4.0 * B * cfg.n_vis * cfg.n_vis * 512, "TFLOP/s"
+            calls = [lambda l=l: ctx.prefill_select2(p2, xs[l], n_vis, k_arr, scratch, d_out, score, kept, keepm)
+                     for l in range(NL)]
+        else:
+            scratch = ctx.predictor2_scratch(B)
+            xs = [wl.device_normal(cfg, wl.S_X_TXT, (B, cfg.hidden), dev, sub=i) for i in range(NL)]
+            d_out = torch.empty(B, 2, dtype=torch.float32, device=dev)
+            keepf = torch.empty(B, dtype=torch.uint8, device=dev)
+            work, unit = (cfg.hidden * 512 + 512 * 256 + 256 * 128) * 2 + B * cfg.hidden * 2, "GB/s"
+            calls = [lambda l=l: ctx.decode_keep2(p2, xs[l], scratch, d_out, keepf) for l in range(NL)]
     elif args.micro == "predictor":
         p = wl.make_predictor(cfg, "img")
         pd = dl.Predictor(wl.to_torch(p.w1, cfg.dtype, dev), torch.from_numpy(p.b1).to(dev),

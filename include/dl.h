@@ -272,6 +272,58 @@ int32_t dl_decode_steps_host(dl_ctx* ctx, const dl_predictor* p_txt, int32_t n_s
                              void* const* k_caches, void* const* v_caches, int32_t cap,
                              int32_t* cache_len, float scale, void* stream);
 
+/* ---- the paper's own predictors (App. "Details of Predictor Architecture") -------------------------------- */
+
+#define DL_PRED2_WIDTH 512      /* width after the input projection; 8 heads of 64; MLP hidden 2048; head 256, 128, 2 */
+
+typedef struct { const void* w; const float* b; } dl_linear;     /* w dev [out][in] bf16, in contiguous; b dev [out] f32 */
+
+/* One pre-norm transformer block over the image tokens of a sequence:
+ *   x = x + proj(MHA(LN1(x)));  x = x + fc2(GELU(fc1(LN2(x))))      LayerNorm eps 1e-6, exact-erf GELU,
+ * bidirectional scaled-dot-product attention, 8 heads of 64.  ln*_g, ln*_b dev [512] f32; qkv [1536][512] (query,
+ * key, value projections stacked, head h owning 64 consecutive outputs of each); proj [512][512]; fc1 [2048][512];
+ * fc2 [512][2048]. */
+typedef struct {
+  const float* ln1_g; const float* ln1_b; dl_linear qkv, proj;
+  const float* ln2_g; const float* ln2_b; dl_linear fc1, fc2;
+} dl_vit_block;
+
+/* A predictor in the paper's architecture: in [512][hidden]; n_blocks transformer blocks (2 for the image predictor,
+ * 0 for the output-text predictor, whose decision depends on the current token alone); head h1 [256][512],
+ * h2 [128][256] (GELU after each), w3 dev [2][128] f32, b3 dev [2] f32.  `blocks` is a HOST array. */
+typedef struct {
+  dl_linear in;
+  int32_t n_blocks;
+  const dl_vit_block* blocks;
+  dl_linear h1, h2;
+  const float* w3; const float* b3;
+} dl_predictor2;
+
+/* Bytes of scratch dl_predictor2_values needs for `rows` rows (B * n_max).  Negative on bad arguments. */
+int64_t dl_predictor2_scratch_bytes(const dl_ctx* ctx, int64_t rows);
+
+/* Decision values of Eq. 5 for every row: D = P(x) in R^{rows x 2}.
+ *   x dev [B][n_max][hidden] bf16; n_vis dev [B] or NULL (= n_max): only the first n_vis[b] rows of sequence b are
+ *   tokens (they alone attend to one another; padding rows give D = 0, score = -inf, keep = 0);
+ *   scratch dev, 256-byte aligned, at least dl_predictor2_scratch_bytes(B * n_max) bytes, caller-owned;
+ *   d_out dev [B * n_max][2] f32 or NULL; score_out dev [B * n_max] f32 or NULL: the raw second value D[:,2], the
+ *   ranking score of Eq. 11; keep_out dev [B * n_max] or NULL: the argmax of Eq. 5, 1 iff D[:,2] > D[:,1]
+ *   (strictly; a NaN drops and records DL_WARN_NAN).  bf16 models only (DL_ERR_UNSUPPORTED otherwise). */
+int32_t dl_predictor2_values(dl_ctx* ctx, const dl_predictor2* p, const void* x, const int32_t* n_vis, int32_t B, int32_t n_max,
+                      void* scratch, int64_t scratch_bytes, float* d_out, float* score_out, uint8_t* keep_out, void* stream);
+
+/* Eq. 11 with the paper's image predictor: D = P^I(x_vis), then the k[b] tokens with the largest D[:,2] per sequence
+ * (ties to the lower index), exactly as dl_prefill_select does with its one-logit predictor. */
+int32_t dl_prefill_select2(dl_ctx* ctx, const dl_predictor2* p_img, const void* x_vis, const int32_t* n_vis,
+                           const int32_t* k, int32_t B, int32_t n_vis_max, void* scratch, int64_t scratch_bytes,
+                           float* d_out, float* score_out, int32_t* kept_idx_out, int32_t k_max, uint8_t* keep_out,
+                           void* stream);
+
+/* Eq. 6's decision with the paper's output-text predictor (n_blocks must be 0): keep[b] = D[b][2] > D[b][1].
+ *   x_t dev [B][hidden]; d_out dev [B][2] or NULL; keep_out dev [B]. */
+int32_t dl_decode_keep2(dl_ctx* ctx, const dl_predictor2* p_txt, const void* x_t, int32_t B, void* scratch,
+                        int64_t scratch_bytes, float* d_out, uint8_t* keep_out, void* stream);
+
 /* ---- diagnostics ----------------------------------------------------------------------- */
 
 /* Self-test of the bounded waits (no counterpart in the paper): launches one small kernel that waits, with

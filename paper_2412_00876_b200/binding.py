@@ -28,6 +28,7 @@ EXPORTS = [
     "dl_sparse_attn_decode", "dl_decode_keep", "dl_commit_len", "dl_decode_step", "dl_decode_step_host",
     "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers", "dl_decode_nocache_select",
     "dl_decode_steps_host", "dl_compact_kv_host", "dl_selftest_wait_timeout", "dl_compact_kv_layers",
+    "dl_predictor2_scratch_bytes", "dl_predictor2_values", "dl_prefill_select2", "dl_decode_keep2",
 ]
 
 
@@ -36,8 +37,42 @@ class ModelDesc(C.Structure):
                 ("pred_hidden", C.c_int32), ("dtype", C.c_int32)]
 
 
+class LinearDesc(C.Structure):
+    _fields_ = [("w", C.c_void_p), ("b", C.c_void_p)]
+
+
+class VitBlockDesc(C.Structure):
+    _fields_ = [("ln1_g", C.c_void_p), ("ln1_b", C.c_void_p), ("qkv", LinearDesc), ("proj", LinearDesc),
+                ("ln2_g", C.c_void_p), ("ln2_b", C.c_void_p), ("fc1", LinearDesc), ("fc2", LinearDesc)]
+
+
+class Predictor2Desc(C.Structure):
+    _fields_ = [("inp", LinearDesc), ("n_blocks", C.c_int32), ("blocks", C.POINTER(VitBlockDesc)),
+                ("h1", LinearDesc), ("h2", LinearDesc), ("w3", C.c_void_p), ("b3", C.c_void_p)]
+
+
 class PredictorDesc(C.Structure):
     _fields_ = [("w1", C.c_void_p), ("b1", C.c_void_p), ("w2", C.c_void_p), ("b2", C.c_float)]
+
+
+class Predictor2:
+    """Device tensors of a predictor in the paper's architecture and the descriptor that points at them.
+    `params` is the dictionary layout of workloads.make_predictor_paper with torch CUDA tensors as values
+    (matrices bf16, vectors float32); the tensors are kept alive here."""
+
+    def __init__(self, params: dict):
+        self.params = params
+        lin = lambda w, b: LinearDesc(w.data_ptr(), b.data_ptr())
+        blocks = params["blocks"]
+        self._blocks = (VitBlockDesc * max(len(blocks), 1))()
+        for i, k in enumerate(blocks):
+            self._blocks[i] = VitBlockDesc(k["ln1_g"].data_ptr(), k["ln1_b"].data_ptr(), lin(k["w_qkv"], k["b_qkv"]),
+                                           lin(k["w_o"], k["b_o"]), k["ln2_g"].data_ptr(), k["ln2_b"].data_ptr(),
+                                           lin(k["w_fc1"], k["b_fc1"]), lin(k["w_fc2"], k["b_fc2"]))
+        h = params["head"]
+        self.desc = Predictor2Desc(lin(params["w_in"], params["b_in"]), len(blocks),
+                                   C.cast(self._blocks, C.POINTER(VitBlockDesc)), lin(h["w1"], h["b1"]),
+                                   lin(h["w2"], h["b2"]), h["w3"].data_ptr(), h["b3"].data_ptr())
 
 
 _lib = None
@@ -76,6 +111,11 @@ def lib() -> C.CDLL:
                                                   f32, vp, vp]),
             "dl_decode_keep": (i32, [vp, P, vp, i32, f32, vp, vp, vp]),
             "dl_selftest_wait_timeout": (i32, [vp, i32, vp]),
+            "dl_predictor2_scratch_bytes": (i64, [vp, i64]),
+            "dl_predictor2_values": (i32, [vp, C.POINTER(Predictor2Desc), vp, vp, i32, i32, vp, i64, vp, vp, vp, vp]),
+            "dl_prefill_select2": (i32, [vp, C.POINTER(Predictor2Desc), vp, vp, vp, i32, i32, vp, i64, vp, vp, vp, i32,
+                                         vp, vp]),
+            "dl_decode_keep2": (i32, [vp, C.POINTER(Predictor2Desc), vp, i32, vp, i64, vp, vp, vp]),
             "dl_decode_nocache_select": (i32, [vp, P, vp, vp, i32, i32, f32, vp, vp, vp]),
             "dl_commit_len": (i32, [vp, vp, i32, i32, vp, vp]),
             "dl_decode_step": (i32, [vp, P, vp, i32, f32, vp, vp, i32, vp, vp, vp, C.POINTER(vp),
@@ -270,6 +310,33 @@ class Context:
     def commit_len(self, keep, cache_len, cap, stream=None):
         self._check(lib().dl_commit_len(self._h, _ptr(keep), keep.shape[0], cap, _ptr(cache_len),
                                         _stream(stream)), "dl_commit_len")
+
+    # ---- the paper's own predictors
+    def predictor2_scratch(self, rows: int) -> torch.Tensor:
+        """Scratch tensor of the size dl_predictor2_values wants for `rows` rows."""
+        n = lib().dl_predictor2_scratch_bytes(self._h, int(rows))
+        if n < 0:
+            raise DlError(int(n), "dl_predictor2_scratch_bytes")
+        return torch.empty(max(int(n), 256), dtype=torch.uint8, device=self.device)
+
+    def predictor2_values(self, p: "Predictor2", x, n_vis, scratch, d_out=None, score_out=None, keep_out=None, stream=None):
+        B, n_max = x.shape[0], x.shape[1]
+        self._check(lib().dl_predictor2_values(self._h, C.byref(p.desc), _ptr(x), _ptr(n_vis), B, n_max, _ptr(scratch),
+                                               scratch.numel(), _ptr(d_out), _ptr(score_out), _ptr(keep_out),
+                                               _stream(stream)), "dl_predictor2_values")
+
+    def prefill_select2(self, p: "Predictor2", x_vis, n_vis, k, scratch, d_out, score_out, kept_idx_out, keep_out,
+                        stream=None):
+        B, n_max = x_vis.shape[0], x_vis.shape[1]
+        self._check(lib().dl_prefill_select2(self._h, C.byref(p.desc), _ptr(x_vis), _ptr(n_vis), _ptr(k), B, n_max,
+                                             _ptr(scratch), scratch.numel(), _ptr(d_out), _ptr(score_out),
+                                             _ptr(kept_idx_out), kept_idx_out.shape[1], _ptr(keep_out), _stream(stream)),
+                    "dl_prefill_select2")
+
+    def decode_keep2(self, p: "Predictor2", x_t, scratch, d_out, keep_out, stream=None):
+        self._check(lib().dl_decode_keep2(self._h, C.byref(p.desc), _ptr(x_t), x_t.shape[0], _ptr(scratch),
+                                          scratch.numel(), _ptr(d_out), _ptr(keep_out), _stream(stream)),
+                    "dl_decode_keep2")
 
     def selftest_wait_timeout(self, polls: int = 64, stream=None):
         self._check(lib().dl_selftest_wait_timeout(self._h, int(polls), _stream(stream)), "dl_selftest_wait_timeout")

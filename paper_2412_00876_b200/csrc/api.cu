@@ -232,6 +232,58 @@ int32_t dl_prefill_select(dl_ctx* ctx, const dl_predictor* p_img, const void* x_
   return dl_topk_from_scores(ctx, score_out, n_vis, k, B, n_vis_max, kept_idx_out, k_max, keep_out, stream);
 }
 
+int64_t dl_predictor2_scratch_bytes(const dl_ctx* ctx, int64_t rows) {
+  if (!ctx || rows < 0) return DL_ERR_INVALID_ARG;
+  return predictor_paper_scratch_bytes(rows);
+}
+
+static int32_t check_predictor2(const dl_ctx* ctx, const dl_predictor2* p) {
+  if (!p || !p->in.w || !p->in.b || !p->h1.w || !p->h1.b || !p->h2.w || !p->h2.b || !p->w3 || !p->b3) return DL_ERR_INVALID_ARG;
+  if (p->n_blocks < 0 || p->n_blocks > 16 || (p->n_blocks > 0 && !p->blocks)) return DL_ERR_INVALID_ARG;
+  for (int i = 0; i < p->n_blocks; ++i) {
+    const dl_vit_block& k = p->blocks[i];
+    if (!k.ln1_g || !k.ln1_b || !k.ln2_g || !k.ln2_b || !k.qkv.w || !k.qkv.b || !k.proj.w || !k.proj.b || !k.fc1.w ||
+        !k.fc1.b || !k.fc2.w || !k.fc2.b)
+      return DL_ERR_INVALID_ARG;
+    if (misaligned(k.qkv.w) || misaligned(k.proj.w) || misaligned(k.fc1.w) || misaligned(k.fc2.w) ||
+        misaligned(k.ln1_g) || misaligned(k.ln1_b) || misaligned(k.ln2_g) || misaligned(k.ln2_b))
+      return DL_ERR_ALIGNMENT;
+  }
+  if (misaligned(p->in.w) || misaligned(p->h1.w) || misaligned(p->h2.w) || misaligned(p->w3)) return DL_ERR_ALIGNMENT;
+  return predictor_paper_supported(ctx) ? DL_OK : DL_ERR_UNSUPPORTED;
+}
+
+int32_t dl_predictor2_values(dl_ctx* ctx, const dl_predictor2* p, const void* x, const int32_t* n_vis, int32_t B, int32_t n_max,
+                      void* scratch, int64_t scratch_bytes, float* d_out, float* score_out, uint8_t* keep_out, void* stream) {
+  if (!ctx || B < 0 || n_max < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || n_max == 0) return DL_OK;
+  if ((int64_t)B * n_max > INT32_MAX / 4) return DL_ERR_UNSUPPORTED;
+  int32_t st = check_predictor2(ctx, p);
+  if (st != DL_OK) return st;
+  if (!x || !scratch) return DL_ERR_INVALID_ARG;
+  if (misaligned(x) || (reinterpret_cast<uintptr_t>(scratch) & 255u)) return DL_ERR_ALIGNMENT;
+  if (scratch_bytes < predictor_paper_scratch_bytes((int64_t)B * n_max)) return DL_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  return cuda_status(ctx, launch_predictor_paper(ctx, p, x, n_vis, B, n_max, scratch, d_out, score_out, keep_out,
+                                                 static_cast<cudaStream_t>(stream)));
+}
+
+int32_t dl_prefill_select2(dl_ctx* ctx, const dl_predictor2* p_img, const void* x_vis, const int32_t* n_vis,
+                           const int32_t* k, int32_t B, int32_t n_vis_max, void* scratch, int64_t scratch_bytes,
+                           float* d_out, float* score_out, int32_t* kept_idx_out, int32_t k_max, uint8_t* keep_out,
+                           void* stream) {
+  if (!score_out) return DL_ERR_INVALID_ARG;
+  int32_t st = dl_predictor2_values(ctx, p_img, x_vis, n_vis, B, n_vis_max, scratch, scratch_bytes, d_out, score_out, nullptr, stream);
+  if (st != DL_OK) return st;
+  return dl_topk_from_scores(ctx, score_out, n_vis, k, B, n_vis_max, kept_idx_out, k_max, keep_out, stream);
+}
+
+int32_t dl_decode_keep2(dl_ctx* ctx, const dl_predictor2* p_txt, const void* x_t, int32_t B, void* scratch,
+                        int64_t scratch_bytes, float* d_out, uint8_t* keep_out, void* stream) {
+  if (!keep_out || (p_txt && p_txt->n_blocks != 0)) return DL_ERR_INVALID_ARG;
+  return dl_predictor2_values(ctx, p_txt, x_t, nullptr, B, 1, scratch, scratch_bytes, d_out, nullptr, keep_out, stream);
+}
+
 int32_t dl_compact_kv(dl_ctx* ctx, const void* k_src, const void* v_src, const uint8_t* keep,
                       int32_t keep_cols, const int32_t* t_src, int32_t B, int32_t t_src_max, void* k_cache, void* v_cache,
                       int32_t cap, int32_t* cache_len, int32_t commit, void* stream) {

@@ -150,4 +150,9 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
                                    float scale, void* out, cudaStream_t s);
 bool attn_prefill_tc_supported(const dl_ctx* ctx);
 
+int64_t predictor_paper_scratch_bytes(int64_t rows);
+bool predictor_paper_supported(const dl_ctx* ctx);
+cudaError_t launch_predictor_paper(dl_ctx* ctx, const dl_predictor2* p, const void* x, const int32_t* n_vis, int32_t B,
+                                   int32_t n_max, void* scratch, float* d_out, float* score, uint8_t* keep, cudaStream_t s);
+
 }  // namespace dl
