@@ -50,6 +50,9 @@ def parse():
     ap.add_argument("--compact-impl", type=int, default=0,
                     help="--micro compact: 0 library's choice, 1 register-staged copy, 2 bulk copy by token tiles, "
                          "3 bulk copy by even row ranges")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time the stages at the paper's operating points (image keep rate 20/50/80 %, output-text "
+                         "keep rate 20/50/80 %, 144 -> 57 tokens) on the workload's shape; one JSON line per point")
     return ap.parse_args()
 
 
@@ -63,7 +66,7 @@ def micro(args, emit=True):
     from paper_2412_00876_b200 import build as dl_build
     from paper_2412_00876_b200 import workloads as wl
     dl_build.build()
-    cfg = wl.CONFIGS[args.config]
+    cfg = wl.CONFIGS[args.config].scaled(**(getattr(args, "shape", None) or {}))
     dev = torch.device("cuda", 0)
     B, H, D, NL = cfg.B, cfg.n_heads, cfg.head_dim, args.micro_layers
     tdt = wl.torch_dtype(cfg.dtype)
@@ -262,6 +265,38 @@ def micro(args, emit=True):
     return rec
 
 
+def sweep(args):
+    """Tab. 5's trade-off axes and the TokenPacker-shaped input of Sec. 4.2, as timings of the stages they change:
+    the image keep rate moves the selection's k, the compaction's volume and the prefill attention's length; the
+    output-text keep rate moves the decode attention's cache length (end state, N_OT generated tokens)."""
+    import types
+    base = __import__("paper_2412_00876_b200.workloads", fromlist=["CONFIGS"]).CONFIGS[args.config]
+    hbm, tfl, src = measured_peaks()
+
+    def run(stage, layers, shape, reps=24):
+        return micro(types.SimpleNamespace(config=args.config, micro=stage, steps=reps, warmup=4, micro_layers=layers,
+                                           micro_len=0, decode_chunk=0, prefill_impl=0, compact_impl=0, shape=shape),
+                     emit=False)
+    points = [("r_I=%d%%" % r, dict(k_vis=max(1, round(base.n_vis * r / 100)))) for r in (20, 50, 80)]
+    points.append(("144->57", dict(n_vis=144, k_vis=57)))
+    for name, shape in points:
+        sel, cmp_, att = run("select", 4, shape), run("compact_layers", 8, shape), run("prefill", 4, shape)
+        cfg = base.scaled(**shape)
+        print(json.dumps({"sweep": name, "workload": base.name, "n_vis": cfg.n_vis, "k_vis": cfg.k_vis, "n0": cfg.n0,
+                          "select_us": sel["median_us"], "select_frac_of_bf16_peak": sel["rate"] / tfl,
+                          "compact_8_layers_us": cmp_["median_us"], "compact_frac_of_hbm_peak": cmp_["rate"] / hbm,
+                          "attn_us_per_layer": att["median_us"], "attn_tflops_causal": att["rate"],
+                          "attn_frac_of_bf16_peak": att["rate"] / tfl, "peaks": src}), flush=True)
+    for r in (20, 50, 80):
+        shape = dict(keep_rate=r / 100)
+        dec = run("decode", 2, shape, reps=30)
+        cfg = base.scaled(**shape)
+        print(json.dumps({"sweep": "r_OT=%d%%" % r, "workload": base.name,
+                          "cache_len_end": cfg.n0 + int(cfg.n_gen * cfg.keep_rate),
+                          "decode_attn_us_single_launch": dec["median_us"], "decode_gbs": dec["rate"],
+                          "decode_frac_of_hbm_peak": dec["rate"] / hbm, "peaks": src}), flush=True)
+
+
 def measured_peaks():
     """(HBM GB/s, bf16 TFLOP/s burst, source): the machine's measured peaks, else the stated fallback."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -446,6 +481,8 @@ def main():
         return reference_arm(args)
     if args.micro:
         return micro(args)
+    if args.sweep:
+        return sweep(args)
     import torch
     import torch.distributed as dist
     from paper_2412_00876_b200 import build as dl_build

@@ -240,6 +240,27 @@ int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, 
                        void* const* v_caches, int32_t cap, int32_t* cache_len, float scale,
                        void* out, void* stream);
 
+/* A decoder's layer stack with the decision taken after its l-th layer (Sec. 3.3.1): the first l_dense layers run
+ * before the decision exists and keep every token, the remaining L - l_dense share the decision.
+ *   k_caches, v_caches: HOST arrays of L dev pointers; entries below l_dense are [B][H][cap_dense][D] caches whose
+ *   lengths are len_dense (dev [B], +1 per step while below cap_dense), the others [B][H][cap][D] caches whose
+ *   lengths are cache_len (dev [B], += keep per step).  The workspace must cover max(cap_dense, cap).
+ *   len_dense may be NULL when l_dense == 0, cache_len when l_dense == L. */
+typedef struct {
+  int32_t L, l_dense;
+  void* const* k_caches; void* const* v_caches;
+  int32_t cap_dense, cap;
+  int32_t* len_dense; int32_t* cache_len;
+} dl_layer_stack;
+
+/* dl_decode_step over such a stack (Eq. 6 with the layer placement of Sec. 3.3.1; with l_dense = 2 and one count of
+ * image tokens this is the layer split Eq. 13's totals in Tab. 1 are made of): the decision, then one attention
+ * launch per layer, dense layers first; the last dense launch advances len_dense, the last launch cache_len.
+ *   q_t, k_t, v_t, out dev [L][B][H][D]. */
+int32_t dl_decode_step_stack(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
+                             float* logit_inout, uint8_t* keep_out, const dl_layer_stack* stack, const void* q_t,
+                             const void* k_t, const void* v_t, float scale, void* out, void* stream);
+
 /* The same step fed from HOST buffers (pinned for full copy speed): copies x_t, q_t, k_t, v_t
  * into the caller's device staging buffers, runs dl_decode_step, copies `out` and `keep` back to
  * the host, all on `stream`; returns after the stream has been synchronised.

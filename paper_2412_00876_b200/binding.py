@@ -29,6 +29,7 @@ EXPORTS = [
     "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers", "dl_decode_nocache_select",
     "dl_decode_steps_host", "dl_compact_kv_host", "dl_selftest_wait_timeout", "dl_compact_kv_layers",
     "dl_predictor2_scratch_bytes", "dl_predictor2_values", "dl_prefill_select2", "dl_decode_keep2",
+    "dl_decode_step_stack",
 ]
 
 
@@ -44,6 +45,12 @@ class LinearDesc(C.Structure):
 class VitBlockDesc(C.Structure):
     _fields_ = [("ln1_g", C.c_void_p), ("ln1_b", C.c_void_p), ("qkv", LinearDesc), ("proj", LinearDesc),
                 ("ln2_g", C.c_void_p), ("ln2_b", C.c_void_p), ("fc1", LinearDesc), ("fc2", LinearDesc)]
+
+
+class LayerStackDesc(C.Structure):
+    _fields_ = [("L", C.c_int32), ("l_dense", C.c_int32), ("k_caches", C.POINTER(C.c_void_p)),
+                ("v_caches", C.POINTER(C.c_void_p)), ("cap_dense", C.c_int32), ("cap", C.c_int32),
+                ("len_dense", C.c_void_p), ("cache_len", C.c_void_p)]
 
 
 class Predictor2Desc(C.Structure):
@@ -120,6 +127,8 @@ def lib() -> C.CDLL:
             "dl_commit_len": (i32, [vp, vp, i32, i32, vp, vp]),
             "dl_decode_step": (i32, [vp, P, vp, i32, f32, vp, vp, i32, vp, vp, vp, C.POINTER(vp),
                                      C.POINTER(vp), i32, vp, f32, vp, vp]),
+            "dl_decode_step_stack": (i32, [vp, P, vp, i32, f32, vp, vp, C.POINTER(LayerStackDesc), vp, vp, vp, f32,
+                                           vp, vp]),
             "dl_decode_step_host": (i32, [vp, P, vp, i32, f32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                           vp, vp, C.POINTER(vp), C.POINTER(vp), i32, vp, f32, vp]),
             "dl_decode_steps_host": (i32, [vp, P, i32, i32, f32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
@@ -354,6 +363,20 @@ class Context:
                                          _ptr(keep_out), L, _ptr(q_t), _ptr(k_t), _ptr(v_t), k_ptrs, v_ptrs, cap,
                                          _ptr(cache_len), float(scale), _ptr(out), _stream(stream)),
                     "dl_decode_step")
+
+    def decode_step_stack(self, p: Predictor | None, x_t, logit_inout, keep_out, k_caches, v_caches, l_dense,
+                          cap_dense, cap, len_dense, cache_len, q_t, k_t, v_t, scale, out, threshold=0.0,
+                          stream=None):
+        """One decode step over a stack whose first l_dense layers keep every token (k_caches / v_caches: lists of
+        the L layers' cache tensors)."""
+        B, L = logit_inout.shape[0], len(k_caches)
+        kp = (C.c_void_p * max(L, 1))(*[t.data_ptr() for t in k_caches])
+        vp_ = (C.c_void_p * max(L, 1))(*[t.data_ptr() for t in v_caches])
+        st = LayerStackDesc(L, l_dense, kp, vp_, cap_dense, cap, _ptr(len_dense), _ptr(cache_len))
+        pd = C.byref(p.desc) if p is not None else None
+        self._check(lib().dl_decode_step_stack(self._h, pd, _ptr(x_t), B, float(threshold), _ptr(logit_inout),
+                                               _ptr(keep_out), C.byref(st), _ptr(q_t), _ptr(k_t), _ptr(v_t),
+                                               float(scale), _ptr(out), _stream(stream)), "dl_decode_step_stack")
 
     def decode_steps_host(self, p: Predictor, x_hosts, q_hosts, k_hosts, v_hosts, out_hosts, keep_hosts, stage_x,
                           stage_q, stage_k, stage_v, stage_out, logit_dev, keep_dev, k_ptrs, v_ptrs, L, cap,

@@ -22,7 +22,8 @@ int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_
   const int32_t rows_pad = (max_rows + kPredRowTile - 1) / kPredRowTile * kPredRowTile;
   const int64_t o_ppart = take((int64_t)kPredMaxSplit * rows_pad * 4);
   const int64_t o_ptick = take((int64_t)(rows_pad / kPredRowTile + 1) * 4);
-  const int64_t o_commit = take(4);
+  const int64_t o_commit = take(2 * 4);
+  const int64_t o_ones = take(max_batch);
   if (ws) {
     char* b = ws->base;
     ws->status = reinterpret_cast<DeviceStatus*>(b + o_status);
@@ -34,6 +35,7 @@ int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_
     ws->pred_partial = reinterpret_cast<float*>(b + o_ppart);
     ws->pred_ticket = reinterpret_cast<int32_t*>(b + o_ptick);
     ws->dec_commit = reinterpret_cast<int32_t*>(b + o_commit);
+    ws->ones = reinterpret_cast<uint8_t*>(b + o_ones);
     ws->pred_rows_padded = rows_pad;
     ws->max_batch = max_batch; ws->max_rows = max_rows; ws->cap = cap;
   }
@@ -149,7 +151,8 @@ int32_t dl_set_workspace(dl_ctx* ctx, void* dev_ptr, int64_t bytes, int32_t max_
     e = cudaMemsetAsync(ctx->ws.dec_ticket, 0, (size_t)kDecodeScratchSets * max_batch * ctx->desc.n_heads * 4, s);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ctx->ws.pred_ticket, 0, (size_t)(ctx->ws.pred_rows_padded / kPredRowTile + 1) * 4, s);
-  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.dec_commit, 0, 4, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.dec_commit, 0, 2 * 4, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.ones, 1, (size_t)max_batch, s);
   return cuda_status(ctx, e);
 }
 
@@ -375,7 +378,7 @@ int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, 
 static int32_t decode_layer(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
                             void* v_cache, const int32_t* cache_len, const uint8_t* keep, int32_t B,
                             int32_t cap, float scale, void* out, bool overlap_prev, int scratch_set, void* stream,
-                            int32_t* commit_len = nullptr) {
+                            int32_t* commit_len = nullptr, int commit_slot = 0) {
   if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
   if (B == 0) return DL_OK;
   if (!q_t || !k_t || !v_t || !k_cache || !v_cache || !cache_len || !out) return DL_ERR_INVALID_ARG;
@@ -387,7 +390,7 @@ static int32_t decode_layer(dl_ctx* ctx, const void* q_t, const void* k_t, const
   DeviceGuard g(ctx->device);
   return cuda_status(ctx, launch_attn_decode(ctx, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, B, cap,
                                              scale, out, overlap_prev, scratch_set, static_cast<cudaStream_t>(stream),
-                                             commit_len));
+                                             commit_len, commit_slot));
 }
 
 int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
@@ -438,18 +441,16 @@ int32_t dl_commit_len(dl_ctx* ctx, const uint8_t* keep, int32_t B, int32_t cap, 
   return cuda_status(ctx, launch_commit_len(keep, B, cap, cache_len, static_cast<cudaStream_t>(stream)));
 }
 
-// The layer stack of a decode step.  commit_len (null or the lengths, writable): the last layer's launch also closes
-// the step, cache_len[b] += keep[b], once every launch of the stack has read the lengths for the last time.
-static int32_t decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
-                             void* const* k_caches, void* const* v_caches, const int32_t* cache_len,
-                             const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out, void* stream,
-                             int32_t* commit_len) {
-  if (!ctx || L < 0 || B < 0) return DL_ERR_INVALID_ARG;
-  if (B == 0 || L == 0) return DL_OK;
-  if (!k_caches || !v_caches || !q_t || !k_t || !v_t || !out) return DL_ERR_INVALID_ARG;
+// Layers [l0, l1) of a decode step's stack, all with the same lengths, decision and capacity.  q_t, k_t, v_t, out
+// and the cache arrays are those of the whole stack (indexed by layer).  commit_len (null or the lengths, writable):
+// the launch of layer l1 - 1 also closes the step for these layers, cache_len[b] += keep[b], once every launch of the
+// group has read the lengths for the last time; groups in flight together use different commit slots.
+static int32_t decode_layer_range(dl_ctx* ctx, int32_t l0, int32_t l1, const void* q_t, const void* k_t,
+                                  const void* v_t, void* const* k_caches, void* const* v_caches,
+                                  const int32_t* cache_len, const uint8_t* keep, int32_t B, int32_t cap, float scale,
+                                  void* out, void* stream, int32_t* commit_len, int commit_slot) {
   const size_t layer_bytes = (size_t)B * ctx->desc.n_heads * ctx->desc.head_dim * elt_bytes(ctx);
-  ctx->opt.in_layer_stack = L > 1 ? 1 : 0;
-  for (int32_t l = 0; l < L; ++l) {
+  for (int32_t l = l0; l < l1; ++l) {
     const char* ql = static_cast<const char*>(q_t) + l * layer_bytes;
     const char* kl = static_cast<const char*>(k_t) + l * layer_bytes;
     const char* vl = static_cast<const char*>(v_t) + l * layer_bytes;
@@ -457,11 +458,24 @@ static int32_t decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void
     // consecutive layers touch different caches and outputs, so layer l may start while layer l-1 drains
     const bool overlap = l > 0 && k_caches[l] != k_caches[l - 1] && v_caches[l] != v_caches[l - 1];
     int32_t st = decode_layer(ctx, ql, kl, vl, k_caches[l], v_caches[l], cache_len, keep, B, cap, scale, ol, overlap,
-                              l % kDecodeScratchSets, stream, l == L - 1 ? commit_len : nullptr);
-    if (st != DL_OK) { ctx->opt.in_layer_stack = 0; return st; }
+                              l % kDecodeScratchSets, stream, l == l1 - 1 ? commit_len : nullptr, commit_slot);
+    if (st != DL_OK) return st;
   }
-  ctx->opt.in_layer_stack = 0;
   return DL_OK;
+}
+
+static int32_t decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
+                             void* const* k_caches, void* const* v_caches, const int32_t* cache_len,
+                             const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out, void* stream,
+                             int32_t* commit_len) {
+  if (!ctx || L < 0 || B < 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || L == 0) return DL_OK;
+  if (!k_caches || !v_caches || !q_t || !k_t || !v_t || !out) return DL_ERR_INVALID_ARG;
+  ctx->opt.in_layer_stack = L > 1 ? 1 : 0;
+  const int32_t st = decode_layer_range(ctx, 0, L, q_t, k_t, v_t, k_caches, v_caches, cache_len, keep, B, cap, scale,
+                                        out, stream, commit_len, 0);
+  ctx->opt.in_layer_stack = 0;
+  return st;
 }
 
 int32_t dl_sparse_attn_decode_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
@@ -485,6 +499,32 @@ int32_t dl_decode_step(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, 
   if (!cache_len) return DL_ERR_INVALID_ARG;
   return decode_layers(ctx, L, q_t, k_t, v_t, k_caches, v_caches, cache_len, keep_out, B, cap, scale, out, stream,
                        cache_len);
+}
+
+int32_t dl_decode_step_stack(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
+                             float* logit_inout, uint8_t* keep_out, const dl_layer_stack* stack, const void* q_t,
+                             const void* k_t, const void* v_t, float scale, void* out, void* stream) {
+  if (!ctx || !stack || B < 0) return DL_ERR_INVALID_ARG;
+  const int32_t L = stack->L, ld = stack->l_dense;
+  if (L < 0 || ld < 0 || ld > L) return DL_ERR_INVALID_ARG;
+  if (B == 0) return DL_OK;
+  if (L > 0 && (!stack->k_caches || !stack->v_caches || !q_t || !k_t || !v_t || !out)) return DL_ERR_INVALID_ARG;
+  if ((ld > 0 && (!stack->len_dense || stack->cap_dense <= 0)) || (ld < L && (!stack->cache_len || stack->cap <= 0)))
+    return DL_ERR_INVALID_ARG;
+  if (!ctx->ws.base || B > ctx->ws.max_batch) return DL_ERR_WORKSPACE;
+  int32_t st = dl_decode_keep(ctx, p_txt, x_t, B, threshold, logit_inout, keep_out, stream);
+  if (st != DL_OK) return st;
+  if (L == 0) return DL_OK;
+  ctx->opt.in_layer_stack = L > 1 ? 1 : 0;
+  // the dense layers keep every token: their decision is a vector of ones, their lengths grow by one per step
+  if (ld > 0)
+    st = decode_layer_range(ctx, 0, ld, q_t, k_t, v_t, stack->k_caches, stack->v_caches, stack->len_dense,
+                            ctx->ws.ones, B, stack->cap_dense, scale, out, stream, stack->len_dense, 1);
+  if (st == DL_OK && ld < L)
+    st = decode_layer_range(ctx, ld, L, q_t, k_t, v_t, stack->k_caches, stack->v_caches, stack->cache_len, keep_out,
+                            B, stack->cap, scale, out, stream, stack->cache_len, 0);
+  ctx->opt.in_layer_stack = 0;
+  return st;
 }
 
 int32_t dl_decode_step_host(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_host, int32_t B,

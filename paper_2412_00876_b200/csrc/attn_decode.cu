@@ -862,13 +862,14 @@ static int scratch_slots(const DecodeArgs& a) { return max_chunks(a) + 1; }
 cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t,
                                void* k_cache, void* v_cache, const int32_t* cache_len,
                                const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                               bool overlap_prev, int scratch_set, cudaStream_t s, int32_t* commit_len) {
+                               bool overlap_prev, int scratch_set, cudaStream_t s, int32_t* commit_len,
+                               int commit_slot) {
   if (B == 0) return cudaSuccess;
   if (B > kMaxDecodeBatch) return cudaErrorInvalidValue;
   const dl_model_desc& d = ctx->desc;
   DecodeArgs a;
   a.commit_len = keep ? commit_len : nullptr;
-  a.commit_count = ctx->ws.dec_commit;
+  a.commit_count = ctx->ws.dec_commit + (commit_slot & 1);
   a.q = q; a.k_t = k_t; a.v_t = v_t; a.k_cache = k_cache; a.v_cache = v_cache;
   a.cache_len = cache_len; a.keep = keep; a.out = out;
   a.status = ctx->ws.status;

@@ -50,7 +50,9 @@ struct Workspace {
   int32_t* dec_ticket = nullptr;      // [3][max_batch * H] arrivals per (b,h); zero between launches
   float* dec_partial = nullptr;       // [3][max_batch * H * dec_slots * (D + 2)]
   int32_t dec_slots = 0;              // partial slots per (b,h)
-  int32_t* dec_commit = nullptr;      // CTAs of a step's last attention launch that have finished; zero between launches
+  int32_t* dec_commit = nullptr;      // [2] CTAs of a committing attention launch that have finished (slot 0: compact
+                                      // layers, slot 1: dense layers); zero between launches
+  uint8_t* ones = nullptr;            // [max_batch] the keep-all decision of dense layers
   float* pred_partial = nullptr;      // [kPredMaxSplit][max_rows padded to kPredRowTile]
   int32_t* pred_ticket = nullptr;     // [row tiles]; zero between launches
   int32_t pred_rows_padded = 0;
@@ -127,7 +129,8 @@ cudaError_t launch_commit_len(const uint8_t* keep, int32_t B, int32_t cap, int32
 cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t,
                                void* k_cache, void* v_cache, const int32_t* cache_len,
                                const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                               bool overlap_prev, int scratch_set, cudaStream_t s, int32_t* commit_len = nullptr);
+                               bool overlap_prev, int scratch_set, cudaStream_t s, int32_t* commit_len = nullptr,
+                               int commit_slot = 0);
 
 cudaError_t launch_predictor_simt(const dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows,
                                   float* score, cudaStream_t s);
