@@ -22,6 +22,8 @@ int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_
   const int32_t rows_pad = (max_rows + kPredRowTile - 1) / kPredRowTile * kPredRowTile;
   const int64_t o_ppart = take((int64_t)kPredMaxSplit * rows_pad * 4);
   const int64_t o_ptick = take((int64_t)(rows_pad / kPredRowTile + 1) * 4);
+  const int64_t o_psplit = take((int64_t)d.pred_hidden * kPredKSplit * kPredRowTile * 4);
+  const int64_t o_pstick = take((int64_t)kPredMaxSplit * 4);
   const int64_t o_commit = take(2 * 4);
   const int64_t o_ones = take(max_batch);
   if (ws) {
@@ -34,6 +36,8 @@ int64_t workspace_layout(const dl_model_desc& d, int32_t max_batch, int32_t max_
     ws->dec_slots = slots;
     ws->pred_partial = reinterpret_cast<float*>(b + o_ppart);
     ws->pred_ticket = reinterpret_cast<int32_t*>(b + o_ptick);
+    ws->pred_split = reinterpret_cast<float*>(b + o_psplit);
+    ws->pred_split_ticket = reinterpret_cast<int32_t*>(b + o_pstick);
     ws->dec_commit = reinterpret_cast<int32_t*>(b + o_commit);
     ws->ones = reinterpret_cast<uint8_t*>(b + o_ones);
     ws->pred_rows_padded = rows_pad;
@@ -152,6 +156,7 @@ int32_t dl_set_workspace(dl_ctx* ctx, void* dev_ptr, int64_t bytes, int32_t max_
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ctx->ws.pred_ticket, 0, (size_t)(ctx->ws.pred_rows_padded / kPredRowTile + 1) * 4, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.dec_commit, 0, 2 * 4, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.pred_split_ticket, 0, (size_t)kPredMaxSplit * 4, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.ones, 1, (size_t)max_batch, s);
   return cuda_status(ctx, e);
 }

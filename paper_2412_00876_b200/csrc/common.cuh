@@ -36,6 +36,7 @@ __device__ __forceinline__ void report_status(DeviceStatus* st, int32_t code, lo
 constexpr int kDecodeMinChunk = 64;   // smallest rows-per-item the decode kernel may be asked for
 constexpr int kDecodeScratchSets = 3; // decode scratch sets (see Workspace)
 constexpr int kPredMaxSplit = 80;     // most unit tiles of the predictor's hidden layer
+constexpr int kPredKSplit = 8;        // most ranges of the hidden dimension a unit tile of the decode-shape predictor is cut into
 constexpr int kPredRowTile = 128;     // rows per predictor row tile (tensor-core kernel)
 
 struct Workspace {
@@ -55,6 +56,8 @@ struct Workspace {
   uint8_t* ones = nullptr;            // [max_batch] the keep-all decision of dense layers
   float* pred_partial = nullptr;      // [kPredMaxSplit][max_rows padded to kPredRowTile]
   int32_t* pred_ticket = nullptr;     // [row tiles]; zero between launches
+  float* pred_split = nullptr;        // [unit tiles][kPredKSplit][kPredRowTile][tile width] raw sums of the decode-shape predictor
+  int32_t* pred_split_ticket = nullptr;   // [kPredMaxSplit]; zero between launches
   int32_t pred_rows_padded = 0;
 };
 

@@ -7,7 +7,9 @@
 // in fp32.  Persistent CTAs walk work items (row tile, unit tile) in an order that lets the CTAs
 // that run side by side share one X tile through L2; a row tile's partial sums (one per unit
 // tile) are added in tile order by the CTA that finishes last (a ticket, not a wait), so the
-// logits are reproducible bit for bit.
+// logits are reproducible bit for bit.  With a single row tile (the decode shape: one row per sequence) the
+// hidden dimension is also split over CTAs: each takes a range of it for its unit tile, leaves the raw fp32
+// sums in scratch, and the last of a unit tile's CTAs to arrive adds the ranges in order before the GELU.
 //   warp 0 : TMA producer (X and W1 tiles, 128-byte swizzle; a ring of 4 stages for prefill shapes, up to 32
 //            short stages for the few rows of a decode step)
 //   warp 1 : tensor-memory allocation and the single MMA-issuing thread
@@ -40,6 +42,9 @@ struct PredTcArgs {
   int32_t stages, stage_bytes, a_bytes;   // ring depth; bytes per stage; bytes of its X part
   int32_t kbs, a_tile, b_tile;            // 64-column blocks of the hidden dimension per stage; bytes of one X / one W1 block
   uint8_t* keep; float threshold;         // decode decision fused into the final sum (keep may be null)
+  int32_t row_box;                        // rows of X fetched per stage (32, 64 or 128); below 128 only with one row tile
+  int32_t k_split, kb_per;                // CTAs per unit tile along the hidden dimension; 64-column blocks each takes
+  float* split; int32_t* split_ticket;    // [n_tiles][k_split][128][bn] raw sums; [n_tiles] arrivals, zero between launches
 };
 
 // score and, if asked for, the decision keep = score > threshold (strictly; a NaN score drops and is reported)
@@ -68,10 +73,11 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
   __shared__ uint32_t sh_tmem;
   __shared__ int sh_abort;
   __shared__ int sh_ticket;
+  __shared__ float sh_red[4][kPtBM];      // sums of the threads that share a row, added in order by the row's first thread
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_flag = &sh_abort;
-  const int items = a.m_tiles * a.n_tiles;
+  const int items = a.m_tiles * a.n_tiles * a.k_split;
 
   if (tid == 0) {
     sh_abort = 0;
@@ -96,8 +102,10 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
       tma_prefetch_desc(&map_w);
       int it = 0, s = 0, ph = 0;                 // stage and phase of fill `it`, kept by counting (NS is a run-time value)
       for (int item = blockIdx.x; item < items && !*abort_flag; item += gridDim.x) {
-        const int mt = item / a.n_tiles, nt = item - mt * a.n_tiles;
-        for (int kb = 0; kb < a.k_blocks; kb += a.kbs, ++it) {
+        const int tile = item / a.k_split, sp = item - tile * a.k_split;
+        const int mt = tile / a.n_tiles, nt = tile - mt * a.n_tiles;
+        const int kb_end = min(a.k_blocks, (sp + 1) * a.kb_per);
+        for (int kb = sp * a.kb_per; kb < kb_end; kb += a.kbs, ++it) {
           if (!mbar_wait(smem_u32(&empty[s]), ph ^ 1, abort_flag)) break;
           const uint32_t fb = smem_u32(&full[s]);
           mbar_expect_tx(fb, (uint32_t)a.a_bytes + b_bytes);
@@ -128,7 +136,9 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         mbar_wait(smem_u32(&acc_empty[buf]), ((j >> 1) & 1) ^ 1, abort_flag);
         tc_fence_after();
         const uint32_t d_tmem = tmem + (uint32_t)(buf * a.bn);
-        for (int kb = 0; kb < a.k_blocks; kb += a.kbs) {
+        const int sp = item % a.k_split;
+        const int kb0 = sp * a.kb_per, kb_end = min(a.k_blocks, kb0 + a.kb_per);
+        for (int kb = kb0; kb < kb_end; kb += a.kbs) {
           mbar_wait(smem_u32(&full[s]), ph, abort_flag);
           tc_fence_after();
           // descriptors differ from the stage-0, block-0, k-0 ones only in the start-address field (16-byte units)
@@ -137,7 +147,7 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
           for (int kk = 0; kk < a.kbs; ++kk, da += a.a_tile >> 4, db += a.b_tile >> 4) {
 #pragma unroll
             for (int k = 0; k < kPtBK / 16; ++k)
-              mma_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | kk | k) != 0);
+              mma_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - kb0) | kk | k) != 0);
           }
           mma_commit(smem_u32(&empty[s]));             // frees the stage when these MMAs have read it
           if (++s == NS) { s = 0; ph ^= 1; }
@@ -151,26 +161,90 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     const int et = (warp - 2) * 32 + lane;              // 0..127 among the epilogue threads
     int j = 0;
     for (int item = blockIdx.x; item < items; item += gridDim.x, ++j) {
-      const int mt = item / a.n_tiles, nt = item - mt * a.n_tiles;
+      const int tile = item / a.k_split, sp = item - tile * a.k_split;
+      const int mt = tile / a.n_tiles, nt = tile - mt * a.n_tiles;
       const int buf = j & 1;
       mbar_wait(smem_u32(&acc_full[buf]), (j >> 1) & 1, abort_flag);
       tc_fence_after();
       const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * a.bn);
       const float* b1 = a.b1 + (size_t)nt * a.bn;
       const float* w2 = a.w2 + (size_t)nt * a.bn;
-      float sum = 0.f;
-      for (int c = 0; c < a.bn; c += 32) {
-        uint32_t r[32];
-        tmem_ld32(t_row + c, r);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-          sum = fmaf(__ldg(w2 + c + i), gelu_erf(__uint_as_float(r[i]) + __ldg(b1 + c + i)), sum);
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
       const int row = mt * kPtBM + quad * 32 + lane;
+      float sum = 0.f;
+      if (a.k_split == 1) {
+        for (int c = 0; c < a.bn; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(t_row + c, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            sum = fmaf(__ldg(w2 + c + i), gelu_erf(__uint_as_float(r[i]) + __ldg(b1 + c + i)), sum);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+      } else {
+        // this CTA's range of the hidden dimension: raw sums out, the last range to arrive finishes the unit tile
+        float* mine = a.split + (((size_t)nt * a.k_split + sp) * kPtBM + (quad * 32 + lane)) * a.bn;
+        for (int c = 0; c < a.bn; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(t_row + c, r);
+          tmem_ld_wait();
+          if (row < a.rows) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              *reinterpret_cast<uint4*>(mine + c + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+        __threadfence();
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        if (et == 0) sh_ticket = atomicAdd(&a.split_ticket[nt], 1);
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        if (sh_ticket != a.k_split - 1) continue;
+        __threadfence();
+        if (et == 0) a.split_ticket[nt] = 0;
+        // all 128 threads share the work: with a short row box several threads take a row, a slice of the unit
+        // tile each; a slice's loads (every range, eight columns) go out together, one round trip per eight columns
+        const int er = quad * 32 + lane, tpr = kPtBM / a.row_box;
+        const int mrow = er % a.row_box, part = er / a.row_box, cw = a.bn / tpr;
+        float ps = 0.f;
+        if (mrow < a.rows) {
+          const float* p0 = a.split + ((size_t)nt * a.k_split * kPtBM + mrow) * a.bn;
+          for (int c = part * cw; c < (part + 1) * cw; c += 8) {
+            float4 v[kPredKSplit][2];
+#pragma unroll
+            for (int q = 0; q < kPredKSplit; ++q) {
+              if (q < a.k_split) {
+                v[q][0] = __ldcg(reinterpret_cast<const float4*>(p0 + (size_t)q * kPtBM * a.bn + c));
+                v[q][1] = __ldcg(reinterpret_cast<const float4*>(p0 + (size_t)q * kPtBM * a.bn + c + 4));
+              }
+            }
+            float4 s0 = v[0][0], s1 = v[0][1];
+#pragma unroll
+            for (int q = 1; q < kPredKSplit; ++q) {
+              if (q < a.k_split) {
+                s0.x += v[q][0].x; s0.y += v[q][0].y; s0.z += v[q][0].z; s0.w += v[q][0].w;
+                s1.x += v[q][1].x; s1.y += v[q][1].y; s1.z += v[q][1].z; s1.w += v[q][1].w;
+              }
+            }
+            ps = fmaf(__ldg(w2 + c), gelu_erf(s0.x + __ldg(b1 + c)), ps);
+            ps = fmaf(__ldg(w2 + c + 1), gelu_erf(s0.y + __ldg(b1 + c + 1)), ps);
+            ps = fmaf(__ldg(w2 + c + 2), gelu_erf(s0.z + __ldg(b1 + c + 2)), ps);
+            ps = fmaf(__ldg(w2 + c + 3), gelu_erf(s0.w + __ldg(b1 + c + 3)), ps);
+            ps = fmaf(__ldg(w2 + c + 4), gelu_erf(s1.x + __ldg(b1 + c + 4)), ps);
+            ps = fmaf(__ldg(w2 + c + 5), gelu_erf(s1.y + __ldg(b1 + c + 5)), ps);
+            ps = fmaf(__ldg(w2 + c + 6), gelu_erf(s1.z + __ldg(b1 + c + 6)), ps);
+            ps = fmaf(__ldg(w2 + c + 7), gelu_erf(s1.w + __ldg(b1 + c + 7)), ps);
+          }
+        }
+        sh_red[part][mrow] = ps;
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        if (part == 0)
+          for (int q = 0; q < tpr; ++q) sum += sh_red[q][mrow];
+      }
       if (a.n_tiles == 1) {
         if (row < a.rows) pt_emit(a, row, sum + a.b2);
         continue;
@@ -182,10 +256,26 @@ predictor_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
       asm volatile("bar.sync 2, 128;" ::: "memory");
       if (sh_ticket == a.n_tiles - 1) {
         __threadfence();
-        const int r2 = mt * kPtBM + et;
-        float tot = 0.f;
-        for (int t = 0; t < a.n_tiles; ++t) tot += __ldcg(a.partial + (size_t)t * a.rows_padded + r2);
-        if (r2 < a.rows) pt_emit(a, r2, tot + a.b2);
+        // threads that share a row take a run of unit tiles each; eight loads go out together
+        const int er = quad * 32 + lane, tpr = kPtBM / a.row_box;
+        const int mrow = er % a.row_box, part = er / a.row_box, tn = (a.n_tiles + tpr - 1) / tpr;
+        const int t_end = min(a.n_tiles, (part + 1) * tn);
+        const float* pr = a.partial + (size_t)mt * kPtBM + mrow;
+        float ps = 0.f;
+        for (int t0 = part * tn; t0 < t_end; t0 += 8) {
+          float v[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v[i] = (t0 + i < t_end) ? __ldcg(pr + (size_t)(t0 + i) * a.rows_padded) : 0.f;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) ps += v[i];
+        }
+        sh_red[part][mrow] = ps;
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        if (part == 0) {
+          float tot = 0.f;
+          for (int q = 0; q < tpr; ++q) tot += sh_red[q][mrow];
+          if (row < a.rows) pt_emit(a, row, tot + a.b2);
+        }
         if (et == 0) a.ticket[mt] = 0;
       }
     }
@@ -237,11 +327,23 @@ cudaError_t launch_predictor_tc(dl_ctx* ctx, const dl_predictor* p, const void* 
   // ... and a copy of a 32 x 64 box costs the producer as much as one of 128 x 64, so a stage of the short form takes
   // four 64-column blocks of the hidden dimension per copy.
   a.kbs = (row_box < kPtBM && a.k_blocks % 4 == 0) ? 4 : 1;
+  a.row_box = row_box;
   a.a_tile = row_box * kPtBK * 2;
   a.b_tile = bn * kPtBK * 2;
   a.a_bytes = a.kbs * a.a_tile;
   a.stage_bytes = a.a_bytes + a.kbs * a.b_tile;
-  a.stages = std::max(2, std::min({kPtMaxStages, (4 * kPtStageBytes) / a.stage_bytes, a.k_blocks / a.kbs}));
+  // One row tile: the hidden dimension is cut into ranges (whole stages each) for as many CTAs as the GPU has SMs.
+  a.k_split = 1;
+  a.kb_per = a.k_blocks;
+  if (m_tiles == 1 && ctx->ws.pred_split != nullptr) {
+    const int want = std::min({ctx->sm_count / a.n_tiles, kPredKSplit, a.k_blocks / a.kbs});
+    if (want > 1) {
+      a.kb_per = ((a.k_blocks + want - 1) / want + a.kbs - 1) / a.kbs * a.kbs;
+      a.k_split = (a.k_blocks + a.kb_per - 1) / a.kb_per;
+    }
+  }
+  a.split = ctx->ws.pred_split; a.split_ticket = ctx->ws.pred_split_ticket;
+  a.stages = std::max(2, std::min({kPtMaxStages, (4 * kPtStageBytes) / a.stage_bytes, a.kb_per / a.kbs}));
   int cols = 32;
   while (cols < 2 * bn) cols <<= 1;
   a.tmem_cols = cols;
@@ -264,7 +366,7 @@ cudaError_t launch_predictor_tc(dl_ctx* ctx, const dl_predictor* p, const void* 
     if (e != cudaSuccess) return e;
     attr_set[ctx->device & 63] = 1;
   }
-  const int grid = min(ctx->sm_count, m_tiles * a.n_tiles);
+  const int grid = min(ctx->sm_count, m_tiles * a.n_tiles * a.k_split);
   predictor_tc_kernel<<<grid, kPtThreads, kPtSmem, s>>>(mx, mw, a);
   return cudaGetLastError();
 }
