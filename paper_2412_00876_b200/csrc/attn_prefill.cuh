@@ -14,6 +14,7 @@ constexpr int kAtOffBar = kAtOffRing + kAtRing * kAtTile;
 constexpr size_t kAtSmem = kAtOffBar + 512;           // 229888 bytes: one CTA per SM
 constexpr uint32_t kAtColO = 0, kAtColS = 128, kAtLaneCols = 256;   // tensor-memory columns of one lane: O | S
 constexpr float kRescaleStep = 8.0f;                  // log2 units by which the maximum may lag
+constexpr int kAtTopRows = 16;                        // a top tile of at most this many rows is left to at_top_rows()
 
 // 2^x on the special-function unit (x <= 0 here; -inf gives 0)
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -65,13 +66,14 @@ __device__ __forceinline__ int at_box(int rows) { return rows > 64 ? 0 : rows > 
 
 struct AtArgs {
   const int32_t* cache_len; __nv_bfloat16* out; DeviceStatus* status;
+  const __nv_bfloat16* q; const __nv_bfloat16* k; const __nv_bfloat16* v;   // the tensors the maps describe
   int32_t B, H, cap, n_max, q_pairs, item_rows;     // item_rows: query rows per work item (256: a pair of tiles; 128)
   float scale_log2;
 };
 
 // Work item -> (b, h, pair p of query tiles).  Pair p counts from the sequence's end: it covers rows
 // [q_hi - 256, q_hi) with q_hi = n - 256 p, clipped at row 0; its keys are [0, q_hi) in n_kv tiles.
-struct AtItem { int b, h, q_hi, n, n_kv, row_base, swap; };
+struct AtItem { int b, h, q_hi, n, n_kv, row_base, swap, cut; };   // cut: a tile of at most `cut` rows is nobody's lane
 
 // One lane's share of an item: rows [q0, q_hi) are owned (the Q tile is loaded from row q0, 128 rows;
 // a tile clipped at the top of the sequence loads rows [0, 128) and owns the first q_hi of them),
@@ -81,7 +83,7 @@ struct AtLane { int q0, q_hi, n_tiles; bool exists; };
 __device__ __forceinline__ AtLane at_lane(const AtItem& I, int lane_id) {
   AtLane L;
   L.q_hi = I.q_hi - (lane_id ^ I.swap) * kAtBM;
-  L.exists = L.q_hi > 0;
+  L.exists = L.q_hi > I.cut;
   L.q0 = max(L.q_hi - kAtBM, 0);
   L.n_tiles = (L.q_hi + kAtBN - 1) / kAtBN;
   return L;
@@ -120,8 +122,9 @@ struct AtWalker {
     sw = 0;
     len = p < a.q_pairs ? ld_early(a.cache_len + b) : 0;
   }
-  // Advances to the next item that exists (a sequence of 256 p rows or fewer has no pair p).
-  __device__ __forceinline__ bool next(AtItem& I) {
+  // Advances to the next item that exists (a sequence of 256 p rows or fewer has no pair p; with cut > 0 neither
+  // has one whose later tile would have at most `cut` rows).
+  __device__ __forceinline__ bool next(AtItem& I, int cut) {
     for (;;) {
       if (p >= a.q_pairs) return false;
       const int cp = p, cb = b, ch = h, clen = len;
@@ -134,7 +137,8 @@ struct AtWalker {
       I.h = ch;
       I.n = min(max(clen, 0), min(a.cap, a.n_max));
       I.q_hi = I.n - cp * a.item_rows;
-      if (I.q_hi <= 0) continue;
+      if (I.q_hi <= cut) continue;
+      I.cut = cut;
       I.n_kv = (I.q_hi + kAtBN - 1) / kAtBN;
       I.row_base = (cb * a.H + ch) * a.cap;                         // first row of this (b, h) in the caches
       I.swap = (kAtSwapLanes && a.item_rows == 2 * kAtBM) ? sw : 0;

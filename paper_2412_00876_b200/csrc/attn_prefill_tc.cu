@@ -29,7 +29,8 @@
 //                top of a sequence, whose surplus rows belong to the next tile, is written with
 //                predicated stores instead.  The Q slot returns to the producer once those stores
 //                have read it.
-//   warp 11    : tensor-memory allocation (all 512 columns: O_A | S_A | O_B | S_B).
+//   warp 11    : tensor-memory allocation (all 512 columns: O_A | S_A | O_B | S_B); then the top rows of sequences
+//                whose length leaves a top tile of at most 16 rows (attn_prefill_top.cuh), which the lanes skip.
 // Barrier phases are driven by running counters (ring tiles, a lane's tiles, a lane's items) that every
 // role advances identically.  Rows past a sequence's length are fetched with the tile (they are
 // masked); where the 16-row rounding of the last tile reaches past the sequence's end, those V rows
@@ -42,6 +43,7 @@
 
 #include "attn_prefill.cuh"
 #include "attn_prefill_softmax.cuh"
+#include "attn_prefill_top.cuh"
 
 namespace dl {
 
@@ -121,7 +123,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       while ((hr || hq) && !*abort_flag) {
         bool prog = false;
         if (hq && need_q) {
-          hq = Wq.next(Iq);
+          hq = Wq.next(Iq, kAtTopRows);
           need_q = false;
           q_todo = hq ? ((at_lane(Iq, 0).exists ? 1 : 0) | (at_lane(Iq, 1).exists ? 2 : 0)) : 0;
           prog = true;
@@ -146,7 +148,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
         }
         if (hq && !need_q && q_todo == 0) need_q = true;
         if (hr && need_r) {
-          hr = Wr.next(Ir);
+          hr = Wr.next(Ir, kAtTopRows);
           need_r = false;
           jr = 0;
           prog = true;
@@ -200,7 +202,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       AtWalker W(a);
       AtItem I;
       int n_item = 0, g0 = 0, T0 = 0;                 // this lane's items / tiles so far; ring tiles before this item
-      while (W.next(I)) {
+      while (W.next(I, kAtTopRows)) {
         const AtLane L = at_lane(I, x);
         auto wait_ring = [&](int T) { mbar_wait_spin(ring_full(T % kAtRing), (T / kAtRing) & 1, abort_flag); };
         const int n_sub = L.exists ? L.n_tiles : 0;
@@ -285,7 +287,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     AtItem I;
     int n_item = 0, g0 = 0, T0 = 0;
     int q_slot_held = -1;                                              // Q slot whose staged stores are still in flight
-    while (W.next(I)) {
+    while (W.next(I, kAtTopRows)) {
       const AtLane L = at_lane(I, x);
       if (!L.exists) { T0 += 2 * I.n_kv; continue; }
       const int grow = L.q0 + row;                                     // row within the sequence
@@ -388,7 +390,15 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     if (q_slot_held >= 0 && lane == 0) { bulk_wait_read<0>(); mbar_arrive(q_done(x, q_slot_held)); }
     if (*abort_flag && row == 0) report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
   } else {
-    reg_dec<kAtRegsSmall>();                             // warp 11: same budget as the rest of its warpgroup
+    // ---------------------------------------------------------------- warp 11: the top rows the lanes leave out
+    reg_dec<kAtRegsSmall>();                             // same budget as the rest of its warpgroup
+    AtWalker W(a);
+    AtItem I;
+    while (W.next(I, 0)) {
+      // the pair's later tile if it is that small, else its earlier one if that is
+      const int s = I.q_hi <= kAtTopRows ? I.q_hi : I.q_hi - kAtBM;
+      if (s > 0 && s <= kAtTopRows) at_top_rows(a, I, s, lane);
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -426,6 +436,8 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
     return cudaErrorInvalidValue;
   AtArgs a;
   a.cache_len = cache_len; a.out = static_cast<__nv_bfloat16*>(out); a.status = ctx->ws.base ? ctx->ws.status : nullptr;
+  a.q = static_cast<const __nv_bfloat16*>(q); a.k = static_cast<const __nv_bfloat16*>(k_cache);
+  a.v = static_cast<const __nv_bfloat16*>(v_cache);
   a.item_rows = 2 * kAtBM;
   a.B = B; a.H = d.n_heads; a.cap = cap; a.n_max = n_max; a.q_pairs = (n_max + a.item_rows - 1) / a.item_rows;
   a.scale_log2 = scale * 1.4426950408889634f;

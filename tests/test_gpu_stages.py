@@ -421,6 +421,14 @@ def test_prefill_attention_tile_pair_boundaries():
     _prefill_case("bf16", 3, 128, [640])
 
 
+def test_prefill_attention_top_rows_of_a_sequence():
+    """Lengths that leave a top tile of 1..16 rows: alone in its pair (n = 256 m + r), beside a full later tile
+    (n = 256 m + 128 + r), as the whole sequence, with r not a multiple of 16; those rows take a path of their own
+    in the tensor-core kernel.  17 rows are the first length that does not."""
+    _prefill_case("bf16", 2, 128, [261, 140, 400, 9, 16, 528, 272, 17])
+    _prefill_case("bf16", 1, 128, [144, 133, 769, 3])
+
+
 def test_prefill_attention_large_scores():
     """Scores whose row maximum keeps growing by far more than 2^8 from one key tile to the next: the
     tensor-core kernel has to rescale its accumulator and redo tiles (its rare path)."""
