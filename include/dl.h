@@ -354,6 +354,30 @@ int32_t dl_decode_keep2(dl_ctx* ctx, const dl_predictor2* p_txt, const void* x_t
  * dl_device_status then reports the code. */
 int32_t dl_selftest_wait_timeout(dl_ctx* ctx, int32_t polls, void* stream);
 
+/* ---- extension, NOT in the paper: K/V cache in 8-bit floating point ---------------------- */
+
+/* Decode attention (Eq. 6) is bound by the bytes of the cache it streams; these two calls store the cache rows as
+ * 8-bit floating point in the OCP E4M3 format (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; largest value
+ * 448; no infinities) with one fp32 scale per head and tensor:  value = decode(byte) * scale[h].
+ * bf16 models with head_dim 128 only (DL_ERR_UNSUPPORTED otherwise). */
+
+/* Rows [0, cache_len[b]) of a bf16 cache as bytes: byte = encode(x / scale[h]), the quotient in fp32, round to
+ * nearest with ties to the even code, magnitudes above 448 clamped to 448.  Rows at and past cache_len[b] are not
+ * written.
+ *   src dev [B][H][cap][128] bf16; scale dev [H] fp32 (> 0); dst dev [B][H][cap][128] uint8 (caller's). */
+int32_t dl_quantize_kv_fp8(dl_ctx* ctx, const void* src, const int32_t* cache_len, const float* scale, int32_t B,
+                           int32_t cap, void* dst, void* stream);
+
+/* dl_sparse_attn_decode over such caches: the cached rows are read as decode(byte) * scale[h]; the current token is
+ * attended with its own bf16 k_t, v_t (kept or not) and, where keep[b] != 0 and the cache has room, appended as
+ * bytes at row cache_len[b] (lengths are NOT advanced: dl_commit_len closes the step).
+ *   q_t, k_t, v_t, out dev [B][H][128] bf16; k_cache, v_cache dev [B][H][cap][128] uint8, read and (row cache_len[b])
+ *   written; k_scale, v_scale dev [H] fp32; keep dev [B] or NULL.  Needs the workspace (split sequences). */
+int32_t dl_sparse_attn_decode_fp8(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
+                                  void* v_cache, const float* k_scale, const float* v_scale,
+                                  const int32_t* cache_len, const uint8_t* keep, int32_t B, int32_t cap, float scale,
+                                  void* out, void* stream);
+
 /* ---- decode attention without any allocation ------------------------------------------- */
 
 /* Size of the library's built-in scratch array (bytes). */

@@ -29,7 +29,7 @@ EXPORTS = [
     "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers", "dl_decode_nocache_select",
     "dl_decode_steps_host", "dl_compact_kv_host", "dl_selftest_wait_timeout", "dl_compact_kv_layers",
     "dl_predictor2_scratch_bytes", "dl_predictor2_values", "dl_prefill_select2", "dl_decode_keep2",
-    "dl_decode_step_stack",
+    "dl_decode_step_stack", "dl_quantize_kv_fp8", "dl_sparse_attn_decode_fp8",
 ]
 
 
@@ -129,6 +129,8 @@ def lib() -> C.CDLL:
                                      C.POINTER(vp), i32, vp, f32, vp, vp]),
             "dl_decode_step_stack": (i32, [vp, P, vp, i32, f32, vp, vp, C.POINTER(LayerStackDesc), vp, vp, vp, f32,
                                            vp, vp]),
+            "dl_quantize_kv_fp8": (i32, [vp, vp, vp, vp, i32, i32, vp, vp]),
+            "dl_sparse_attn_decode_fp8": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp]),
             "dl_decode_step_host": (i32, [vp, P, vp, i32, f32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                           vp, vp, C.POINTER(vp), C.POINTER(vp), i32, vp, f32, vp]),
             "dl_decode_steps_host": (i32, [vp, P, i32, i32, f32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
@@ -285,6 +287,20 @@ class Context:
         self._check(lib().dl_sparse_attn_decode(self._h, _ptr(q_t), _ptr(k_t), _ptr(v_t), _ptr(k_cache),
                                                 _ptr(v_cache), _ptr(cache_len), _ptr(keep), B, cap, float(scale),
                                                 _ptr(out), _stream(stream)), "dl_sparse_attn_decode")
+
+    def quantize_kv_fp8(self, src, cache_len, scale, dst, stream=None):
+        """Extension (not in the paper): rows of a bf16 cache as E4M3 bytes under per-head scales."""
+        B, cap = src.shape[0], src.shape[2]
+        self._check(lib().dl_quantize_kv_fp8(self._h, _ptr(src), _ptr(cache_len), _ptr(scale), B, cap, _ptr(dst),
+                                             _stream(stream)), "dl_quantize_kv_fp8")
+
+    def sparse_attn_decode_fp8(self, q_t, k_t, v_t, k_cache, v_cache, k_scale, v_scale, cache_len, keep, scale, out,
+                               stream=None):
+        B, cap = k_cache.shape[0], k_cache.shape[2]
+        self._check(lib().dl_sparse_attn_decode_fp8(self._h, _ptr(q_t), _ptr(k_t), _ptr(v_t), _ptr(k_cache),
+                                                    _ptr(v_cache), _ptr(k_scale), _ptr(v_scale), _ptr(cache_len),
+                                                    _ptr(keep), B, cap, float(scale), _ptr(out), _stream(stream)),
+                    "dl_sparse_attn_decode_fp8")
 
     def sparse_attn_decode_static(self, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, scale, out, stream=None):
         """dl_sparse_attn_decode for callers that may not allocate device memory: the kernel's scratch

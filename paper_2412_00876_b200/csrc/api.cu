@@ -404,6 +404,37 @@ int32_t dl_sparse_attn_decode(dl_ctx* ctx, const void* q_t, const void* k_t, con
   return decode_layer(ctx, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, B, cap, scale, out, false, 0, stream);
 }
 
+int32_t dl_quantize_kv_fp8(dl_ctx* ctx, const void* src, const int32_t* cache_len, const float* scale, int32_t B,
+                           int32_t cap, void* dst, void* stream) {
+  if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
+  if (B == 0) return DL_OK;
+  if (!src || !cache_len || !scale || !dst) return DL_ERR_INVALID_ARG;
+  if (misaligned(src) || misaligned(dst)) return DL_ERR_ALIGNMENT;
+  if (ctx->desc.dtype != DL_BF16 || ctx->desc.head_dim != 128) return DL_ERR_UNSUPPORTED;
+  DeviceGuard g(ctx->device);
+  return cuda_status(ctx, launch_quantize_kv_fp8(ctx, src, cache_len, scale, B, cap, dst,
+                                                 static_cast<cudaStream_t>(stream)));
+}
+
+int32_t dl_sparse_attn_decode_fp8(dl_ctx* ctx, const void* q_t, const void* k_t, const void* v_t, void* k_cache,
+                                  void* v_cache, const float* k_scale, const float* v_scale,
+                                  const int32_t* cache_len, const uint8_t* keep, int32_t B, int32_t cap, float scale,
+                                  void* out, void* stream) {
+  if (!ctx || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
+  if (B == 0) return DL_OK;
+  if (!q_t || !k_t || !v_t || !k_cache || !v_cache || !k_scale || !v_scale || !cache_len || !out)
+    return DL_ERR_INVALID_ARG;
+  if (misaligned(q_t) || misaligned(k_t) || misaligned(v_t) || misaligned(k_cache) || misaligned(v_cache) ||
+      misaligned(out))
+    return DL_ERR_ALIGNMENT;
+  if (ctx->desc.dtype != DL_BF16 || ctx->desc.head_dim != 128 || !ctx->tmap_encode) return DL_ERR_UNSUPPORTED;
+  if (!ctx->ws.base || B > ctx->ws.max_batch || cap > ctx->ws.cap) return DL_ERR_WORKSPACE;
+  if (B > 2048) return DL_ERR_UNSUPPORTED;
+  DeviceGuard g(ctx->device);
+  return cuda_status(ctx, launch_attn_decode_fp8(ctx, q_t, k_t, v_t, k_cache, v_cache, k_scale, v_scale, cache_len,
+                                                 keep, B, cap, scale, out, static_cast<cudaStream_t>(stream)));
+}
+
 int32_t dl_decode_keep(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
                        float* logit_inout, uint8_t* keep_out, void* stream) {
   if (!ctx || B < 0) return DL_ERR_INVALID_ARG;

@@ -135,6 +135,13 @@ cudaError_t launch_attn_decode(const dl_ctx* ctx, const void* q, const void* k_t
                                bool overlap_prev, int scratch_set, cudaStream_t s, int32_t* commit_len = nullptr,
                                int commit_slot = 0);
 
+cudaError_t launch_quantize_kv_fp8(const dl_ctx* ctx, const void* src, const int32_t* cache_len, const float* scale,
+                                   int32_t B, int32_t cap, void* dst, cudaStream_t s);
+cudaError_t launch_attn_decode_fp8(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t, void* k_cache,
+                                   void* v_cache, const float* k_scale, const float* v_scale, const int32_t* cache_len,
+                                   const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
+                                   cudaStream_t s);
+
 cudaError_t launch_predictor_simt(const dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows,
                                   float* score, cudaStream_t s);
 // keep != nullptr: also keep[r] = score[r] > threshold (the decode decision, taken where the score is completed)

@@ -1,0 +1,111 @@
+"""GPU parity of the 8-bit K/V cache extension (not in the paper) against oracle/fp8_cache.py: the stored bytes are
+compared bit for bit, the attention output within the bf16 path's tolerances against the oracle ON THE SAME BYTES;
+what quantisation itself costs against the unquantised oracle is printed, not bounded."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dl_oracle as orc
+from oracle import fp8_cache as f8
+from paper_2412_00876_b200 import workloads as wl
+from tests.path_check import att_errors, check_att
+
+pytestmark = pytest.mark.gpu
+DEV = torch.device("cuda", 0)
+
+
+def _setup(B, H, cap, seed):
+    from paper_2412_00876_b200 import binding as dl
+    D = 128
+    rng = np.random.default_rng(seed)
+    ctx = dl.Context(256, H, D, 64, torch.bfloat16, 0, max_batch=B, max_rows=B, cap=cap)
+    r = lambda *shape: wl.round_to_storage(rng.normal(0, 1, shape).astype(np.float32), "bf16")
+    return dl, ctx, rng, r, D
+
+
+def test_quantise_is_bit_exact():
+    B, H, cap = 3, 4, 80
+    dl, ctx, rng, r, D = _setup(B, H, cap, 1)
+    src = r(B, H, cap, D)
+    src[0, 0, 0, :8] = [0.0, -0.0, 1e-4, -1e-4, 500.0, -500.0, 0.0625, 3.0]       # zeros, tiny, clamped values
+    scale = np.array([0.01, 0.05, 0.5, 2.0 ** -6], np.float32)
+    lens = np.array([80, 17, 0], np.int32)
+    dst = torch.full((B, H, cap, D), 0xAB, dtype=torch.uint8, device=DEV)
+    ctx.quantize_kv_fp8(wl.to_torch(src, "bf16", DEV), torch.from_numpy(lens).to(DEV), torch.from_numpy(scale).to(DEV), dst)
+    got = dst.cpu().numpy()
+    ref = f8.quantize_rows(src, scale[None, :, None, None])
+    for b in range(B):
+        assert np.array_equal(got[b, :, : lens[b]], ref[b, :, : lens[b]]), f"sequence {b}"
+        assert np.all(got[b, :, lens[b]:] == 0xAB)                    # rows past the length are not written
+    assert ctx.device_status()[0] == 0
+    ctx.close()
+
+
+@pytest.mark.parametrize("B,H,cap,lens", [(4, 4, 320, [0, 1, 31, 300]), (2, 8, 1408, [1300, 777]),
+                                           (5, 2, 128, [32, 33, 64, 100, 127])])
+def test_decode_attention_and_append_over_the_byte_cache(B, H, cap, lens):
+    """Ragged lengths over several 32-row tiles and split sequences; kept tokens are appended as bytes."""
+    dl, ctx, rng, r, D = _setup(B, H, cap, 7 + B)
+    lens = np.array(lens, np.int32)
+    k_src, v_src = r(B, H, cap, D), r(B, H, cap, D)
+    k_scale = (np.abs(k_src).max(axis=(0, 2, 3)) / 448.0 * rng.uniform(1.0, 1.5, H)).astype(np.float32)
+    v_scale = (np.abs(v_src).max(axis=(0, 2, 3)) / 448.0 * rng.uniform(1.0, 1.5, H)).astype(np.float32)
+    q, kt, vt = r(B, H, D), r(B, H, D), r(B, H, D)
+    keep = (np.arange(B) % 2 == 0).astype(np.uint8)
+    ln = torch.from_numpy(lens).to(DEV)
+    kc = torch.zeros(B, H, cap, D, dtype=torch.uint8, device=DEV)
+    vc = torch.zeros(B, H, cap, D, dtype=torch.uint8, device=DEV)
+    ks_d, vs_d = torch.from_numpy(k_scale).to(DEV), torch.from_numpy(v_scale).to(DEV)
+    ctx.quantize_kv_fp8(wl.to_torch(k_src, "bf16", DEV), ln, ks_d, kc)
+    ctx.quantize_kv_fp8(wl.to_torch(v_src, "bf16", DEV), ln, vs_d, vc)
+    # rows past the lengths hold bytes that decode to NaN: they must never reach a result
+    for b in range(B):
+        kc[b, :, lens[b]:] = 0x7F
+        vc[b, :, lens[b]:] = 0xFF
+    o_k = f8.quantize_rows(k_src, k_scale[None, :, None, None])
+    o_v = f8.quantize_rows(v_src, v_scale[None, :, None, None])
+    scale = 1.0 / np.sqrt(D)
+    out = torch.zeros(B, H, D, dtype=torch.bfloat16, device=DEV)
+    ctx.sparse_attn_decode_fp8(wl.to_torch(q, "bf16", DEV), wl.to_torch(kt, "bf16", DEV), wl.to_torch(vt, "bf16", DEV),
+                               kc, vc, ks_d, vs_d, ln, torch.from_numpy(keep).to(DEV), scale, out)
+    got = wl.from_torch(out)
+    gk, gv = kc.cpu().numpy(), vc.cpu().numpy()
+    ref = np.empty((B, H, D))
+    plain = np.empty((B, H, D))
+    for b in range(B):
+        n = int(lens[b])
+        for h in range(H):
+            ref[b, h] = f8.attention_decode_fp8(q[b, h], kt[b, h], vt[b, h], o_k[b, h], o_v[b, h], k_scale[h], v_scale[h], n, scale)
+            plain[b, h] = orc.attention_decode_compact(q[b, h], kt[b, h], vt[b, h], k_src[b, h].astype(np.float64),
+                                                       v_src[b, h].astype(np.float64), n, scale)
+            # the cache below the length is untouched; a kept token's row is the oracle's bytes
+            assert np.array_equal(gk[b, h, :n], o_k[b, h, :n]) and np.array_equal(gv[b, h, :n], o_v[b, h, :n])
+            if keep[b] and n < cap:
+                assert np.array_equal(gk[b, h, n], f8.quantize_rows(kt[b, h], k_scale[h])), f"appended K row {b},{h}"
+                assert np.array_equal(gv[b, h, n], f8.quantize_rows(vt[b, h], v_scale[h])), f"appended V row {b},{h}"
+            elif n < cap:
+                assert np.all(gk[b, h, n] == 0x7F) and np.all(gv[b, h, n] == 0xFF)
+    check_att(got, ref, "fp8 decode attention against the oracle on the same bytes")
+    mx, rl = att_errors(got, plain)
+    print(f"cost of quantisation against the unquantised oracle: max-abs {mx:.3e}, relative L2 {rl:.3e}")
+    assert ctx.device_status()[0] == 0
+    ctx.close()
+
+
+def test_full_cache_is_left_untouched_and_reported():
+    B, H, cap = 2, 2, 64
+    dl, ctx, rng, r, D = _setup(B, H, cap, 3)
+    lens = torch.tensor([cap, 10], dtype=torch.int32, device=DEV)
+    kc = torch.full((B, H, cap, D), 0x38, dtype=torch.uint8, device=DEV)
+    vc = torch.full((B, H, cap, D), 0x38, dtype=torch.uint8, device=DEV)
+    one = torch.ones(H, dtype=torch.float32, device=DEV)
+    t = lambda x: wl.to_torch(x, "bf16", DEV)
+    out = torch.zeros(B, H, D, dtype=torch.bfloat16, device=DEV)
+    before = kc.clone()
+    ctx.sparse_attn_decode_fp8(t(r(B, H, D)), t(r(B, H, D)), t(r(B, H, D)), kc, vc, one, one, lens,
+                               torch.ones(B, dtype=torch.uint8, device=DEV), 0.1, out)
+    torch.cuda.synchronize()
+    assert torch.equal(kc[0], before[0])
+    code, detail = ctx.device_status()
+    assert code == dl.DL_ERR_CAPACITY and detail == 0
+    ctx.close()
