@@ -109,3 +109,45 @@ def test_full_cache_is_left_untouched_and_reported():
     code, detail = ctx.device_status()
     assert code == dl.DL_ERR_CAPACITY and detail == 0
     ctx.close()
+
+
+def test_full_size_launch_on_sampled_heads():
+    """The launch bench.py times (`--micro decode_fp8`, config 3: B = 32, H = 32, cap 1344, lengths 784 +- 16, every
+    sequence kept), checked on sampled (sequence, head) pairs the oracle recomputes one by one, plus what holds at
+    any size: bytes below the lengths untouched, appended rows equal to the oracle's bytes."""
+    from paper_2412_00876_b200 import binding as dl
+    cfg = wl.CONFIGS[3]
+    B, H, D, cap = cfg.B, cfg.n_heads, cfg.head_dim, cfg.cap
+    g = torch.Generator(device=DEV).manual_seed(33)
+    mk = lambda: (torch.randint(0, 0x7E, (B, H, cap, D), dtype=torch.uint8, device=DEV, generator=g) |
+                  (torch.randint(0, 2, (B, H, cap, D), dtype=torch.uint8, device=DEV, generator=g) << 7))
+    kc, vc = mk(), mk()
+    k0, v0 = kc.clone(), vc.clone()
+    rng = np.random.default_rng(4)
+    lens = np.clip(784 + rng.integers(-16, 17, B), 0, cap - 1).astype(np.int32)
+    ks = rng.uniform(1 / 96, 1 / 48, H).astype(np.float32)
+    vs = rng.uniform(1 / 96, 1 / 48, H).astype(np.float32)
+    r = lambda *shape: wl.round_to_storage(rng.normal(0, 1, shape).astype(np.float32), "bf16")
+    q, kt, vt = r(B, H, D), r(B, H, D), r(B, H, D)
+    t = lambda x: wl.to_torch(x, "bf16", DEV)
+    ctx = dl.Context(cfg.hidden, H, D, cfg.pred_hidden, torch.bfloat16, 0, max_batch=B, max_rows=B, cap=cap)
+    out = torch.zeros(B, H, D, dtype=torch.bfloat16, device=DEV)
+    scale = 1.0 / np.sqrt(D)
+    ctx.sparse_attn_decode_fp8(t(q), t(kt), t(vt), kc, vc, torch.from_numpy(ks).to(DEV), torch.from_numpy(vs).to(DEV),
+                               torch.from_numpy(lens).to(DEV), torch.ones(B, dtype=torch.uint8, device=DEV), scale, out)
+    got = wl.from_torch(out)
+    pairs = [(0, 0), (B - 1, H - 1)] + [(int(rng.integers(0, B)), int(rng.integers(0, H))) for _ in range(14)]
+    for b, h in pairs:
+        n = int(lens[b])
+        ck, cv = k0[b, h].cpu().numpy(), v0[b, h].cpu().numpy()
+        ref = f8.attention_decode_fp8(q[b, h], kt[b, h], vt[b, h], ck, cv, ks[h], vs[h], n, scale)
+        check_att(got[b, h][None], ref[None], f"fp8 decode attention, full size, b={b} h={h}")
+        assert np.array_equal(kc[b, h, n].cpu().numpy(), f8.quantize_rows(kt[b, h], ks[h]))
+        assert np.array_equal(vc[b, h, n].cpu().numpy(), f8.quantize_rows(vt[b, h], vs[h]))
+    # nothing but row lens[b] of each (b, h) has changed
+    rows = torch.arange(cap, device=DEV)[None, None, :, None]
+    untouched = rows != torch.from_numpy(lens).to(DEV).long()[:, None, None, None]
+    assert torch.equal(torch.where(untouched, kc, 0), torch.where(untouched, k0, 0))
+    assert torch.equal(torch.where(untouched, vc, 0), torch.where(untouched, v0, 0))
+    assert ctx.device_status()[0] == 0
+    ctx.close()
