@@ -180,6 +180,11 @@ class BatchRunner:
         self.h_x_dec, self.h_q_dec = pin(self.x_dec), pin(self.q_dec)
         self.h_k_dec, self.h_v_dec = pin(self.k_dec), pin(self.v_dec)
         self.h_prefill_out = torch.empty_like(self.prefill_out, device="cpu").pin_memory()
+        # the host-fed prefill copies a layer's output out on a side stream while the next layer runs: two device buffers
+        self.prefill_out2 = [self.prefill_out, torch.empty_like(self.prefill_out)]
+        self.out_stream = torch.cuda.Stream(device=self.prefill_out.device)
+        self.out_done = [torch.cuda.Event(), torch.cuda.Event()]
+        self.out_ready = [torch.cuda.Event(), torch.cuda.Event()]
         self.h_dec_out = torch.empty_like(self.dec_out, device="cpu").pin_memory()
         self.h_keep = torch.empty(self.cfg.B, dtype=torch.uint8).pin_memory()
         # two staging sets each: the pipelined host-fed decode copies step t+1 in while step t computes
@@ -214,15 +219,23 @@ class BatchRunner:
             h2d += kept_bytes
             ctx.compact_kv_host(self.h_q_src[i], None, self.keep_vis, self.t_src, self.q_cache, None, self.q_len,
                                 commit=False)
-            ctx.sparse_attn_prefill(self.q_cache, self.k_cache[l], self.v_cache[l], self.cache_len, c.n0, self.scale,
-                                    self.prefill_out)
-            self.h_prefill_out.copy_(self.prefill_out, non_blocking=True)
-            d2h += self.prefill_out.numel() * self.prefill_out.element_size()
+            buf = self.prefill_out2[l & 1]
+            main = torch.cuda.current_stream()
+            if l >= 2:
+                main.wait_event(self.out_done[l & 1])          # the copy out of this buffer, two layers ago
+            ctx.sparse_attn_prefill(self.q_cache, self.k_cache[l], self.v_cache[l], self.cache_len, c.n0, self.scale, buf)
+            self.out_ready[l & 1].record(main)
+            with torch.cuda.stream(self.out_stream):
+                self.out_stream.wait_event(self.out_ready[l & 1])
+                self.h_prefill_out.copy_(buf, non_blocking=True)
+                self.out_done[l & 1].record(self.out_stream)
+            d2h += buf.numel() * buf.element_size()
+        torch.cuda.current_stream().wait_stream(self.out_stream)
         per_step_in = (self.s_x[0].numel() + 3 * self.s_q[0].numel()) * self.s_x.element_size()
         per_step_out = self.dec_out.numel() * self.dec_out.element_size() + c.B
         # the decode steps as one pipelined host-fed call per chunk of steps (results land in two host
         # buffers in turn: a consumer would read step t's while step t+1 computes)
-        chunk = 64
+        chunk = 256
         for t0 in range(0, c.n_gen, chunk):
             steps = range(t0, min(c.n_gen, t0 + chunk))
             pool = [t % self.step_pool for t in steps]
