@@ -386,14 +386,14 @@ class ClockSampler:
 # ------------------------------------------------------------------------------ CPU oracle leg
 def oracle_sample(cfg, budget_s: float = 20.0):
     """Times the oracle, as it stands, on a bounded sample of the workload and extrapolates to the
-    whole batch: prefill select for 2 sequences; compaction, prefill attention (4 heads) for one
-    layer of 2 sequences; decode attention + append for one layer, 2 sequences, all heads at three
-    cache lengths.  Returns (tokens/s, cores, sample description)."""
+    whole batch: prefill select for 8 sequences; compaction, prefill attention (16 heads) for one
+    layer of those sequences; decode attention + append for one layer, all heads at three cache
+    lengths, three times over (about 10 s of CPU work).  Returns (tokens/s, cores, sample description)."""
     import numpy as np
     from oracle import dl_oracle as orc
     from paper_2412_00876_b200 import workloads as wl
     t_all, cpu_all = time.perf_counter(), time.process_time()
-    Bs, H, D = min(2, cfg.B), cfg.n_heads, cfg.head_dim
+    Bs, H, D = min(8, cfg.B), cfg.n_heads, cfg.head_dim
     sc = cfg.scaled(B=Bs)
     scale = 1 / np.sqrt(D)
     p_img, p_txt = wl.make_predictor(cfg, "img"), wl.make_predictor(cfg, "txt")
@@ -413,7 +413,7 @@ def oracle_sample(cfg, budget_s: float = 20.0):
     t0 = time.perf_counter()
     orc.append_rows(ks, vs, mask, None, kc, vc, ln)
     t_compact = (time.perf_counter() - t0) / Bs * 1.5               # K, V and Q: 3 tensors vs the 2 timed
-    hs = min(4, H)
+    hs = min(16, H)
     t0 = time.perf_counter()
     for b in range(Bs):
         for h in range(hs):
@@ -429,14 +429,15 @@ def oracle_sample(cfg, budget_s: float = 20.0):
     kc = wl.host_normal(sc, wl.S_CACHE_K, (Bs, H, cfg.cap, D))
     vc = wl.host_normal(sc, wl.S_CACHE_V, (Bs, H, cfg.cap, D))
     q = wl.host_normal(sc, wl.S_DEC_Q, (Bs, H, D))
-    t_dec = []
+    t_dec, reps = [], 3
     for n in lens:
         t0 = time.perf_counter()
-        for b in range(Bs):
-            for h in range(H):
-                orc.attention_decode_compact(q[b, h], q[b, h], q[b, h], kc[b, h], vc[b, h], n, scale)
-        orc.append_rows(q[:, None], q[:, None], np.ones((Bs, 1), np.uint8), None, kc, vc, np.full(Bs, n, np.int32))
-        t_dec.append((time.perf_counter() - t0) / Bs)               # per sequence per layer per step
+        for _ in range(reps):
+            for b in range(Bs):
+                for h in range(H):
+                    orc.attention_decode_compact(q[b, h], q[b, h], q[b, h], kc[b, h], vc[b, h], n, scale)
+            orc.append_rows(q[:, None], q[:, None], np.ones((Bs, 1), np.uint8), None, kc, vc, np.full(Bs, n, np.int32))
+        t_dec.append((time.perf_counter() - t0) / (Bs * reps))      # per sequence per layer per step
     # whole batch: prefill once, then n_gen steps whose attention time grows linearly with the length
     L, B = cfg.n_layers, cfg.B
     t_prefill = B * (t_select + L * (t_compact + t_pattn))
@@ -451,7 +452,7 @@ def oracle_sample(cfg, budget_s: float = 20.0):
     wall = time.perf_counter() - t_all
     cores = max(1, int(round((time.process_time() - cpu_all) / max(wall, 1e-9))))
     sample = (f"{Bs} sequences: prefill select; 1 layer compaction; prefill attention {hs}/{H} heads; decode "
-              f"attention+append 1 layer, all heads at cache lengths {lens}; extrapolated linearly to "
+              f"attention+append 1 layer, all heads at cache lengths {lens}, {reps} times; extrapolated linearly to "
               f"B={B}, L={L}, {cfg.n_gen} decode steps (sample took {wall:.1f} s on "
               f"{len(os.sched_getaffinity(0))} available host cores)")
     return B * cfg.n_gen / total, cores, sample
