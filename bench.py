@@ -384,16 +384,17 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------ CPU oracle leg
-def oracle_sample(cfg, budget_s: float = 20.0):
+def oracle_sample(cfg, small: bool = False):
     """Times the oracle, as it stands, on a bounded sample of the workload and extrapolates to the
     whole batch: prefill select for 8 sequences; compaction, prefill attention (16 heads) for one
     layer of those sequences; decode attention + append for one layer, all heads at three cache
-    lengths, three times over (about 10 s of CPU work).  Returns (tokens/s, cores, sample description)."""
+    lengths, three times over (about 10 s of CPU work); `small`: 2 sequences, 4 heads, one pass (about 1 s), for
+    runs that time many steps.  Returns (tokens/s, cores, sample description)."""
     import numpy as np
     from oracle import dl_oracle as orc
     from paper_2412_00876_b200 import workloads as wl
     t_all, cpu_all = time.perf_counter(), time.process_time()
-    Bs, H, D = min(8, cfg.B), cfg.n_heads, cfg.head_dim
+    Bs, H, D = min(2 if small else 8, cfg.B), cfg.n_heads, cfg.head_dim
     sc = cfg.scaled(B=Bs)
     scale = 1 / np.sqrt(D)
     p_img, p_txt = wl.make_predictor(cfg, "img"), wl.make_predictor(cfg, "txt")
@@ -413,7 +414,7 @@ def oracle_sample(cfg, budget_s: float = 20.0):
     t0 = time.perf_counter()
     orc.append_rows(ks, vs, mask, None, kc, vc, ln)
     t_compact = (time.perf_counter() - t0) / Bs * 1.5               # K, V and Q: 3 tensors vs the 2 timed
-    hs = min(16, H)
+    hs = min(4 if small else 16, H)
     t0 = time.perf_counter()
     for b in range(Bs):
         for h in range(hs):
@@ -429,7 +430,7 @@ def oracle_sample(cfg, budget_s: float = 20.0):
     kc = wl.host_normal(sc, wl.S_CACHE_K, (Bs, H, cfg.cap, D))
     vc = wl.host_normal(sc, wl.S_CACHE_V, (Bs, H, cfg.cap, D))
     q = wl.host_normal(sc, wl.S_DEC_Q, (Bs, H, D))
-    t_dec, reps = [], 3
+    t_dec, reps = [], (1 if small else 3)
     for n in lens:
         t0 = time.perf_counter()
         for _ in range(reps):
@@ -474,9 +475,10 @@ def reference_arm(args):
         return
     cfg = wl.CONFIGS[args.config]
     vals, sample, cores = [], "", 1
+    small = args.warmup + args.steps > 6          # many steps: a smaller sample per step keeps the run within minutes
     for i in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        v, cores, sample = oracle_sample(cfg)
+        v, cores, sample = oracle_sample(cfg, small=small)
         if i >= args.warmup:
             vals.append((v, time.perf_counter() - t0))
         if i == 0 and (time.perf_counter() - t0) * (args.warmup + args.steps) > 240:
