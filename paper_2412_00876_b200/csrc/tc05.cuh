@@ -1,6 +1,6 @@
 // Blackwell (sm_100a) tensor-core plumbing in inline PTX: tensor memory allocation, shared-memory
-// matrix descriptors, tcgen05.mma / commit / ld, and TMA tile loads.  cta_group::1 only; no
-// multicast anywhere.
+// matrix descriptors, tcgen05.mma / commit / ld, and TMA tile loads.  cta_group::1 only; every
+// copy has one destination CTA.
 #pragma once
 
 #include <cuda.h>
@@ -135,7 +135,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// ---- TMA tile loads (no multicast) ----------------------------------------------------------------
+// ---- TMA tile loads (one destination CTA each) ------------------------------------------------------
 // x is the innermost (contiguous) coordinate in elements: x * element size must be a multiple of 16.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
