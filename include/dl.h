@@ -46,6 +46,7 @@ enum {
   DL_ERR_CUDA = -5,          /* a CUDA runtime call failed (see dl_last_cuda_error) */
   DL_ERR_CAPACITY = -6,      /* device status: kept rows did not fit into the cache */
   DL_ERR_TIMEOUT = -7,       /* device status: a bounded wait ran out */
+  DL_ERR_BOUNDS = -8,        /* device status (checked build only): an index fell outside its buffer; the access was skipped */
   DL_WARN_NAN = 1            /* device status: a NaN score was ranked as -inf / dropped */
 };
 
@@ -377,6 +378,22 @@ int32_t dl_sparse_attn_decode_fp8(dl_ctx* ctx, const void* q_t, const void* k_t,
                                   void* v_cache, const float* k_scale, const float* v_scale,
                                   const int32_t* cache_len, const uint8_t* keep, int32_t B, int32_t cap, float scale,
                                   void* out, void* stream);
+
+/* ---- checked build ---------------------------------------------------------------------- */
+
+/* The library can be built with -DDL_BOUNDS=1 (libdl_sparse_checked.so): every store a kernel makes through an
+ * index it computed (cache rows, outputs, partial sums, masks, index lists) is then compared with the extent of its
+ * buffer first; an index outside it is NOT used: the store is skipped and DL_ERR_BOUNDS is recorded in the status
+ * word with detail = (kernel id << 48) | index.  Nothing traps.  Copies made by the TMA unit are clipped by their
+ * tensor maps in either build.  Results are the same as the normal build's; it is slower. */
+
+/* 1 in the checked build, 0 otherwise. */
+int32_t dl_build_is_checked(void);
+
+/* Makes one checked store with an index one past the end of a small buffer inside the workspace.  Checked build:
+ * the store is skipped, the buffer unchanged, DL_ERR_BOUNDS recorded (kernel id 0x7e, index 64); normal build:
+ * DL_ERR_UNSUPPORTED, nothing launched.  Asynchronous on `stream`; needs the workspace. */
+int32_t dl_selftest_bounds(dl_ctx* ctx, void* stream);
 
 /* ---- decode attention without any allocation ------------------------------------------- */
 

@@ -12,12 +12,16 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdl_sparse.so")
+# DL_SPARSE_CHECKED=1 in the environment selects the checked twin (stores through computed indices are compared with
+# their buffers first; see include/dl.h)
+LIB_PATH = os.path.join(_HERE, "libdl_sparse_checked.so" if os.environ.get("DL_SPARSE_CHECKED") == "1"
+                        else "libdl_sparse.so")
 
 DL_F32, DL_BF16 = 0, 1
 DL_OK = 0
 DL_ERR_INVALID_ARG, DL_ERR_ALIGNMENT, DL_ERR_UNSUPPORTED, DL_ERR_WORKSPACE = -1, -2, -3, -4
 DL_ERR_CUDA, DL_ERR_CAPACITY, DL_ERR_TIMEOUT, DL_WARN_NAN = -5, -6, -7, 1
+DL_ERR_BOUNDS = -8
 DL_OPT_PREDICTOR_IMPL, DL_OPT_PREFILL_ATTN_IMPL, DL_OPT_DECODE_CHUNK, DL_OPT_DECODE_IMPL = 1, 2, 3, 4
 DL_OPT_COMPACT_IMPL = 5
 
@@ -29,7 +33,8 @@ EXPORTS = [
     "dl_sparse_attn_decode_static", "dl_sparse_attn_decode_layers", "dl_decode_nocache_select",
     "dl_decode_steps_host", "dl_compact_kv_host", "dl_selftest_wait_timeout", "dl_compact_kv_layers",
     "dl_predictor2_scratch_bytes", "dl_predictor2_values", "dl_prefill_select2", "dl_decode_keep2",
-    "dl_decode_step_stack", "dl_quantize_kv_fp8", "dl_sparse_attn_decode_fp8",
+    "dl_decode_step_stack", "dl_quantize_kv_fp8", "dl_sparse_attn_decode_fp8", "dl_build_is_checked",
+    "dl_selftest_bounds",
 ]
 
 
@@ -129,6 +134,8 @@ def lib() -> C.CDLL:
                                      C.POINTER(vp), i32, vp, f32, vp, vp]),
             "dl_decode_step_stack": (i32, [vp, P, vp, i32, f32, vp, vp, C.POINTER(LayerStackDesc), vp, vp, vp, f32,
                                            vp, vp]),
+            "dl_build_is_checked": (i32, []),
+            "dl_selftest_bounds": (i32, [vp, vp]),
             "dl_quantize_kv_fp8": (i32, [vp, vp, vp, vp, i32, i32, vp, vp]),
             "dl_sparse_attn_decode_fp8": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp]),
             "dl_decode_step_host": (i32, [vp, P, vp, i32, f32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
@@ -287,6 +294,10 @@ class Context:
         self._check(lib().dl_sparse_attn_decode(self._h, _ptr(q_t), _ptr(k_t), _ptr(v_t), _ptr(k_cache),
                                                 _ptr(v_cache), _ptr(cache_len), _ptr(keep), B, cap, float(scale),
                                                 _ptr(out), _stream(stream)), "dl_sparse_attn_decode")
+
+    def selftest_bounds(self, stream=None):
+        """Checked build: one store a word past a buffer's end, which must be skipped and recorded."""
+        return lib().dl_selftest_bounds(self._h, _stream(stream))
 
     def quantize_kv_fp8(self, src, cache_len, scale, dst, stream=None):
         """Extension (not in the paper): rows of a bf16 cache as E4M3 bytes under per-head scales."""

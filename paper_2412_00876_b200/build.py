@@ -1,4 +1,5 @@
-"""Builds the CUDA library in-tree: csrc/*.cu -> libdl_sparse.so (sm_100a only).
+"""Builds the CUDA library in-tree: csrc/*.cu -> libdl_sparse.so (sm_100a only), and its checked twin
+libdl_sparse_checked.so (-DDL_BOUNDS=1: stores through computed indices are compared with their buffers first).
 
 Usage:  python -m paper_2412_00876_b200.build [--force] [--verbose]
 """
@@ -13,19 +14,19 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdl_sparse.so")
+LIB_CHECKED = os.path.join(HERE, "libdl_sparse_checked.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
-STAMP = LIB + ".src_hash"
 
 
 def _sources():
     return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cu"))
 
 
-def source_hash() -> str:
+def source_hash(extra_flags=()) -> str:
     """SHA-256 over every file the library is built from (sources, headers, the C header) and the flags."""
     import hashlib
-    h = hashlib.sha256(" ".join(FLAGS).encode())
+    h = hashlib.sha256(" ".join([*FLAGS, *extra_flags]).encode())
     paths = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC))
     paths.append(os.path.join(os.path.dirname(HERE), "include", "dl.h"))
     for p in paths:
@@ -34,14 +35,19 @@ def source_hash() -> str:
     return h.hexdigest()
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Builds the library unless the one in place was built from exactly these sources: the decision is taken on
-    a hash of the sources stored beside the library, not on file times (a snapshot copied elsewhere keeps neither)."""
-    want = source_hash()
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Builds the library (or its checked twin) unless the one in place was built from exactly these sources: the
+    decision is taken on a hash of the sources stored beside the library, not on file times (a snapshot copied
+    elsewhere keeps neither)."""
+    variant = ["-DDL_BOUNDS=1"] if checked else []
+    LIB = LIB_CHECKED if checked else globals()["LIB"]
+    OBJ = globals()["OBJ"] + ("_checked" if checked else "")
+    STAMP = LIB + ".src_hash"
+    want = source_hash(variant)
     if not force and os.path.exists(LIB) and os.path.exists(STAMP) and open(STAMP).read().strip() == want:
         return LIB
     os.makedirs(OBJ, exist_ok=True)
-    extra = ["-Xptxas", "-v"] if verbose else []
+    extra = variant + (["-Xptxas", "-v"] if verbose else [])
 
     def compile_one(src):
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
@@ -64,5 +70,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_all(force: bool = False, verbose: bool = False):
+    return build(force, verbose), build(force, verbose, checked=True)
+
+
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(*build_all(force="--force" in sys.argv, verbose="--verbose" in sys.argv))

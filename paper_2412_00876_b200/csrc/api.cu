@@ -199,6 +199,7 @@ const char* dl_status_str(int32_t status) {
     case DL_ERR_CUDA: return "CUDA runtime error";
     case DL_ERR_CAPACITY: return "kept rows do not fit into the cache";
     case DL_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case DL_ERR_BOUNDS: return "checked build: an index fell outside its buffer (access skipped)";
     case DL_WARN_NAN: return "NaN score ranked as -inf / dropped";
     default: return "unknown status";
   }

@@ -599,8 +599,10 @@ attn_decode_mma_kernel(const __grid_constant__ TmapPair maps, const DecodeArgs a
     if (I.c == 0 && a.keep != nullptr && a.keep[I.b] != 0) {
       if (I.n_b < a.cap) {
         const size_t dst = (bh * a.cap + I.n_b) * RB + lane * 8;
-        *reinterpret_cast<uint2*>((char*)a.k_cache + dst) = nks;
-        *reinterpret_cast<uint2*>((char*)a.v_cache + dst) = nvs;
+        if (DL_IN_BOUNDS(a.status, KID_DECODE_MMA, dst + 7, (size_t)a.B * a.H * a.cap * RB)) {
+          *reinterpret_cast<uint2*>((char*)a.k_cache + dst) = nks;
+          *reinterpret_cast<uint2*>((char*)a.v_cache + dst) = nvs;
+        }
       } else if (lane == 0 && I.h == 0) {
         report_status(a.status, DL_ERR_CAPACITY, I.b);
       }
@@ -690,7 +692,7 @@ attn_decode_mma_kernel(const __grid_constant__ TmapPair maps, const DecodeArgs a
       const float wc = (m_run == -INFINITY) ? 0.f : exp2f(m_run - M2);
       const float we = exp2f(s_e - M2);
       const float inv = 1.f / (l_run * wc + we);
-      if (row0_lane) {
+      if (row0_lane && DL_IN_BOUNDS(a.status, KID_DECODE_MMA, bh * RB + RB - 1, (size_t)a.B * a.H * RB)) {
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
           const uint32_t vw = __ldg(vtw + i * 4 + t4);
@@ -701,7 +703,8 @@ attn_decode_mma_kernel(const __grid_constant__ TmapPair maps, const DecodeArgs a
       continue;
     }
     float* part = a.partial + (bh * a.slots + I.c) * (size_t)(D + 2);
-    if (row0_lane) {
+    if (row0_lane && DL_IN_BOUNDS(a.status, KID_DECODE_MMA, (bh * a.slots + I.c) * (size_t)(D + 2) + D + 1,
+                                  (size_t)a.B * a.H * a.slots * (D + 2))) {
 #pragma unroll
       for (int i = 0; i < 16; ++i) *reinterpret_cast<float2*>(part + i * 8 + 2 * t4) = make_float2(acc[i][0], acc[i][1]);
     }

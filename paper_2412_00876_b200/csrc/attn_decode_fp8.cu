@@ -232,8 +232,10 @@ attn_decode_fp8_kernel(const __grid_constant__ F8Maps maps, const F8Args a) {
                             (f8_encode_pair(__fdiv_rn(bf16lo(nks.y), ksc), __fdiv_rn(bf16hi(nks.y), ksc)) << 16);
         const uint32_t vb = f8_encode_pair(__fdiv_rn(bf16lo(nvs.x), v_scale), __fdiv_rn(bf16hi(nvs.x), v_scale)) |
                             (f8_encode_pair(__fdiv_rn(bf16lo(nvs.y), v_scale), __fdiv_rn(bf16hi(nvs.y), v_scale)) << 16);
-        *reinterpret_cast<uint32_t*>(a.k_cache + dst) = kb;
-        *reinterpret_cast<uint32_t*>(a.v_cache + dst) = vb;
+        if (DL_IN_BOUNDS(a.status, KID_DECODE_FP8, dst + 3, (size_t)a.B * a.H * a.cap * 128)) {
+          *reinterpret_cast<uint32_t*>(a.k_cache + dst) = kb;
+          *reinterpret_cast<uint32_t*>(a.v_cache + dst) = vb;
+        }
       } else if (lane == 0 && I.h == 0) {
         report_status(a.status, DL_ERR_CAPACITY, I.b);
       }
@@ -342,7 +344,7 @@ attn_decode_fp8_kernel(const __grid_constant__ F8Maps maps, const F8Args a) {
       const float we = exp2f(s_e - M2);
       const float inv = 1.f / (l_run * wn + we);
       const float wc = wn * v_scale;
-      if (row0_lane) {
+      if (row0_lane && DL_IN_BOUNDS(a.status, KID_DECODE_FP8, bh * RB + RB - 1, (size_t)a.B * a.H * RB)) {
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           const uint2 vw = __ldg(reinterpret_cast<const uint2*>(vtb + (16 * c + 4 * t4) * 2));
@@ -429,7 +431,7 @@ attn_decode_fp8_kernel(const __grid_constant__ F8Maps maps, const F8Args a) {
 // nearest code (ties to even), clamped to +-448.  One thread per 8 elements.
 __global__ void quantize_kv_fp8_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ cache_len,
                                        const float* __restrict__ scale, int32_t H, int32_t cap, long long n8,
-                                       uint2* __restrict__ dst) {
+                                       uint2* __restrict__ dst, DeviceStatus* st) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n8) return;
   const long long row = i >> 4;                     // 16 groups of 8 per 128-dim row
@@ -444,7 +446,7 @@ __global__ void quantize_kv_fp8_kernel(const uint4* __restrict__ src, const int3
         (f8_encode_pair(__fdiv_rn(bf16lo(v.y), sc), __fdiv_rn(bf16hi(v.y), sc)) << 16);
   o.y = f8_encode_pair(__fdiv_rn(bf16lo(v.z), sc), __fdiv_rn(bf16hi(v.z), sc)) |
         (f8_encode_pair(__fdiv_rn(bf16lo(v.w), sc), __fdiv_rn(bf16hi(v.w), sc)) << 16);
-  dst[i] = o;
+  if (DL_IN_BOUNDS(st, KID_QUANTIZE, i, n8)) dst[i] = o;
 }
 
 cudaError_t launch_quantize_kv_fp8(const dl_ctx* ctx, const void* src, const int32_t* cache_len, const float* scale,
@@ -454,7 +456,8 @@ cudaError_t launch_quantize_kv_fp8(const dl_ctx* ctx, const void* src, const int
   const long long blocks = (n8 + 255) / 256;
   if (blocks >= (1LL << 31)) return cudaErrorInvalidValue;
   quantize_kv_fp8_kernel<<<(unsigned)blocks, 256, 0, s>>>(static_cast<const uint4*>(src), cache_len, scale,
-                                                           ctx->desc.n_heads, cap, n8, static_cast<uint2*>(dst));
+                                                           ctx->desc.n_heads, cap, n8, static_cast<uint2*>(dst),
+                                                           ctx->ws.base ? ctx->ws.status : nullptr);
   return cudaGetLastError();
 }
 

@@ -14,7 +14,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kPfWarps * 32)
 attn_prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc,
                          const int32_t* __restrict__ cache_len, int32_t H, int32_t cap, int32_t n_max,
-                         float scale_log2, T* __restrict__ out) {
+                         float scale_log2, T* __restrict__ out, DeviceStatus* st) {
   __shared__ float Kt[D][33];
   __shared__ float Vs[32][D];
   __shared__ float Qs[kPfWarps][D];
@@ -68,7 +68,8 @@ attn_prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ kc, cons
       for (int c = 0; c < D / 32; ++c) acc[c] = fmaf(pj, Vs[j][lane + 32 * c], acc[c]);
     }
   }
-  if (row_ok) {
+  if (row_ok && DL_IN_BOUNDS(st, KID_PREFILL_SIMT, (((size_t)b * n_max + i) * H + h) * D + D - 1,
+                             (size_t)gridDim.z * n_max * H * D)) {
     const float inv = 1.f / l_run;
     T* o = out + (((size_t)b * n_max + i) * H + h) * D;
 #pragma unroll
@@ -86,7 +87,8 @@ cudaError_t launch_attn_prefill_simt(const dl_ctx* ctx, const void* q, const voi
 #define DL_LAUNCH(T, DD)                                                                              \
   attn_prefill_simt_kernel<T, DD><<<grid, kPfWarps * 32, 0, s>>>((const T*)q, (const T*)k_cache,       \
                                                                  (const T*)v_cache, cache_len, d.n_heads, \
-                                                                 cap, n_max, sl, (T*)out)
+                                                                 cap, n_max, sl, (T*)out,                        \
+                                                                 ctx->ws.base ? ctx->ws.status : nullptr)
   if (d.dtype == DL_BF16) {
     if (d.head_dim == 128) DL_LAUNCH(__nv_bfloat16, 128);
     else if (d.head_dim == 64) DL_LAUNCH(__nv_bfloat16, 64);

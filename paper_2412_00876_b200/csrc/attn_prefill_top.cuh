@@ -86,6 +86,9 @@ static __device__ __forceinline__ void at_top_rows(const AtArgs& a, const AtItem
     for (int hf = 0; hf < 2; ++hf) {
       const int r = g + 8 * hf;
       if (r >= s) continue;
+      if (!DL_IN_BOUNDS(a.status, KID_PREFILL_TOP, (((size_t)I.b * a.n_max + r) * a.H + I.h) * 128 + 127,
+                        (size_t)a.B * a.n_max * a.H * 128))
+        continue;
       uint32_t* orow = reinterpret_cast<uint32_t*>(a.out + (((size_t)I.b * a.n_max + r) * a.H + I.h) * 128 + pass * 32 + 2 * t);
 #pragma unroll
       for (int nb = 0; nb < 4; ++nb) orow[nb * 4] = cvt_bf16x2(o[nb][2 * hf] * inv[hf], o[nb][2 * hf + 1] * inv[hf]);

@@ -30,6 +30,24 @@ __device__ __forceinline__ void report_status(DeviceStatus* st, int32_t code, lo
   }
 }
 
+// Checked build (-DDL_BOUNDS=1): DL_IN_BOUNDS(status, kernel id, index, extent) is false for an index outside
+// [0, extent) and records it; the caller skips the access.  In the normal build it is the constant true.
+enum KernelId : int {
+  KID_DECODE_MMA = 1, KID_DECODE_SIMT = 2, KID_DECODE_FP8 = 3, KID_COMPACT_PLAN = 4, KID_COMPACT_COPY = 5,
+  KID_TOPK = 6, KID_KEEP = 7, KID_PREFILL_TOP = 8, KID_PREFILL_SIMT = 9, KID_PREFILL_TC = 10, KID_QUANTIZE = 11,
+  KID_PREDICTOR = 12, KID_SELFTEST = 0x7e
+};
+#ifdef DL_BOUNDS
+__device__ __forceinline__ bool bounds_ok(DeviceStatus* st, int kid, long long idx, long long extent) {
+  if (idx >= 0 && idx < extent) return true;
+  report_status(st, DL_ERR_BOUNDS, ((long long)kid << 48) | (idx & 0xFFFFFFFFFFFFll));
+  return false;
+}
+#define DL_IN_BOUNDS(st, kid, idx, extent) dl::bounds_ok((st), (kid), (long long)(idx), (long long)(extent))
+#else
+#define DL_IN_BOUNDS(st, kid, idx, extent) true
+#endif
+
 // ---------------------------------------------------------------------------------------
 // Workspace layout (all offsets 256-byte aligned).
 // ---------------------------------------------------------------------------------------

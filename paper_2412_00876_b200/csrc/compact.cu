@@ -88,7 +88,7 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
                     const uint8_t* __restrict__ keep, int32_t keep_cols, const int32_t* __restrict__ t_src,
                     int32_t t_max, uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, int32_t cap, int32_t H,
                     int32_t row_units, int32_t piece_units, const int32_t* plan_base,
-                    const int32_t* plan_count, int32_t chained) {
+                    const int32_t* plan_count, int32_t chained, DeviceStatus* st) {
   __shared__ int sh[8];
   __shared__ int tile_tok[kTileTokens];
   __shared__ int tile_kept;
@@ -157,7 +157,8 @@ compact_copy_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v
         int u = u0 + i * 32 + lane;
         if (u < row_units) {
           int h = u / piece_units, o = u - h * piece_units;
-          dst[dst_b + (size_t)h * head_stride + dst_row + o] = r[i];
+          const size_t at = dst_b + (size_t)h * head_stride + dst_row + o;
+          if (DL_IN_BOUNDS(st, KID_COMPACT_COPY, at, (size_t)gridDim.y * H * head_stride)) dst[at] = r[i];
         }
       }
     }
@@ -431,7 +432,7 @@ cudaError_t launch_compact(const dl_ctx* ctx, const void* k_src, const void* v_s
   return cudaLaunchKernelEx(&cfg, compact_copy_kernel, (const uint4*)k_src, (const uint4*)v_src, keep, (int32_t)keep_cols,
                             t_src, (int32_t)t_src_max, (uint4*)k_cache, (uint4*)v_cache, (int32_t)cap, (int32_t)d.n_heads,
                             (int32_t)row_units, (int32_t)piece_units, (const int32_t*)ctx->ws.plan_base,
-                            (const int32_t*)ctx->ws.plan_count, (int32_t)chained);
+                            (const int32_t*)ctx->ws.plan_count, (int32_t)chained, ctx->ws.status);
 }
 
 __global__ void commit_len_kernel(const uint8_t* __restrict__ keep, int32_t B, int32_t cap,

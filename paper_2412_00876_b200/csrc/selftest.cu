@@ -25,7 +25,41 @@ __global__ void wait_timeout_kernel(int polls, DeviceStatus* st) {
   if (threadIdx.x == 0 && !ok && !ok2 && *abort_flag) report_status(st, DL_ERR_TIMEOUT, 0x5e1f);
 }
 
+// One checked store one element past the end of a 64-word buffer: the checked build must skip it and record it.
+__global__ void bounds_selftest_kernel(int32_t* buf, int32_t n, DeviceStatus* st) {
+  const int idx = n;                                    // one past the end
+  if (DL_IN_BOUNDS(st, KID_SELFTEST, idx, n)) buf[idx] = 0x0bad;
+}
+
 }  // namespace dl
+
+extern "C" int32_t dl_build_is_checked(void) {
+#ifdef DL_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+extern "C" int32_t dl_selftest_bounds(dl_ctx* ctx, void* stream) {
+  if (!ctx) return DL_ERR_INVALID_ARG;
+  if (!ctx->ws.base) return DL_ERR_WORKSPACE;
+#ifndef DL_BOUNDS
+  (void)stream;
+  return DL_ERR_UNSUPPORTED;
+#else
+  int prev = -1;
+  cudaGetDevice(&prev);
+  if (prev != ctx->device) cudaSetDevice(ctx->device);
+  // the plan arrays of the workspace (max_batch words each, at least 64 with the padding of the layout) stand in
+  // for "a small buffer"; the kernel is given 64 words of plan_base and must not touch word 64
+  dl::bounds_selftest_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(ctx->ws.plan_base, 64, ctx->ws.status);
+  cudaError_t e = cudaGetLastError();
+  if (prev != ctx->device) cudaSetDevice(prev);
+  if (e != cudaSuccess) { ctx->last_cuda = e; return DL_ERR_CUDA; }
+  return DL_OK;
+#endif
+}
 
 extern "C" int32_t dl_selftest_wait_timeout(dl_ctx* ctx, int32_t polls, void* stream) {
   if (!ctx || polls < 1 || polls > (1 << 16)) return DL_ERR_INVALID_ARG;

@@ -146,8 +146,10 @@ topk_kernel(const float* __restrict__ score, const int32_t* __restrict__ n_vis,
   uint8_t* kp_out = keep + (size_t)b * n_max;
   for (int i = i0; i < min(n_max, i0 + ipt); ++i) {
     bool kp = (kk > 0) && (i < n) && (keys[i] != 0u);
-    kp_out[i] = kp ? 1 : 0;
-    if (kp && kept_idx && out_pos < k_max) kept_idx[(size_t)b * k_max + out_pos] = i;
+    if (DL_IN_BOUNDS(st, KID_TOPK, (size_t)b * n_max + i, (size_t)gridDim.x * n_max)) kp_out[i] = kp ? 1 : 0;
+    if (kp && kept_idx && out_pos < k_max &&
+        DL_IN_BOUNDS(st, KID_TOPK, (size_t)b * k_max + out_pos, (size_t)gridDim.x * k_max))
+      kept_idx[(size_t)b * k_max + out_pos] = i;
     out_pos += kp;
   }
   if (kept_idx)

@@ -25,6 +25,15 @@ def test_header_and_binding_agree_and_symbols_exist():
     assert b"cache" in binding.lib().dl_status_str(binding.DL_ERR_CAPACITY)
 
 
+def test_checked_twin_exports_the_same_and_says_so():
+    """libdl_sparse_checked.so (-DDL_BOUNDS=1) has the same interface; the two tell themselves apart."""
+    from paper_2412_00876_b200 import build
+    normal, checked = ctypes.CDLL(build.build()), ctypes.CDLL(build.build(checked=True))
+    for n in declared_functions():
+        assert hasattr(checked, n), f"{n} missing from the checked build"
+    assert normal.dl_build_is_checked() == 0 and checked.dl_build_is_checked() == 1
+
+
 def test_product_code_never_imports_the_oracle():
     pkg = os.path.join(ROOT, "paper_2412_00876_b200")
     for dirpath, _, files in os.walk(pkg):
