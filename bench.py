@@ -40,7 +40,7 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-record", action="store_true")
     ap.add_argument("--sample-every", type=int, default=64, help="decode steps between timed attention launches")
-    ap.add_argument("--micro", default="", choices=["", "decode", "decode_fp8", "keep", "select2", "keep2", "predictor", "select", "compact", "compact_layers", "prefill", "nocache"],
+    ap.add_argument("--micro", default="", choices=["", "decode", "decode_fp8", "decode_fp8_stack", "keep", "select2", "keep2", "predictor", "select", "compact", "compact_layers", "prefill", "nocache"],
                     help="time one stage alone on the config's shapes (small memory; used for ncu captures)")
     ap.add_argument("--micro-layers", type=int, default=2, help="layers of cache / source held in --micro mode")
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
@@ -95,6 +95,24 @@ def micro(args, emit=True):
         work = (2 * (int(lens.sum()) + B) + 2 * B) * H * D * cfg.elt_bytes
         calls = [lambda l=l: ctx.sparse_attn_decode(q[l], kt[l], vt[l], kc[l], vc[l], ln, keep, scale, out[l])
                  for l in range(NL)]
+    elif args.micro == "decode_fp8_stack":
+        # extension, not in the paper: `micro_layers` layers of byte caches in ONE call (launches overlap); the rate
+        # is per call, i.e. over all layers
+        n = args.micro_len or min(cfg.cap - 1, cfg.n0 + int(cfg.n_gen * cfg.keep_rate))
+        mk = lambda: torch.randint(0, 0x7E, (B, H, cfg.cap, D), dtype=torch.uint8, device=dev)
+        kc, vc = [mk() for _ in range(NL)], [mk() for _ in range(NL)]
+        ksc = torch.full((NL, H), 1.0 / 64, dtype=torch.float32, device=dev)
+        vsc = torch.full((NL, H), 1.0 / 64, dtype=torch.float32, device=dev)
+        q = wl.device_normal(cfg, wl.S_DEC_Q, (NL, B, H, D), dev)
+        kt = wl.device_normal(cfg, wl.S_DEC_K, (NL, B, H, D), dev)
+        vt = wl.device_normal(cfg, wl.S_DEC_V, (NL, B, H, D), dev)
+        out = torch.empty(NL, B, H, D, dtype=tdt, device=dev)
+        lens = np.clip(n + wl.host_rng(cfg.cid, wl.S_LEN).integers(-16, 17, B), 0, cfg.cap - 1).astype(np.int32)
+        ln = torch.from_numpy(lens).to(dev)
+        keep = torch.ones(B, dtype=torch.uint8, device=dev)
+        work = NL * (2 * (int(lens.sum()) + B) * 1 + 4 * B * cfg.elt_bytes) * H * D
+        calls = [lambda: ctx.sparse_attn_decode_fp8_layers(q, kt, vt, kc, vc, ksc, vsc, ln, keep, scale, out)]
+        NL = 1
     elif args.micro == "decode_fp8":
         # extension, not in the paper: the same launch over caches held as E4M3 bytes with per-head scales
         n = args.micro_len or min(cfg.cap - 1, cfg.n0 + int(cfg.n_gen * cfg.keep_rate))

@@ -379,6 +379,15 @@ int32_t dl_sparse_attn_decode_fp8(dl_ctx* ctx, const void* q_t, const void* k_t,
                                   const int32_t* cache_len, const uint8_t* keep, int32_t B, int32_t cap, float scale,
                                   void* out, void* stream);
 
+/* The layer stack of a decode step over 8-bit caches (the counterpart of dl_sparse_attn_decode_layers): L launches
+ * that overlap on the GPU; with commit != 0 the lengths advance once behind the last layer (cache_len[b] += keep[b]).
+ *   q_t, k_t, v_t, out dev [L][B][H][128] bf16; k_caches, v_caches HOST arrays of L dev byte caches [B][H][cap][128];
+ *   k_scales, v_scales dev [L][H] fp32; cache_len dev [B], read by every layer, written only with commit. */
+int32_t dl_sparse_attn_decode_fp8_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
+                                         void* const* k_caches, void* const* v_caches, const float* k_scales,
+                                         const float* v_scales, int32_t* cache_len, const uint8_t* keep, int32_t B,
+                                         int32_t cap, float scale, void* out, int32_t commit, void* stream);
+
 /* ---- checked build ---------------------------------------------------------------------- */
 
 /* The library can be built with -DDL_BOUNDS=1 (libdl_sparse_checked.so): every store a kernel makes through an

@@ -34,7 +34,7 @@ EXPORTS = [
     "dl_decode_steps_host", "dl_compact_kv_host", "dl_selftest_wait_timeout", "dl_compact_kv_layers",
     "dl_predictor2_scratch_bytes", "dl_predictor2_values", "dl_prefill_select2", "dl_decode_keep2",
     "dl_decode_step_stack", "dl_quantize_kv_fp8", "dl_sparse_attn_decode_fp8", "dl_build_is_checked",
-    "dl_selftest_bounds",
+    "dl_selftest_bounds", "dl_sparse_attn_decode_fp8_layers",
 ]
 
 
@@ -134,6 +134,8 @@ def lib() -> C.CDLL:
                                      C.POINTER(vp), i32, vp, f32, vp, vp]),
             "dl_decode_step_stack": (i32, [vp, P, vp, i32, f32, vp, vp, C.POINTER(LayerStackDesc), vp, vp, vp, f32,
                                            vp, vp]),
+            "dl_sparse_attn_decode_fp8_layers": (i32, [vp, i32, vp, vp, vp, C.POINTER(vp), C.POINTER(vp), vp, vp, vp, vp,
+                                                       i32, i32, f32, vp, i32, vp]),
             "dl_build_is_checked": (i32, []),
             "dl_selftest_bounds": (i32, [vp, vp]),
             "dl_quantize_kv_fp8": (i32, [vp, vp, vp, vp, i32, i32, vp, vp]),
@@ -312,6 +314,16 @@ class Context:
                                                     _ptr(v_cache), _ptr(k_scale), _ptr(v_scale), _ptr(cache_len),
                                                     _ptr(keep), B, cap, float(scale), _ptr(out), _stream(stream)),
                     "dl_sparse_attn_decode_fp8")
+
+    def sparse_attn_decode_fp8_layers(self, q_t, k_t, v_t, k_caches, v_caches, k_scales, v_scales, cache_len, keep,
+                                      scale, out, commit=False, stream=None):
+        """k_caches / v_caches: lists of the L layers' byte caches; k_scales / v_scales [L][H]."""
+        L, B, cap = len(k_caches), k_caches[0].shape[0], k_caches[0].shape[2]
+        kp, vp_ = self.pointer_array(k_caches), self.pointer_array(v_caches)
+        self._check(lib().dl_sparse_attn_decode_fp8_layers(
+            self._h, L, _ptr(q_t), _ptr(k_t), _ptr(v_t), kp, vp_, _ptr(k_scales), _ptr(v_scales), _ptr(cache_len),
+            _ptr(keep), B, cap, float(scale), _ptr(out), int(bool(commit)), _stream(stream)),
+            "dl_sparse_attn_decode_fp8_layers")
 
     def sparse_attn_decode_static(self, q_t, k_t, v_t, k_cache, v_cache, cache_len, keep, scale, out, stream=None):
         """dl_sparse_attn_decode for callers that may not allocate device memory: the kernel's scratch

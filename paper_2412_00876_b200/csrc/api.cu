@@ -436,6 +436,41 @@ int32_t dl_sparse_attn_decode_fp8(dl_ctx* ctx, const void* q_t, const void* k_t,
                                                  keep, B, cap, scale, out, static_cast<cudaStream_t>(stream)));
 }
 
+int32_t dl_sparse_attn_decode_fp8_layers(dl_ctx* ctx, int32_t L, const void* q_t, const void* k_t, const void* v_t,
+                                         void* const* k_caches, void* const* v_caches, const float* k_scales,
+                                         const float* v_scales, int32_t* cache_len, const uint8_t* keep, int32_t B,
+                                         int32_t cap, float scale, void* out, int32_t commit, void* stream) {
+  if (!ctx || L < 0 || B < 0 || cap <= 0) return DL_ERR_INVALID_ARG;
+  if (B == 0 || L == 0) return DL_OK;
+  if (!q_t || !k_t || !v_t || !k_caches || !v_caches || !k_scales || !v_scales || !cache_len || !out)
+    return DL_ERR_INVALID_ARG;
+  if (commit && !keep) return DL_ERR_INVALID_ARG;
+  const size_t layer_bytes = (size_t)B * ctx->desc.n_heads * ctx->desc.head_dim * elt_bytes(ctx);
+  for (int32_t l = 0; l < L; ++l) {
+    const char* ql = static_cast<const char*>(q_t) + l * layer_bytes;
+    const char* kl = static_cast<const char*>(k_t) + l * layer_bytes;
+    const char* vl = static_cast<const char*>(v_t) + l * layer_bytes;
+    char* ol = static_cast<char*>(out) + l * layer_bytes;
+    if (!k_caches[l] || !v_caches[l]) return DL_ERR_INVALID_ARG;
+    if (misaligned(ql) || misaligned(k_caches[l]) || misaligned(v_caches[l]) || misaligned(ol)) return DL_ERR_ALIGNMENT;
+    if (ctx->desc.dtype != DL_BF16 || ctx->desc.head_dim != 128 || !ctx->tmap_encode) return DL_ERR_UNSUPPORTED;
+    if (!ctx->ws.base || B > ctx->ws.max_batch || cap > ctx->ws.cap) return DL_ERR_WORKSPACE;
+    if (B > 2048) return DL_ERR_UNSUPPORTED;
+    DeviceGuard g(ctx->device);
+    // consecutive layers touch different caches and outputs, so layer l may start while layer l-1 drains
+    const bool overlap = l > 0 && k_caches[l] != k_caches[l - 1] && v_caches[l] != v_caches[l - 1];
+    const int32_t st = cuda_status(ctx, launch_attn_decode_fp8(
+        ctx, ql, kl, vl, k_caches[l], v_caches[l], k_scales + (size_t)l * ctx->desc.n_heads,
+        v_scales + (size_t)l * ctx->desc.n_heads, cache_len, keep, B, cap, scale, ol,
+        static_cast<cudaStream_t>(stream), L > 1, overlap, l % kDecodeScratchSets));
+    if (st != DL_OK) return st;
+  }
+  // every layer has appended with the shared decision: the lengths advance once (stream order: after the last layer,
+  // whose grid-dependency wait means all earlier layers are complete too)
+  if (commit) return dl_commit_len(ctx, keep, B, cap, cache_len, stream);
+  return DL_OK;
+}
+
 int32_t dl_decode_keep(dl_ctx* ctx, const dl_predictor* p_txt, const void* x_t, int32_t B, float threshold,
                        float* logit_inout, uint8_t* keep_out, void* stream) {
   if (!ctx || B < 0) return DL_ERR_INVALID_ARG;

@@ -34,6 +34,7 @@ struct F8Args {
   void* out;                                                // bf16 [B][H][128]
   float* partial; int32_t* ticket; DeviceStatus* status;
   int32_t B, H, cap, per_bh, slots, n_stages;
+  int32_t overlap;        // launched with programmatic stream serialisation: may start while its predecessor drains
   float scale_log2;
 };
 
@@ -111,6 +112,9 @@ attn_decode_fp8_kernel(const __grid_constant__ F8Maps maps, const F8Args a) {
   __shared__ int sh_abort;
   volatile int* abort_flag = &sh_abort;
 
+  // Let the next kernel of the stream start as soon as SMs free up (it only matters when that kernel was launched
+  // with programmatic stream serialisation; a no-op otherwise).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) sh_abort = 0;
   if (lane == 0) {
     for (int s = 0; s < NS; ++s) mbar_init(smem_u32(&bars[s]), 1);
@@ -418,6 +422,9 @@ attn_decode_fp8_kernel(const __grid_constant__ F8Maps maps, const F8Args a) {
     }
   }
 
+  // A kernel that was allowed to start early must not finish before its predecessor has: whatever follows in the
+  // stream relies on all earlier layers being done.
+  if (a.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (*abort_flag) {
     if (lane == 0) {
       report_status(a.status, DL_ERR_TIMEOUT, blockIdx.x);
@@ -466,7 +473,7 @@ static int f8_max_chunks(const F8Args& a) { return max(1, min(a.per_bh, a.cap / 
 cudaError_t launch_attn_decode_fp8(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t, void* k_cache,
                                    void* v_cache, const float* k_scale, const float* v_scale, const int32_t* cache_len,
                                    const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                                   cudaStream_t s) {
+                                   cudaStream_t s, bool in_stack, bool overlap_prev, int scratch_set) {
   if (B == 0) return cudaSuccess;
   const dl_model_desc& d = ctx->desc;
   if (d.dtype != DL_BF16 || d.head_dim != 128 || ctx->tmap_encode == nullptr) return cudaErrorInvalidValue;
@@ -474,7 +481,12 @@ cudaError_t launch_attn_decode_fp8(const dl_ctx* ctx, const void* q, const void*
   a.q = q; a.k_t = k_t; a.v_t = v_t;
   a.k_cache = static_cast<uint8_t*>(k_cache); a.v_cache = static_cast<uint8_t*>(v_cache);
   a.k_scale = k_scale; a.v_scale = v_scale; a.cache_len = cache_len; a.keep = keep; a.out = out;
-  a.partial = ctx->ws.dec_partial; a.ticket = ctx->ws.dec_ticket; a.status = ctx->ws.status;
+  // the scratch of split sequences: one of three sets, so that launches in flight together differ (see
+  // launch_attn_decode for why three are enough)
+  const size_t set = (size_t)(scratch_set % kDecodeScratchSets);
+  a.ticket = ctx->ws.dec_ticket + set * (size_t)ctx->ws.max_batch * d.n_heads;
+  a.partial = ctx->ws.dec_partial + set * (size_t)ctx->ws.max_batch * d.n_heads * ctx->ws.dec_slots * (d.head_dim + 2);
+  a.status = ctx->ws.status;
   a.B = B; a.H = d.n_heads; a.cap = cap; a.slots = ctx->ws.dec_slots;
   const long long warps = (long long)ctx->sm_count * kF8Warps * kF8Ctas;
   a.per_bh = (int)max(1LL, warps / ((long long)B * d.n_heads));
@@ -504,9 +516,31 @@ cudaError_t launch_attn_decode_fp8(const dl_ctx* ctx, const void* q, const void*
     attr_set_for = (int)smem;
   }
   const long long max_items = (long long)B * d.n_heads * f8_max_chunks(a);
-  const int grid = (int)max(1LL, min((long long)ctx->sm_count * kF8Ctas, max_items));
-  attn_decode_fp8_kernel<<<grid, kF8Warps * 32, smem, s>>>(maps, a);
-  return cudaGetLastError();
+  // Inside a layer stack a launch takes ONE of the two CTA slots of an SM and may start while its predecessor
+  // drains, so that two layers stream side by side (as the bf16 kernel does); that counts on exactly two CTAs of
+  // this kernel fitting an SM.
+  static int occ_for[64], occ_val[64];
+  if (occ_for[ctx->device & 63] != (int)smem) {
+    int nb = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, attn_decode_fp8_kernel, kF8Warps * 32, smem);
+    if (e != cudaSuccess) return e;
+    occ_val[ctx->device & 63] = nb;
+    occ_for[ctx->device & 63] = (int)smem;
+  }
+  const bool one_slot = in_stack && max_items >= ctx->sm_count && occ_val[ctx->device & 63] == kF8Ctas;
+  a.overlap = (overlap_prev && (one_slot || f8_max_chunks(a) == 1)) ? 1 : 0;
+  const int grid = (int)max(1LL, min((long long)ctx->sm_count * (one_slot ? 1 : kF8Ctas), max_items));
+  if (!a.overlap) {
+    attn_decode_fp8_kernel<<<grid, kF8Warps * 32, smem, s>>>(maps, a);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kF8Warps * 32); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, attn_decode_fp8_kernel, maps, a);
 }
 
 }  // namespace dl

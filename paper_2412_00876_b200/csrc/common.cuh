@@ -158,7 +158,7 @@ cudaError_t launch_quantize_kv_fp8(const dl_ctx* ctx, const void* src, const int
 cudaError_t launch_attn_decode_fp8(const dl_ctx* ctx, const void* q, const void* k_t, const void* v_t, void* k_cache,
                                    void* v_cache, const float* k_scale, const float* v_scale, const int32_t* cache_len,
                                    const uint8_t* keep, int32_t B, int32_t cap, float scale, void* out,
-                                   cudaStream_t s);
+                                   cudaStream_t s, bool in_stack = false, bool overlap_prev = false, int scratch_set = 0);
 
 cudaError_t launch_predictor_simt(const dl_ctx* ctx, const dl_predictor* p, const void* x, int32_t rows,
                                   float* score, cudaStream_t s);

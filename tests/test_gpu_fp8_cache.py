@@ -151,3 +151,47 @@ def test_full_size_launch_on_sampled_heads():
     assert torch.equal(torch.where(untouched, vc, 0), torch.where(untouched, v0, 0))
     assert ctx.device_status()[0] == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("B,H,L,cap", [(32, 32, 4, 512), (3, 4, 5, 320)])
+def test_layer_stack_over_byte_caches_equals_per_layer_calls(B, H, L, cap):
+    """L overlapped launches (one CTA slot per SM each at the large shape, split sequences sharing the scratch sets
+    in rotation at the small one) give bit for bit what separate calls give, every time, and the lengths advance
+    once behind the last layer."""
+    from paper_2412_00876_b200 import binding as dl
+    D = 128
+    g = torch.Generator(device=DEV).manual_seed(5)
+    mk = lambda: (torch.randint(0, 0x7E, (B, H, cap, D), dtype=torch.uint8, device=DEV, generator=g) |
+                  (torch.randint(0, 2, (B, H, cap, D), dtype=torch.uint8, device=DEV, generator=g) << 7))
+    base_k, base_v = [mk() for _ in range(L)], [mk() for _ in range(L)]
+    rng = np.random.default_rng(6)
+    r = lambda *shape: wl.to_torch(wl.round_to_storage(rng.normal(0, 1, shape).astype(np.float32), "bf16"), "bf16", DEV)
+    q, kt, vt = r(L, B, H, D), r(L, B, H, D), r(L, B, H, D)
+    ks = torch.from_numpy(rng.uniform(1 / 96, 1 / 48, (L, H)).astype(np.float32)).to(DEV)
+    vs = torch.from_numpy(rng.uniform(1 / 96, 1 / 48, (L, H)).astype(np.float32)).to(DEV)
+    lens = rng.integers(0, cap, B).astype(np.int32)
+    keep = torch.from_numpy((np.arange(B) % 3 != 0).astype(np.uint8)).to(DEV)
+    ctx = dl.Context(256, H, D, 64, torch.bfloat16, 0, max_batch=B, max_rows=B, cap=cap)
+    scale = 1 / np.sqrt(D)
+    results = []
+    for mode in ("per-layer", "stack", "stack", "stack"):
+        kc, vc = [t.clone() for t in base_k], [t.clone() for t in base_v]
+        ln = torch.from_numpy(lens).to(DEV)
+        out = torch.zeros(L, B, H, D, dtype=torch.bfloat16, device=DEV)
+        if mode == "per-layer":
+            for l in range(L):
+                ctx.sparse_attn_decode_fp8(q[l], kt[l], vt[l], kc[l], vc[l], ks[l], vs[l], ln, keep, scale, out[l])
+            ctx.commit_len(keep, ln, cap)
+        else:
+            ctx.sparse_attn_decode_fp8_layers(q, kt, vt, kc, vc, ks, vs, ln, keep, scale, out, commit=True)
+        torch.cuda.synchronize()
+        results.append((out, kc, vc, ln.cpu().numpy()))
+    ref = results[0]
+    assert np.array_equal(ref[3], lens + (keep.cpu().numpy() != 0) * (lens < cap))
+    for out, kc, vc, ln in results[1:]:
+        assert torch.equal(out.view(torch.int16), ref[0].view(torch.int16))
+        assert np.array_equal(ln, ref[3])
+        for l in range(L):
+            assert torch.equal(kc[l], ref[1][l]) and torch.equal(vc[l], ref[2][l])
+    assert ctx.device_status()[0] == 0
+    ctx.close()
