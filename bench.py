@@ -39,6 +39,8 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-record", action="store_true")
+    ap.add_argument("--no-fp8-extra", action="store_true",
+                    help="skip the extra record of the decode phase over an 8-bit K/V cache (extension, not in the paper)")
     ap.add_argument("--sample-every", type=int, default=64, help="decode steps between timed attention launches")
     ap.add_argument("--micro", default="", choices=["", "decode", "decode_fp8", "decode_fp8_stack", "keep", "select2", "keep2", "predictor", "select", "compact", "compact_layers", "prefill", "nocache"],
                     help="time one stage alone on the config's shapes (small memory; used for ncu captures)")
@@ -332,6 +334,50 @@ def sweep(args):
                           "cache_len_end": cfg.n0 + int(cfg.n_gen * cfg.keep_rate),
                           "decode_attn_us_single_launch": dec["median_us"], "decode_gbs": dec["rate"],
                           "decode_frac_of_hbm_peak": dec["rate"] / hbm, "peaks": src}), flush=True)
+
+
+def fp8_extension_record(runner, cfg):
+    """Extension, NOT in the paper and not part of the metric: the decode phase of the same batch with the K/V
+    caches held as E4M3 bytes (per-layer, per-head scales from the prefill rows' largest magnitude).  The prefill
+    runs as usual, its caches are quantised, then N_OT decode steps run as keep decision + the 8-bit layer stack
+    (lengths advanced behind the last layer).  Returns decode-phase tokens/s and the time per step."""
+    import torch
+    if cfg.dtype != "bf16" or cfg.head_dim != 128:
+        return None
+    need = 2 * cfg.n_layers * cfg.B * cfg.n_heads * cfg.cap * cfg.head_dim * 1.2
+    if torch.cuda.mem_get_info()[0] < need:
+        return {"skipped": "not enough free device memory for the byte caches"}
+    r, ctx, L, B, H = runner, runner.ctx, cfg.n_layers, cfg.B, cfg.n_heads
+    dev = r.dev
+    kc8 = [torch.empty(B, H, r.cap, cfg.head_dim, dtype=torch.uint8, device=dev) for _ in range(L)]
+    vc8 = [torch.empty(B, H, r.cap, cfg.head_dim, dtype=torch.uint8, device=dev) for _ in range(L)]
+    ks = torch.empty(L, H, dtype=torch.float32, device=dev)
+    vs = torch.empty(L, H, dtype=torch.float32, device=dev)
+
+    def one_pass(timed):
+        r.prefill()
+        for l in range(L):
+            ks[l] = r.k_cache[l][:, :, : cfg.n0].abs().amax(dim=(0, 2, 3)).float() * (1.5 / 448.0)
+            vs[l] = r.v_cache[l][:, :, : cfg.n0].abs().amax(dim=(0, 2, 3)).float() * (1.5 / 448.0)
+            ctx.quantize_kv_fp8(r.k_cache[l], r.cache_len, ks[l], kc8[l])
+            ctx.quantize_kv_fp8(r.v_cache[l], r.cache_len, vs[l], vc8[l])
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for t in range(cfg.n_gen):
+            i = t % r.step_pool
+            ctx.decode_keep(r.p_txt, r.x_dec[i], r.logit, r.keep_t)
+            ctx.sparse_attn_decode_fp8_layers(r.q_dec[i], r.k_dec[i], r.v_dec[i], kc8, vc8, ks, vs, r.cache_len,
+                                              r.keep_t, r.scale, r.dec_out, commit=True)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+    one_pass(False)
+    ms = one_pass(True)
+    code, _ = ctx.device_status()
+    return {"note": "extension, not in the paper, not the metric: decode phase only, K/V caches as E4M3 bytes with "
+                    "per-head scales; the metric above keeps the bf16 cache",
+            "decode_tokens_per_s": B * cfg.n_gen / (ms * 1e-3), "ms_per_decode_step": ms / cfg.n_gen,
+            "launches_per_step": 2 + L, "device_status": code}
 
 
 def measured_peaks():
@@ -630,6 +676,10 @@ def main():
         roofline["single_launch_gbs"] = one["rate"]
         roofline["frac_single_launch"] = one["rate"] / peak
 
+    fp8_extra = None
+    if rank == 0 and world == 1 and not args.no_fp8_extra:
+        fp8_extra = fp8_extension_record(runner, cfg)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, cores, sample = oracle_sample(cfg)
@@ -641,7 +691,7 @@ def main():
                 "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
                 "config": config_of(cfg, world), "decode_steps_from_cuda_graphs": use_graphs,
                 "roofline": roofline, "prefill": prefill, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
-                "clocks": clocks}
+                "clocks": clocks, "extension_fp8_kv_cache": fp8_extra}
         print(json.dumps(line), flush=True)
     runner.close()
     if world > 1:
