@@ -7,7 +7,7 @@
 // persistent CTAs over (row tile, column tile) items with the column tiles of one row tile side by side (they
 // share the A tile through L2).
 //   warp 0 : TMA producer      warp 1 : tensor-memory allocation + the MMA-issuing thread
-//   warps 2-5 : epilogue, one TMEM lane quadrant each, one output row per thread
+//   warps 2-9 : epilogue, two warps per TMEM lane quadrant (32-column chunks in turn), one output row per thread
 // Every wait is bounded (pipeline.cuh); an abort leaves DL_ERR_TIMEOUT in the status word.
 #include <algorithm>
 
@@ -16,7 +16,7 @@
 
 namespace dl {
 
-constexpr int kGmStages = 4, kGmBM = 128, kGmBK = 64, kGmMaxBN = 256, kGmThreads = 192;
+constexpr int kGmStages = 4, kGmBM = 128, kGmBK = 64, kGmMaxBN = 256, kGmThreads = 320;
 constexpr int kGmATile = kGmBM * kGmBK * 2, kGmBTile = kGmMaxBN * kGmBK * 2, kGmStageBytes = kGmATile + kGmBTile;
 constexpr size_t kGmSmem = (size_t)kGmStages * kGmStageBytes + 1024 + 256;
 
@@ -46,7 +46,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (tid == 0) {
     sh_abort = 0;
     for (int s = 0; s < kGmStages; ++s) { mbar_init(smem_u32(&full[s]), 1); mbar_init(smem_u32(&empty[s]), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), 8); }
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -108,7 +108,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else {
-    const int quad = warp & 3;
+    // a warp reads the TMEM lanes of quadrant warp % 4; the two warps of a quadrant take the 32-column chunks in turn
+    const int quad = warp & 3, half = (warp - 2) >> 2;
     int j = 0;
     for (int item = blockIdx.x; item < items; item += gridDim.x, ++j) {
       const int mt = item / a.n_tiles, nt = item - mt * a.n_tiles;
@@ -118,11 +119,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * a.bn);
       const int row = mt * kGmBM + quad * 32 + lane;
       const int col0 = nt * a.bn;
-      for (int c = 0; c < a.bn; c += 32) {
+      if (32 * half >= a.bn) {                      // a tile of one chunk: nothing for the second warp of the quadrant
+        if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+        continue;
+      }
+      for (int c = 32 * half; c < a.bn; c += 64) {
         uint32_t r[32];
         tmem_ld32(t_row + c, r);
         tmem_ld_wait();
-        if (c + 32 >= a.bn) {                       // the accumulator is in registers: the next tile may use it
+        if (c + 64 >= a.bn) {                       // this warp's share is in registers: the next tile may use it
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
