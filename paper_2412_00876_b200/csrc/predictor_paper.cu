@@ -94,7 +94,8 @@ __device__ __forceinline__ uint32_t pack_bf162(float lo, float hi) {
 __global__ void __launch_bounds__(128)
 vit_attn_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ n_vis, int n_max,
                 __nv_bfloat16* __restrict__ out, float scale_log2) {
-  __shared__ __align__(16) __nv_bfloat16 sq[kVaRows * kVaStride], sk[kVaRows * kVaStride], sv[kVaRows * kVaStride];
+  // K and V tiles are double-buffered: the copies of the next tile run under the arithmetic of this one
+  __shared__ __align__(16) __nv_bfloat16 sq[kVaRows * kVaStride], skb[2][kVaRows * kVaStride], svb[2][kVaRows * kVaStride];
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * kVaRows;
   const int n = n_vis ? min(max(n_vis[b], 0), n_max) : n_max;
   if (q0 >= n) return;
@@ -110,7 +111,20 @@ vit_attn_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __restrict
       *reinterpret_cast<uint4*>(dst + r * kVaStride + c) = w;
     }
   };
+  // the same tile as asynchronous 16-byte copies (rows past the sequence: zero-filled, from a valid address)
+  auto load_tile_async = [&](__nv_bfloat16* dst, int r0, int col0) {
+    for (int u = tid; u < kVaRows * 8; u += 128) {
+      const int r = u >> 3, c = (u & 7) * 8;
+      const bool ok = r0 + r < n;
+      const __nv_bfloat16* src = qkv + (row_base + (ok ? r0 + r : 0)) * LD + col0 + c;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst + r * kVaStride + c)),
+                   "l"(src), "r"(ok ? 16 : 0) : "memory");
+    }
+  };
   load_tile(sq, q0, h * kPpHeadDim);
+  load_tile_async(skb[0], 0, kPpWidth + h * kPpHeadDim);
+  load_tile_async(svb[0], 0, 2 * kPpWidth + h * kPpHeadDim);
+  asm volatile("cp.async.commit_group;" ::: "memory");
   __syncthreads();
   // this warp's 16 query rows as A fragments of the four 16-dim steps
   uint32_t qa[4][4];
@@ -125,11 +139,16 @@ vit_attn_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __restrict
   for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};      // rows lane/4 and lane/4 + 8 of the warp's 16
 
-  for (int k0 = 0; k0 < n; k0 += kVaRows) {
-    __syncthreads();                                  // the previous tile has been read
-    load_tile(sk, k0, kPpWidth + h * kPpHeadDim);
-    load_tile(sv, k0, 2 * kPpWidth + h * kPpHeadDim);
-    __syncthreads();
+  for (int k0 = 0, it = 0; k0 < n; k0 += kVaRows, ++it) {
+    const __nv_bfloat16* sk = skb[it & 1];
+    const __nv_bfloat16* sv = svb[it & 1];
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();                                  // this tile has landed for everyone; the other buffer has been read
+    if (k0 + kVaRows < n) {
+      load_tile_async(skb[(it + 1) & 1], k0 + kVaRows, kPpWidth + h * kPpHeadDim);
+      load_tile_async(svb[(it + 1) & 1], k0 + kVaRows, 2 * kPpWidth + h * kPpHeadDim);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
     // S = Q K^T for 64 keys: eight blocks of 8 keys
     float s[8][4];
 #pragma unroll
