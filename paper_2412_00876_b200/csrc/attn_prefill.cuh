@@ -154,4 +154,37 @@ constexpr int kAtRegsSmall = 72, kAtRegsSoftmax = 216;
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
+// Host side, shared by the launchers: the tensor maps of one call and the kernel's arguments.
+inline cudaError_t at_prepare(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max, float scale, void* out,
+                              AtMaps* maps, AtArgs* a, long long* items) {
+  const dl_model_desc& d = ctx->desc;
+  const long long rows = (long long)B * d.n_heads * cap;
+  if (rows >= (1LL << 31)) return cudaErrorInvalidValue;
+  const uint64_t dims[2] = {128ull, (uint64_t)rows};
+  const uint64_t strides[1] = {256ull};
+  // out [B][n_max][H][128]: 32 rows x 32 columns of one head per store
+  const uint64_t dims_o[4] = {128ull, (uint64_t)d.n_heads, (uint64_t)n_max, (uint64_t)B};
+  const uint64_t strides_o[3] = {256ull, 256ull * d.n_heads, 256ull * d.n_heads * n_max};
+  const uint32_t box_o[4] = {32u, 1u, 32u, 1u};
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t box[2] = {64u, 128u >> i};
+    if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps->q[i]), q, 2, dims, strides, box) ||
+        !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps->k[i]), k_cache, 2, dims, strides, box) ||
+        !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps->v[i]), v_cache, 2, dims, strides, box))
+      return cudaErrorInvalidValue;
+  }
+  if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps->o), out, 4, dims_o, strides_o, box_o,
+                       CU_TENSOR_MAP_SWIZZLE_64B))
+    return cudaErrorInvalidValue;
+  a->cache_len = cache_len; a->out = static_cast<__nv_bfloat16*>(out); a->status = ctx->ws.base ? ctx->ws.status : nullptr;
+  a->q = static_cast<const __nv_bfloat16*>(q); a->k = static_cast<const __nv_bfloat16*>(k_cache);
+  a->v = static_cast<const __nv_bfloat16*>(v_cache);
+  a->item_rows = 2 * kAtBM;
+  a->B = B; a->H = d.n_heads; a->cap = cap; a->n_max = n_max; a->q_pairs = (n_max + a->item_rows - 1) / a->item_rows;
+  a->scale_log2 = scale * 1.4426950408889634f;
+  *items = (long long)B * d.n_heads * a->q_pairs;
+  return *items >= (1LL << 31) ? cudaErrorInvalidValue : cudaSuccess;
+}
+
 }  // namespace dl

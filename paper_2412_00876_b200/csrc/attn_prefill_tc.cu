@@ -414,41 +414,17 @@ cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cac
                                    const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max, float scale,
                                    void* out, cudaStream_t s) {
   if (B == 0 || n_max == 0) return cudaSuccess;
-  const dl_model_desc& d = ctx->desc;
-  const long long rows = (long long)B * d.n_heads * cap;
-  if (rows >= (1LL << 31)) return cudaErrorInvalidValue;
   AtMaps maps;
-  const uint64_t dims[2] = {128ull, (uint64_t)rows};
-  const uint64_t strides[1] = {256ull};
-  // out [B][n_max][H][128]: 32 rows x 32 columns of one head per store
-  const uint64_t dims_o[4] = {128ull, (uint64_t)d.n_heads, (uint64_t)n_max, (uint64_t)B};
-  const uint64_t strides_o[3] = {256ull, 256ull * d.n_heads, 256ull * d.n_heads * n_max};
-  const uint32_t box_o[4] = {32u, 1u, 32u, 1u};
-  for (int i = 0; i < 4; ++i) {
-    const uint32_t box[2] = {64u, 128u >> i};
-    if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.q[i]), q, 2, dims, strides, box) ||
-        !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.k[i]), k_cache, 2, dims, strides, box) ||
-        !encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.v[i]), v_cache, 2, dims, strides, box))
-      return cudaErrorInvalidValue;
-  }
-  if (!encode_bf16_map(ctx->tmap_encode, reinterpret_cast<CUtensorMap*>(maps.o), out, 4, dims_o, strides_o, box_o,
-                       CU_TENSOR_MAP_SWIZZLE_64B))
-    return cudaErrorInvalidValue;
   AtArgs a;
-  a.cache_len = cache_len; a.out = static_cast<__nv_bfloat16*>(out); a.status = ctx->ws.base ? ctx->ws.status : nullptr;
-  a.q = static_cast<const __nv_bfloat16*>(q); a.k = static_cast<const __nv_bfloat16*>(k_cache);
-  a.v = static_cast<const __nv_bfloat16*>(v_cache);
-  a.item_rows = 2 * kAtBM;
-  a.B = B; a.H = d.n_heads; a.cap = cap; a.n_max = n_max; a.q_pairs = (n_max + a.item_rows - 1) / a.item_rows;
-  a.scale_log2 = scale * 1.4426950408889634f;
+  long long items = 0;
+  cudaError_t e = at_prepare(ctx, q, k_cache, v_cache, cache_len, B, cap, n_max, scale, out, &maps, &a, &items);
+  if (e != cudaSuccess) return e;
   static int attr_set[64];
   if (!attr_set[ctx->device & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
+    e = cudaFuncSetAttribute(attn_prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem);
     if (e != cudaSuccess) return e;
     attr_set[ctx->device & 63] = 1;
   }
-  const long long items = (long long)B * d.n_heads * a.q_pairs;
-  if (items >= (1LL << 31)) return cudaErrorInvalidValue;
   const int grid = (int)std::min<long long>(items, (long long)ctx->sm_count);
   attn_prefill_tc_kernel<<<grid, kAtThreads, kAtSmem, s>>>(maps, a);
   return cudaGetLastError();
