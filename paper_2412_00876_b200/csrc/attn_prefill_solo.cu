@@ -171,8 +171,8 @@ attn_prefill_solo_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       ++issued[1 + is_v];
     };
     AtWalker W(a);
-    AtItem I, In;
-    AtLane L, Ln;
+    AtItem I, In, In2;                                                 // this item, the next, the one after
+    AtLane L, Ln, Ln2;
     auto next_own = [&](AtItem& It, AtLane& Lt) {                      // the next item in which this lane has a tile
       while (W.next(It, kAtTopRows)) {
         Lt = at_lane(It, x);
@@ -184,7 +184,10 @@ attn_prefill_solo_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       const unsigned char (*mp)[128] = issue_q ? maps.q : issue_k ? maps.k : maps.v;
       for (int i = 0; i < 4; ++i) tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(mp[i]));
     }
+    // The walk runs two items ahead: the step to item i + 2 is taken while item i waits for its last P V (idle time;
+    // at the top of the loop it would sit in front of the first softmax, 1 k cycles of cold code per item).
     bool have = next_own(I, L);
+    bool have_next = have && next_own(In, Ln);
     if (have) {
       if (issue_q) load_q(I, L);
       if (issue_k) load_kv(I, L, 0, 0);
@@ -192,7 +195,6 @@ attn_prefill_solo_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
     }
     int g0 = 0;
     while (have) {
-      const bool have_next = next_own(In, Ln);
       const int grow = L.q0 + row;                                     // row within the sequence
       const int r0 = L.q0 + quad * 32;                                 // this warp's first row
       float m_used = -INFINITY, l_run = 0.f;
@@ -261,6 +263,7 @@ attn_prefill_solo_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       // ---- epilogue: O / l -> bf16 -> out[b][row][h][:], 32 columns at a time, two blocks per round through this
       // warp's staging (16-byte units XOR-swizzled by row pair: the 64-byte swizzle of the tensor map)
       const int gl = g0 + n_sub - 1;
+      const bool have_next2 = have_next && next_own(In2, Ln2);
       mbar_wait_spin(bar(x, PV_DONE), (uint32_t)gl & 1u, abort_flag);   // MMAs complete in order: all of O is in
       if (issue_v && have_next && !*abort_flag) load_kv(In, Ln, 0, 1);   // and the V slot is free
       __syncwarp();
@@ -270,60 +273,55 @@ attn_prefill_solo_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
       const bool whole = rows_here >= 32;                              // warp-uniform
       __nv_bfloat16* otile = a.out + (((size_t)I.b * a.n_max + r0) * a.H + I.h) * 128;
 #pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {                   // not unrolled: once per item, short code counts for more
-        uint32_t o[32];
-        tmem_ld32(o_addr + cc * 32, o);
+      for (int rd = 0; rd < 2; ++rd) {                   // not unrolled: once per item, short code counts for more
+        uint32_t o[64];
+        tmem_ld64(o_addr + rd * 64, o);
+        // the stores that read this staging last (the previous round, or the previous item) must have read it
+        if (lane == 0) bulk_wait_read<0>();
         tmem_ld_wait();
-        if (cc == 3) {                                   // all of O is in registers: the next item may overwrite it
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar(x, O_FREE));
-        }
-        char* sb = so + (cc & 1) * 2048;
-        if ((cc & 1) == 0) {
-          // the stores that read this staging last (the previous round, or the previous item) must have read it
-          if (lane == 0) bulk_wait_read<0>();
-          __syncwarp();
-        }
+        if (rd == 1) tc_fence_before();                  // all of O is in registers: the next item may overwrite it
+        __syncwarp();
+        if (rd == 1 && lane == 0) mbar_arrive(bar(x, O_FREE));
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          uint4 w;
-          w.x = cvt_bf16x2(__uint_as_float(o[8 * u]) * inv, __uint_as_float(o[8 * u + 1]) * inv);
-          w.y = cvt_bf16x2(__uint_as_float(o[8 * u + 2]) * inv, __uint_as_float(o[8 * u + 3]) * inv);
-          w.z = cvt_bf16x2(__uint_as_float(o[8 * u + 4]) * inv, __uint_as_float(o[8 * u + 5]) * inv);
-          w.w = cvt_bf16x2(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
-          *reinterpret_cast<uint4*>(sb + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
-        }
-        if (cc & 1) {
-          if (whole) {
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) {
-              tma_store_4d(mo, smem_u32(so), (cc - 1) * 32, I.h, r0, I.b);
-              tma_store_4d(mo, smem_u32(so + 2048), cc * 32, I.h, r0, I.b);
-              bulk_commit();
-            }
-          } else {
-            __syncwarp();
+        for (int blk = 0; blk < 2; ++blk) {
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-#pragma unroll
-              for (int it = 0; it < 4; ++it) {
-                const int r = it * 8 + (lane >> 2), u = lane & 3;
-                const uint4 w = *reinterpret_cast<const uint4*>(so + half * 2048 + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
-                if (r < rows_here && DL_IN_BOUNDS(a.status, KID_PREFILL_TC, (((size_t)I.b * a.n_max + r0 + r) * a.H + I.h) * 128 + 127,
-                                                  (size_t)a.B * a.n_max * a.H * 128))
-                  *reinterpret_cast<uint4*>(otile + (size_t)r * a.H * 128 + (cc - 1 + half) * 32 + u * 8) = w;
-              }
-            }
-            __syncwarp();                                // the next round overwrites what these loads read
+          for (int u = 0; u < 4; ++u) {
+            const uint32_t* ob = o + 32 * blk + 8 * u;
+            uint4 w;
+            w.x = cvt_bf16x2(__uint_as_float(ob[0]) * inv, __uint_as_float(ob[1]) * inv);
+            w.y = cvt_bf16x2(__uint_as_float(ob[2]) * inv, __uint_as_float(ob[3]) * inv);
+            w.z = cvt_bf16x2(__uint_as_float(ob[4]) * inv, __uint_as_float(ob[5]) * inv);
+            w.w = cvt_bf16x2(__uint_as_float(ob[6]) * inv, __uint_as_float(ob[7]) * inv);
+            *reinterpret_cast<uint4*>(so + blk * 2048 + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) = w;
           }
+        }
+        if (whole) {
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_4d(mo, smem_u32(so), rd * 64, I.h, r0, I.b);
+            tma_store_4d(mo, smem_u32(so + 2048), rd * 64 + 32, I.h, r0, I.b);
+            bulk_commit();
+          }
+        } else {
+          __syncwarp();
+#pragma unroll
+          for (int blk = 0; blk < 2; ++blk) {
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+              const int r = it * 8 + (lane >> 2), u = lane & 3;
+              const uint4 w = *reinterpret_cast<const uint4*>(so + blk * 2048 + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
+              if (r < rows_here && DL_IN_BOUNDS(a.status, KID_PREFILL_TC, (((size_t)I.b * a.n_max + r0 + r) * a.H + I.h) * 128 + 127,
+                                                (size_t)a.B * a.n_max * a.H * 128))
+                *reinterpret_cast<uint4*>(otile + (size_t)r * a.H * 128 + (2 * rd + blk) * 32 + u * 8) = w;
+            }
+          }
+          __syncwarp();                                  // the next round overwrites what these loads read
         }
       }
       g0 += n_sub;
-      I = In;
-      L = Ln;
-      have = have_next;
+      I = In; L = Ln; have = have_next;
+      In = In2; Ln = Ln2; have_next = have_next2;
     }
     if (lane == 0) bulk_wait_read<0>();                  // staged data must be read before shared memory goes
     if (lane == 0 && quad < 3 && *abort_flag) {
