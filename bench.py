@@ -48,7 +48,7 @@ def parse():
     ap.add_argument("--micro-len", type=int, default=0, help="cache length per sequence in --micro decode (0: end state)")
     ap.add_argument("--decode-chunk", type=int, default=0, help="--micro decode: rows per work item (0: library's choice)")
     ap.add_argument("--prefill-impl", type=int, default=0,
-                    help="--micro prefill/nocache: 0 library's choice, 1 CUDA-core kernel, 2 / 3 tensor-core kernel with shared / per-lane K/V")
+                    help="--micro prefill/nocache: 0 library's choice, 1 CUDA-core kernel, 2 tensor-core kernel")
     ap.add_argument("--compact-impl", type=int, default=0,
                     help="--micro compact: 0 library's choice, 1 register-staged copy, 2 bulk copy by token tiles, "
                          "3 bulk copy by even row ranges")

@@ -53,8 +53,7 @@ enum {
 /* Implementation selectors for dl_set_option. */
 enum {
   DL_OPT_PREDICTOR_IMPL = 1,    /* 0 auto, 1 CUDA-core kernel, 2 tcgen05 tensor-core kernel (bf16) */
-  DL_OPT_PREFILL_ATTN_IMPL = 2, /* 0 auto, 1 CUDA-core kernel; tcgen05 tensor-core kernels (bf16, D=128): 2 K/V ring shared by
-                                   a pair of query tiles, 3 K/V fetched per query tile (what auto picks) */
+  DL_OPT_PREFILL_ATTN_IMPL = 2, /* 0 auto, 1 CUDA-core kernel, 2 tcgen05 tensor-core kernel (bf16, D=128) */
   DL_OPT_DECODE_CHUNK = 3,      /* cache rows per decode work item (0 = chosen by the library) */
   DL_OPT_DECODE_IMPL = 4,       /* 0 auto, 1 CUDA-core kernel, 2 tensor-core (mma.sync) kernel (bf16, D=128) */
   DL_OPT_COMPACT_IMPL = 5       /* 0 auto, 1 register-staged copy kernel, 2 bulk-copy (TMA) kernel over even ranges of kept

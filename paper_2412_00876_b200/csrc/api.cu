@@ -165,7 +165,7 @@ int32_t dl_set_option(dl_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx || value < 0) return DL_ERR_INVALID_ARG;
   switch (option) {
     case DL_OPT_PREDICTOR_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.predictor_impl = value; break;
-    case DL_OPT_PREFILL_ATTN_IMPL: if (value > 3) return DL_ERR_INVALID_ARG; ctx->opt.prefill_attn_impl = value; break;
+    case DL_OPT_PREFILL_ATTN_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.prefill_attn_impl = value; break;
     case DL_OPT_DECODE_CHUNK: ctx->opt.decode_chunk = value; break;
     case DL_OPT_DECODE_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.decode_impl = value; break;
     case DL_OPT_COMPACT_IMPL: if (value > 2) return DL_ERR_INVALID_ARG; ctx->opt.compact_impl = value; break;
@@ -370,11 +370,9 @@ int32_t dl_sparse_attn_prefill(dl_ctx* ctx, const void* q, const void* k_cache, 
   DeviceGuard g(ctx->device);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int impl = ctx->opt.prefill_attn_impl;
-  if (impl == 0) impl = attn_prefill_tc_supported(ctx) ? 3 : 1;
+  if (impl == 0) impl = attn_prefill_tc_supported(ctx) ? 2 : 1;
   if (impl >= 2) {
     if (!attn_prefill_tc_supported(ctx)) return DL_ERR_UNSUPPORTED;
-    if (impl == 3)
-      return cuda_status(ctx, launch_attn_prefill_solo(ctx, q, k_cache, v_cache, cache_len, B, cap, n_max, scale, out, s));
     return cuda_status(ctx, launch_attn_prefill_tc(ctx, q, k_cache, v_cache, cache_len, B, cap, n_max, scale, out, s));
   }
   return cuda_status(ctx, launch_attn_prefill_simt(ctx, q, k_cache, v_cache, cache_len, B, cap, n_max, scale, out, s));

@@ -7,10 +7,9 @@
 
 namespace dl {
 
-constexpr int kAtBM = 128, kAtBN = 128, kAtThreads = 384, kAtRing = 3;
+constexpr int kAtBM = 128, kAtBN = 128, kAtThreads = 384;
 constexpr int kAtTile = 2 * 128 * 128;                // 32 KB: two [128 rows][64 dims] halves
-constexpr int kAtOffRing = 4 * kAtTile;               // Q: [lane][slot] tiles first
-constexpr int kAtOffBar = kAtOffRing + kAtRing * kAtTile;
+constexpr int kAtOffBar = 7 * kAtTile;                // seven tiles (see attn_prefill_tc.cu), then the barriers
 constexpr size_t kAtSmem = kAtOffBar + 512;           // 229888 bytes: one CTA per SM
 constexpr uint32_t kAtColO = 0, kAtColS = 128, kAtLaneCols = 256;   // tensor-memory columns of one lane: O | S
 constexpr float kRescaleStep = 8.0f;                  // log2 units by which the maximum may lag

@@ -85,40 +85,42 @@ __device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t* r) {
       : "r"(taddr) : "memory");
 }
 
-// Softmax of one 128 x 128 score tile, one query row per thread, in two halves of 64 columns: P = 2^(S * scale_log2
-// - m_used) goes, as bf16 pairs, over the first 64 columns of the score buffer (half by half: the scores it
-// overwrites are in registers by then) and the row sum is added to l_run.  The maximum in use lags: a half whose
+// Softmax of one 128 x 128 score tile, one query row per thread, in four steps of 32 columns: P = 2^(S * scale_log2
+// - m_used) goes, as bf16 pairs, over the first 64 columns of the score buffer (step by step: the scores it
+// overwrites are in registers by then) and the row sum is added to l_run.  The maximum in use lags: a step whose
 // own maximum is more than 2^8 above it raises it first (rescaling what the row holds so far, see at_rescale_row),
-// so that no exponential exceeds 2^8; a row's first half sets it.  Per half: mask (only where the half reaches
+// so that no exponential exceeds 2^8; a row's first step sets it.  Per step: mask (only where the chunk reaches
 // past the warp's first row), maximum, all multiply-adds, then the registers of the raw scores take the next
-// half's load while the exponentials run (NPOLY of every four pairs as a cubic on the FMA pipe, the rest on the
+// chunk's load while the exponentials run (NPOLY of every four pairs as a cubic on the FMA pipe, the rest on the
 // special-function unit), row sums, packing, store.
-// The loop over the halves is NOT unrolled: a warp alone on its scheduler is bound by instruction fetch once the
-// body of a tile outgrows the scheduler's instruction cache, which the four-chunk unrolled form did.
-//   n_ch: 32-column chunks that some row of the warp may see (halves beyond get P = 0); column c is visible to this
+// The loop is NOT unrolled, and its body is kept small: a warp is bound by instruction fetch once the body of a
+// tile outgrows its scheduler's instruction cache, which it shares with the other lane's warp of the same
+// quadrant.  Fully unrolled (4 chunks) the pass cost 15 % of the kernel's time more than in two rolled halves of 64
+// columns, and those 3 % more than this form on short contexts.
+//   n_ch: 32-column chunks that some row of the warp may see (chunks beyond get P = 0); column c is visible to this
 //   row iff c <= vis; owned: the row belongs to this tile; o_valid: the item has accumulated into O already.
 template <int NPOLY>
-__device__ __forceinline__ void at_softmax_halves(uint32_t s_addr, uint32_t o_addr, int n_ch, int vis, int c0_minus_r0,
+__device__ __forceinline__ void at_softmax_chunks(uint32_t s_addr, uint32_t o_addr, int n_ch, int vis, int c0_minus_r0,
                                                   bool owned, int o_valid, float scale_log2, float& m_used, float& l_run) {
-  const int n_half = min(2, (n_ch + 1) >> 1);
+  const int n_q = max(min(4, n_ch), 0);
   const uint64_t sc2 = pack2(scale_log2, scale_log2);
-  uint32_t buf[64];
+  uint32_t buf[32];
   uint64_t l2[4] = {0ull, 0ull, 0ull, 0ull};
-  if (n_half > 0) {
-    tmem_ld64(s_addr, buf);
+  if (n_q > 0) {
+    tmem_ld32(s_addr, buf);
     tmem_ld_wait();
   }
 #pragma unroll 1
-  for (int hf = 0; hf < n_half; ++hf) {
-    if (c0_minus_r0 + 64 * hf + 63 > 0) {                        // the half reaches past the warp's first row
-      const int v = vis - 64 * hf;
+  for (int q = 0; q < n_q; ++q) {
+    if (c0_minus_r0 + 32 * q + 31 > 0) {                         // the chunk reaches past the warp's first row
+      const int v = vis - 32 * q;
 #pragma unroll
-      for (int c = 0; c < 64; ++c)
+      for (int c = 0; c < 32; ++c)
         if (c > v) buf[c] = 0xFF800000u;                         // -inf
     }
     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-    for (int c = 0; c < 64; c += 8) {
+    for (int c = 0; c < 32; c += 8) {
 #pragma unroll
       for (int w = 0; w < 4; ++w)
         mx4[w] = fmax3(mx4[w], __uint_as_float(buf[c + 2 * w]), __uint_as_float(buf[c + 2 * w + 1]));
@@ -132,17 +134,17 @@ __device__ __forceinline__ void at_softmax_halves(uint32_t s_addr, uint32_t o_ad
       const uint64_t corr2 = pack2(corr, corr);
 #pragma unroll
       for (int i = 0; i < 4; ++i) l2[i] = fmul2(l2[i], corr2);
-      at_rescale_row(o_addr, s_addr, 2 * hf, corr, o_valid);
+      at_rescale_row(o_addr, s_addr, q, corr, o_valid);
     }
     const uint64_t nm2 = pack2(-m_used, -m_used);
-    uint64_t t[32];
+    uint64_t t[16];
 #pragma unroll
-    for (int c = 0; c < 32; ++c)
+    for (int c = 0; c < 16; ++c)
       t[c] = ffma2(pack2(__uint_as_float(buf[2 * c]), __uint_as_float(buf[2 * c + 1])), sc2, nm2);
-    if (hf + 1 < n_half) tmem_ld64(s_addr + 64 * (hf + 1), buf); // the raw scores are used up: next half into their registers
-    uint32_t pk[32];
+    if (q + 1 < n_q) tmem_ld32(s_addr + 32 * (q + 1), buf);      // the raw scores are used up: next chunk into their registers
+    uint32_t pk[16];
 #pragma unroll
-    for (int c = 0; c < 32; ++c) {
+    for (int c = 0; c < 16; ++c) {
       float e0, e1;
       if ((c & 3) < NPOLY) {
         poly_exp2_x2(t[c], e0, e1);
@@ -154,15 +156,15 @@ __device__ __forceinline__ void at_softmax_halves(uint32_t s_addr, uint32_t o_ad
       l2[c & 3] = fadd2(l2[c & 3], pack2(e0, e1));
       pk[c] = cvt_bf16x2(e0, e1);
     }
-    tmem_st32(s_addr + 32 * hf, pk);
+    tmem_st16(s_addr + 16 * q, pk);
     tmem_ld_wait();
   }
-  if (n_half < 2) {
-    uint32_t z[32];
+  if (n_q < 4) {
+    uint32_t z[16];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) z[i] = 0u;
+    for (int i = 0; i < 16; ++i) z[i] = 0u;
 #pragma unroll 1
-    for (int hf = max(n_half, 0); hf < 2; ++hf) tmem_st32(s_addr + 32 * hf, z);
+    for (int q = n_q; q < 4; ++q) tmem_st16(s_addr + 16 * q, z);
   }
   float la, lb;
   unpack2(fadd2(fadd2(l2[0], l2[1]), fadd2(l2[2], l2[3])), la, lb);

@@ -179,9 +179,6 @@ cudaError_t launch_attn_prefill_simt(const dl_ctx* ctx, const void* q, const voi
 cudaError_t launch_attn_prefill_tc(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                    const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max,
                                    float scale, void* out, cudaStream_t s);
-cudaError_t launch_attn_prefill_solo(dl_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
-                                     const int32_t* cache_len, int32_t B, int32_t cap, int32_t n_max,
-                                     float scale, void* out, cudaStream_t s);
 bool attn_prefill_tc_supported(const dl_ctx* ctx);
 
 int64_t predictor_paper_scratch_bytes(int64_t rows);

@@ -383,7 +383,7 @@ def _prefill_case(dtype, H, D, lens, amp=1.0):
         q, k = q * amp, k * amp
     scale = 1 / np.sqrt(D)
     n_max = max(lens)
-    for impl in (1, 2, 3):                       # CUDA cores; tensor cores, K/V ring shared by the lanes / per lane
+    for impl in (1, 2):                          # CUDA cores; tensor cores
         ctx = _ctx(dtype, H, D, B=B, cap=cap)
         ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, impl)
         out = torch.full((B, n_max, H, D), 7.0, dtype=wl.torch_dtype(dtype), device=DEV)
@@ -446,7 +446,7 @@ def test_prefill_attention_large_grid_is_reproducible():
     ln = torch.full((B,), n, dtype=torch.int32, device=DEV)
     scale = 1 / np.sqrt(D)
     outs = {}
-    for impl in (2, 3, 1):
+    for impl in (2, 1):
         ctx = _ctx("bf16", H, D, B=B, cap=cap)
         ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, impl)
         first = None
@@ -460,6 +460,6 @@ def test_prefill_attention_large_grid_is_reproducible():
                 assert torch.equal(first.view(torch.int16), out.view(torch.int16)), f"run {rep} differs"
         outs[impl] = wl.from_torch(first)
         assert ctx.device_status()[0] == 0
-    for impl in (2, 3):
+    for impl in (2,):
         mx, rl = pc.att_errors(outs[impl], outs[1])
         assert mx <= pc.ATT_MAXABS and rl <= pc.ATT_RELL2, (impl, mx, rl)
