@@ -116,14 +116,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtMaps maps, const AtArgs a) {
           else mbar_wait_spin(bar(x, Q_FULL), (uint32_t)n_item & 1u, abort_flag);
           if (has_qk) mbar_wait_spin(bar(x, K_FULL), (uint32_t)(g + 1) & 1u, abort_flag);
           if (u == 0) mbar_wait_spin(bar(x, O_FREE), ((uint32_t)n_item & 1u) ^ 1u, abort_flag);   // previous item's O has been read
-          if (has_pv) {
-            // polled without suspending: the wake-up of a suspended wait costs this thread ~600 cycles per tile
-            const uint32_t pb = bar(x, P_FULL), ph = (uint32_t)g & 1u;
-            int spins = 0;
-            while (!mbar_test(pb, ph)) {
-              if ((++spins & 1023) == 0 && (*abort_flag || spins > (kSpinLimitBusy << 4))) { *abort_flag = 1; break; }
-            }
-          }
+          if (has_pv) mbar_wait_spin(bar(x, P_FULL), (uint32_t)g & 1u, abort_flag);
           tc_fence_after();
           if (has_pv) {
             uint64_t vd = v_desc0;
