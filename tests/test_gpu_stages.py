@@ -429,6 +429,39 @@ def test_prefill_attention_top_rows_of_a_sequence():
     _prefill_case("bf16", 1, 128, [144, 133, 769, 3])
 
 
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_prefill_attention_random_ragged_batches(seed):
+    """Many sequences of random lengths in one call (empty ones, lengths that leave a lane without a tile, top tiles of
+    1..16 rows, several waves of items per CTA): the tensor-core kernel against the CUDA-core one, which the oracle
+    checks in the cases above.  Rows past a sequence's length must stay untouched."""
+    from paper_2412_00876_b200 import binding as dl
+    rng = np.random.default_rng(100 + seed)
+    B, H, D = 40, 8, 128
+    lens = [int(v) for v in rng.integers(0, 900, B)]
+    lens[3], lens[7], lens[11] = 0, 16, 128 + 16
+    cap = (max(lens) + 63) // 64 * 64
+    n_max = max(lens)
+    cfg = wl.CONFIGS[5]
+    mk = lambda s: wl.device_normal(cfg, s, (B, H, cap, D), DEV, sub=seed)
+    q, k, v = mk(wl.S_Q), mk(wl.S_K), mk(wl.S_V)
+    ln = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    outs = {}
+    for impl in (2, 1):
+        ctx = _ctx("bf16", H, D, B=B, cap=cap)
+        ctx.set_option(dl.DL_OPT_PREFILL_ATTN_IMPL, impl)
+        out = torch.full((B, n_max, H, D), 7.0, dtype=torch.bfloat16, device=DEV)
+        ctx.sparse_attn_prefill(q, k, v, ln, n_max, 1 / np.sqrt(D), out)
+        torch.cuda.synchronize()
+        assert ctx.device_status()[0] == 0
+        outs[impl] = wl.from_torch(out)
+    for b in range(B):
+        n = lens[b]
+        assert np.all(outs[2][b, n:] == 7.0), b
+        if n:
+            mx, rl = pc.att_errors(outs[2][b, :n], outs[1][b, :n])
+            assert mx <= pc.ATT_MAXABS and rl <= pc.ATT_RELL2, (b, n, mx, rl)
+
+
 def test_prefill_attention_large_scores():
     """Scores whose row maximum keeps growing by far more than 2^8 from one key tile to the next: the
     tensor-core kernel has to rescale its accumulator and redo tiles (its rare path)."""
